@@ -1,0 +1,277 @@
+"""Float64 CPU oracle for the LM-head log-probability + GRPO policy-loss path.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition that the
+CUDA library is checked against.  Nothing in the product path may import it;
+it imports nothing from the product.  Every function works on float64 numpy
+arrays (bf16 inputs are widened exactly by the caller) and follows the
+definitions in the order the paper states them; the only library primitive
+used as a step is a dense matrix product.
+
+Notation (paper section 2.2 and 3.1): T token rows, d hidden size, V vocabulary
+size; h_t the hidden state whose next-token distribution scores the sampled
+token y_t; z_t = W h_t the logits; pi_theta(.|s_t) = softmax(z_t).
+
+Readings of the paper that this oracle fixes (the paper prints no formula or
+leaves a choice open for each of them):
+  * GRPO "group-based normalization" (section 4.2): A_i = (r_i - mean_g) /
+    (std_g + eps_std) with the sample standard deviation (ddof=1) by default.
+  * PPO clipped surrogate (section 3.1): the standard pessimistic form
+    min(r*A, clip(r, 1-eps_low, 1+eps_high)*A).  The form as literally printed,
+    min(r, clip(r))*A, is available with literal_clip=True for a test that
+    documents the difference; the two agree for A >= 0.
+  * KL-to-reference (section 2.2 "Regularization", section 3.1 Omega): the
+    sampled-token k3 estimator exp(delta) - delta - 1, delta = ref_logp - logp.
+  * Eq. 6 is maximised; the loss returned here is its negative, to be minimised.
+  * Entropy bonus (section 2.2): natural-log entropy of the full next-token
+    distribution, entering the loss as  - ent_coef * H.
+  * Token aggregation: weights w_t = m_t / sum(m) (token mean) unless the caller
+    passes token_weight.
+
+Parity pins: every function here is pinned by tests/test_oracle_pins.py against
+brute force, closed forms, finite differences and library second opinions.
+What cannot be pinned from the paper is WHICH estimator / aggregation the
+authors' code uses (the three readings above): parity unpinned with respect to
+the authors' repository, pinned with respect to the readings stated here.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------- #
+# Algorithm 1, "compute estimating advantages" step; section 3.2.2 advantage
+# estimation stage; section 4.2 "GRPO's group-based normalization".
+# --------------------------------------------------------------------------- #
+def grpo_advantages(rewards, group_size, ddof=1, eps_std=1e-6):
+    """Per-response GRPO advantages.
+
+    rewards: [B] one scalar per trajectory (section 3.2.2 scoring stage), the
+    K = group_size responses of one prompt stored consecutively.
+    Returns adv[B] with adv_i = (r_i - mean_g) / (std_g + eps_std).
+    A group whose rewards are all equal gets advantage exactly 0.
+    """
+    r = np.asarray(rewards, dtype=np.float64)
+    B = r.shape[0]
+    if group_size < 2 or B % group_size != 0:
+        raise ValueError("group_size must be >= 2 and divide the number of responses")
+    adv = np.zeros(B, dtype=np.float64)
+    for g in range(B // group_size):
+        grp = r[g * group_size:(g + 1) * group_size]
+        mu = grp.sum() / group_size
+        var = ((grp - mu) ** 2).sum() / (group_size - ddof)
+        sigma = np.sqrt(var)
+        if np.all(grp == grp[0]):
+            adv[g * group_size:(g + 1) * group_size] = 0.0
+        else:
+            adv[g * group_size:(g + 1) * group_size] = (grp - mu) / (sigma + eps_std)
+    return adv
+
+
+def broadcast_to_tokens(adv_seq, seq_offsets, T):
+    """Outcome supervision: every token of response i carries A_i
+    (Algorithm 1: one advantage per time step from one reward per trajectory)."""
+    adv_tok = np.zeros(T, dtype=np.float64)
+    for i in range(len(adv_seq)):
+        adv_tok[seq_offsets[i]:seq_offsets[i + 1]] = adv_seq[i]
+    return adv_tok
+
+
+# --------------------------------------------------------------------------- #
+# Section 2.2: the policy is the next-token distribution over the vocabulary.
+# --------------------------------------------------------------------------- #
+def logits(H, W):
+    """z[t, j] = sum_k H[t, k] * W[j, k]."""
+    H = np.asarray(H, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    return H @ W.T
+
+
+def log_softmax_stats(Z):
+    """From logits Z[T, V]: lse[T], log-probabilities LP[T, V], entropy[T].
+
+    lse_t = log sum_j exp(z_tj) (computed with the usual max shift),
+    LP_tj = z_tj - lse_t,  Ent_t = - sum_j p_tj * LP_tj with p = exp(LP)
+    (section 2.2 "Regularization": entropy of pi_theta(.|s_t)).
+    """
+    M = Z.max(axis=1, keepdims=True)
+    lse = M[:, 0] + np.log(np.exp(Z - M).sum(axis=1))
+    LP = Z - lse[:, None]
+    P = np.exp(LP)
+    ent = -(P * LP).sum(axis=1)
+    return lse, LP, ent
+
+
+def token_logprobs(H, W, tokens, mask=None):
+    """log pi_theta(y_t | s_t), entropy and lse per row; masked rows give 0.
+
+    Section 2.2 "Adaptation for Off-Policy": the log-probability of the sampled
+    token is what enters the importance ratio.
+    """
+    T = H.shape[0]
+    tokens = np.asarray(tokens)
+    m = np.ones(T, dtype=bool) if mask is None else np.asarray(mask).astype(bool)
+    logp = np.zeros(T)
+    ent = np.zeros(T)
+    lse = np.zeros(T)
+    rows = np.nonzero(m)[0]
+    if rows.size:
+        Z = logits(np.asarray(H, dtype=np.float64)[rows], W)
+        lse_r, LP, ent_r = log_softmax_stats(Z)
+        logp[rows] = LP[np.arange(rows.size), tokens[rows]]
+        ent[rows] = ent_r
+        lse[rows] = lse_r
+    return logp, ent, lse
+
+
+# --------------------------------------------------------------------------- #
+# Eq. 6 with L^PG = PPO clipped surrogate (section 3.1) and Omega = KL-to-
+# reference + entropy bonus (section 2.2 "Regularization").
+# --------------------------------------------------------------------------- #
+def token_weights(mask):
+    """Token-mean weights w_t = m_t / sum(m) (length-masked token mean)."""
+    m = np.asarray(mask).astype(np.float64)
+    n = m.sum()
+    return m / n if n > 0 else np.zeros_like(m)
+
+
+def per_token_terms(logp, old_logp, ref_logp, adv, eps_low, eps_high, beta,
+                    literal_clip=False):
+    """Per-token surrogate s_t, k3_t, ratio rho_t and d(loss_t)/d(logp_t) (unweighted).
+
+    rho = exp(logp - old)                       (section 2.2, importance ratio)
+    s   = min(rho*A, clip(rho,1-eps_low,1+eps_high)*A)      (section 3.1)
+    k3  = exp(delta) - delta - 1, delta = ref - logp        (reading of Omega)
+    loss_t = -s + beta*k3 (entropy handled by the caller).
+    """
+    rho = np.exp(logp - old_logp)
+    clipped = np.clip(rho, 1.0 - eps_low, 1.0 + eps_high)
+    if literal_clip:
+        s = np.minimum(rho, clipped) * adv
+        active = (rho <= clipped)
+    else:
+        s = np.minimum(rho * adv, clipped * adv)
+        # the unclipped branch is the minimum (ties count as unclipped)
+        active = (rho * adv <= clipped * adv)
+    if beta != 0.0:
+        delta = ref_logp - logp
+        k3 = np.exp(delta) - delta - 1.0
+        dk3 = 1.0 - np.exp(delta)          # d k3 / d logp
+    else:
+        k3 = np.zeros_like(logp)
+        dk3 = np.zeros_like(logp)
+    # d s / d logp = A * rho on the unclipped branch, 0 on the clipped one
+    dlogp = -(adv * rho * active) + beta * dk3
+    return s, k3, rho, active, dlogp
+
+
+def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
+                        eps_low, eps_high, beta, ent_coef=0.0,
+                        token_weight=None, literal_clip=False):
+    """Loss of Eq. 6 (negated) and its gradients with respect to H and W.
+
+    Returns a dict with loss, dH[T,d], dW[V,d], logp, entropy, lse, G (the
+    gradient with respect to the logits on valid rows, [n_valid, V]) and the
+    usual scalar metrics.  Rows with mask 0 contribute nothing and get dH = 0.
+    """
+    H = np.asarray(H, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    tokens = np.asarray(tokens)
+    T, d = H.shape
+    V = W.shape[0]
+    m = np.asarray(mask).astype(bool)
+    w = token_weights(m) if token_weight is None else np.asarray(token_weight, dtype=np.float64) * m
+    old_logp = np.asarray(old_logp, dtype=np.float64)
+    adv = np.asarray(adv, dtype=np.float64)
+    ref = np.zeros(T) if ref_logp is None else np.asarray(ref_logp, dtype=np.float64)
+
+    rows = np.nonzero(m)[0]
+    out = dict(loss=0.0, dH=np.zeros((T, d)), dW=np.zeros((V, d)),
+               logp=np.zeros(T), entropy=np.zeros(T), lse=np.zeros(T),
+               G=np.zeros((0, V)), rows=rows)
+    if rows.size == 0:
+        out.update(pg_loss=0.0, kl_mean=0.0, entropy_mean=0.0, clip_frac=0.0)
+        return out
+
+    Hr = H[rows]
+    y = tokens[rows]
+    Z = logits(Hr, W)                               # [n, V]
+    lse, LP, ent = log_softmax_stats(Z)
+    P = np.exp(LP)
+    logp = LP[np.arange(rows.size), y]
+
+    s, k3, rho, active, dlogp = per_token_terms(
+        logp, old_logp[rows], ref[rows], adv[rows], eps_low, eps_high, beta, literal_clip)
+    wr = w[rows]
+    loss_t = -s + beta * k3 - ent_coef * ent
+    loss = float((wr * loss_t).sum())
+
+    # gradient with respect to the logits:
+    #   d logp_t / d z_tj = 1[j = y_t] - p_tj
+    #   d Ent_t  / d z_tj = -p_tj * (log p_tj + Ent_t)
+    onehot = np.zeros_like(P)
+    onehot[np.arange(rows.size), y] = 1.0
+    G = (wr * dlogp)[:, None] * (onehot - P)
+    if ent_coef != 0.0:
+        G += (wr * ent_coef)[:, None] * P * (LP + ent[:, None])
+
+    out["dH"][rows] = G @ W                         # dH_tk = sum_j g_tj W_jk
+    out["dW"] = G.T @ Hr                            # dW_jk = sum_t g_tj H_tk
+    out["loss"] = loss
+    out["logp"][rows] = logp
+    out["entropy"][rows] = ent
+    out["lse"][rows] = lse
+    out["G"] = G
+    out["pg_loss"] = float((wr * -s).sum())
+    out["kl_mean"] = float((wr * k3).sum())
+    out["entropy_mean"] = float((wr * ent).sum())
+    out["clip_frac"] = float((wr * (~active)).sum())
+    out["rho"] = rho
+    out["active"] = active
+    return out
+
+
+# --------------------------------------------------------------------------- #
+# Sampled checks at sizes where the full gradient is too slow to form: one
+# row of dH needs only that row; one row of dW needs that vocabulary row of
+# the logits for every valid token plus per-token statistics.
+# --------------------------------------------------------------------------- #
+def dH_rows(H_rows, W, tokens_rows, old_rows, ref_rows, adv_rows, w_rows,
+            eps_low, eps_high, beta, ent_coef=0.0):
+    """dH for a subset of valid rows whose token weights w_rows are given."""
+    H_rows = np.asarray(H_rows, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    n = H_rows.shape[0]
+    Z = logits(H_rows, W)
+    lse, LP, ent = log_softmax_stats(Z)
+    P = np.exp(LP)
+    y = np.asarray(tokens_rows)
+    logp = LP[np.arange(n), y]
+    ref = np.zeros(n) if ref_rows is None else np.asarray(ref_rows, dtype=np.float64)
+    s, k3, rho, active, dlogp = per_token_terms(
+        logp, np.asarray(old_rows, dtype=np.float64), ref,
+        np.asarray(adv_rows, dtype=np.float64), eps_low, eps_high, beta)
+    onehot = np.zeros_like(P)
+    onehot[np.arange(n), y] = 1.0
+    w_rows = np.asarray(w_rows, dtype=np.float64)
+    G = (w_rows * dlogp)[:, None] * (onehot - P)
+    if ent_coef != 0.0:
+        G += (w_rows * ent_coef)[:, None] * P * (LP + ent[:, None])
+    return dict(dH=G @ W, logp=logp, entropy=ent, lse=lse,
+                loss_t=-s + beta * k3 - ent_coef * ent)
+
+
+def dW_rows(H_valid, W_sel, sel, tokens_valid, lse, ent, dlogp_w, ent_w):
+    """dW[j, :] for the vocabulary rows j in `sel`.
+
+    H_valid [n,d]: hidden states of every valid token; W_sel = W[sel];
+    lse, ent [n]: per-token log-sum-exp and entropy; dlogp_w[n] = w_t * d loss_t /
+    d logp_t; ent_w[n] = w_t * ent_coef.  g_tj as in policy_loss_fwd_bwd.
+    """
+    H_valid = np.asarray(H_valid, dtype=np.float64)
+    Zs = H_valid @ np.asarray(W_sel, dtype=np.float64).T        # [n, |sel|]
+    LP = Zs - np.asarray(lse, dtype=np.float64)[:, None]
+    P = np.exp(LP)
+    onehot = (np.asarray(tokens_valid)[:, None] == np.asarray(sel)[None, :]).astype(np.float64)
+    G = np.asarray(dlogp_w, dtype=np.float64)[:, None] * (onehot - P)
+    G += np.asarray(ent_w, dtype=np.float64)[:, None] * P * (LP + np.asarray(ent, dtype=np.float64)[:, None])
+    return G.T @ H_valid

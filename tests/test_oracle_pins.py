@@ -1,0 +1,364 @@
+"""Pins for the float64 oracle: brute force, closed forms, invariants, finite
+differences and library second opinions.  CPU only."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import grpo_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden(name):
+    vals = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, v = line.split()
+            vals[k] = float(v)
+    return vals
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+# ----------------------------------------------------------------------------- softmax / logp
+def test_logits_index_order_tiny():
+    # z[t, j] = sum_k H[t,k] W[j,k], checked with python loops on a non-square case
+    H = _rng(0).normal(size=(3, 5))
+    W = _rng(1).normal(size=(7, 5))
+    Z = O.logits(H, W)
+    assert Z.shape == (3, 7)
+    for t in range(3):
+        for j in range(7):
+            assert abs(Z[t, j] - sum(H[t, k] * W[j, k] for k in range(5))) < 1e-13
+
+
+def test_softmax_bruteforce_no_shift():
+    rng = _rng(2)
+    for V in (2, 5, 16):
+        Z = rng.normal(size=(4, V)) * 3.0
+        lse, LP, ent = O.log_softmax_stats(Z)
+        for t in range(4):
+            denom = sum(math.exp(z) for z in Z[t])
+            for j in range(V):
+                p = math.exp(Z[t, j]) / denom
+                assert abs(math.exp(LP[t, j]) - p) < 1e-13
+            assert abs(lse[t] - math.log(denom)) < 1e-12
+            naive_ent = -sum((math.exp(z) / denom) * math.log(math.exp(z) / denom) for z in Z[t])
+            assert abs(ent[t] - naive_ent) < 1e-12
+
+
+def test_softmax_invariants_and_bounds():
+    rng = _rng(3)
+    V = 37
+    Z = rng.normal(size=(9, V)) * 5.0
+    lse, LP, ent = O.log_softmax_stats(Z)
+    assert np.allclose(np.exp(LP).sum(axis=1), 1.0, atol=1e-13)
+    assert np.all(lse >= Z.max(axis=1)) and np.all(lse <= Z.max(axis=1) + math.log(V))
+    assert np.all(LP <= 0)
+    assert np.all(ent >= 0) and np.all(ent <= math.log(V) + 1e-12)
+    # shift invariance: adding a constant to every logit of a row changes lse by it, nothing else
+    lse2, LP2, ent2 = O.log_softmax_stats(Z + 7.25)
+    assert np.allclose(lse2, lse + 7.25, atol=1e-12)
+    assert np.allclose(LP2, LP, atol=1e-12) and np.allclose(ent2, ent, atol=1e-12)
+    # large logits must not overflow
+    lse3, _, _ = O.log_softmax_stats(Z + 900.0)
+    assert np.all(np.isfinite(lse3))
+
+
+def test_special_cases_uniform_and_dominant():
+    T, d, V = 5, 8, 11
+    H = _rng(4).normal(size=(T, d))
+    tokens = _rng(5).integers(0, V, size=T)
+    logp, ent, lse = O.token_logprobs(H, np.zeros((V, d)), tokens)
+    assert np.allclose(logp, -math.log(V), atol=1e-14)
+    assert np.allclose(ent, math.log(V), atol=1e-14)
+    # one dominant logit: logp -> 0, entropy -> 0
+    W = np.zeros((V, d))
+    W[3, 0] = 50.0
+    H1 = np.zeros((1, d))
+    H1[0, 0] = 1.0
+    logp, ent, _ = O.token_logprobs(H1, W, np.array([3]))
+    assert abs(logp[0]) < 1e-20 + 1e-15 and ent[0] < 1e-18 + 1e-15
+
+
+def test_token_logprobs_vs_torch_library():
+    T, d, V = 12, 16, 50
+    rng = _rng(6)
+    H = rng.normal(size=(T, d))
+    W = rng.normal(size=(V, d)) * 0.3
+    tokens = rng.integers(0, V, size=T)
+    mask = np.ones(T, dtype=np.uint8)
+    mask[[2, 7]] = 0
+    logp, ent, lse = O.token_logprobs(H, W, tokens, mask)
+    Zt = torch.from_numpy(H) @ torch.from_numpy(W).T
+    lp_t = -torch.nn.functional.cross_entropy(Zt, torch.from_numpy(tokens), reduction="none")
+    ent_t = torch.distributions.Categorical(logits=Zt).entropy()
+    m = mask.astype(bool)
+    assert np.allclose(logp[m], lp_t.numpy()[m], atol=1e-12)
+    assert np.allclose(ent[m], ent_t.numpy()[m], atol=1e-12)
+    assert np.allclose(lse[m], torch.logsumexp(Zt, dim=1).numpy()[m], atol=1e-12)
+    assert np.all(logp[~m] == 0) and np.all(ent[~m] == 0)
+
+
+# ----------------------------------------------------------------------------- advantages
+def test_advantages_mean0_std1():
+    rng = _rng(7)
+    for G in (4, 5, 8, 16):
+        for ddof in (0, 1):
+            r = rng.uniform(size=6 * G)
+            a = O.grpo_advantages(r, G, ddof=ddof, eps_std=1e-6).reshape(6, G)
+            rs = r.reshape(6, G)
+            sig = rs.std(axis=1, ddof=ddof)
+            assert np.allclose(a.mean(axis=1), 0.0, atol=1e-12)
+            assert np.allclose(a.std(axis=1, ddof=ddof), sig / (sig + 1e-6), atol=1e-12)
+
+
+def test_advantages_bernoulli_closed_form():
+    # k ones among G: sigma^2 = (k/G)(1-k/G) * G/(G-ddof)
+    for G in (4, 8, 16):
+        for k in range(1, G):
+            for ddof in (0, 1):
+                r = np.array([1.0] * k + [0.0] * (G - k))
+                a = O.grpo_advantages(r, G, ddof=ddof, eps_std=1e-6)
+                sigma = math.sqrt((k / G) * (1 - k / G) * G / (G - ddof))
+                assert np.allclose(a[:k], (1 - k / G) / (sigma + 1e-6), atol=1e-12)
+                assert np.allclose(a[k:], (0 - k / G) / (sigma + 1e-6), atol=1e-12)
+    # the worked case G=4, k=1, sample std: sigma = 0.5 -> {+1.5, -0.5, -0.5, -0.5} / (1 + 2e-6)
+    a = O.grpo_advantages(np.array([1.0, 0, 0, 0]), 4)
+    assert np.allclose(a, np.array([1.5, -0.5, -0.5, -0.5]) / (1 + 2e-6), atol=1e-12)
+
+
+def test_advantages_zero_variance_affine_permutation():
+    assert np.all(O.grpo_advantages(np.array([0.3, 0.3, 0.3, 1.0, 1.0, 1.0]), 3) == 0.0)
+    rng = _rng(8)
+    r = rng.normal(size=16)
+    a = O.grpo_advantages(r, 8, eps_std=0.0)
+    a2 = O.grpo_advantages(3.5 * r - 2.0, 8, eps_std=0.0)
+    assert np.allclose(a, a2, atol=1e-12)
+    perm = rng.permutation(8)
+    r2 = r.copy()
+    r2[:8] = r[:8][perm]
+    a3 = O.grpo_advantages(r2, 8, eps_std=0.0)
+    assert np.allclose(a3[:8], a[:8][perm], atol=1e-12)
+    assert np.allclose(a3[8:], a[8:], atol=1e-12)       # groups do not interact
+    with pytest.raises(ValueError):
+        O.grpo_advantages(r, 1)
+    with pytest.raises(ValueError):
+        O.grpo_advantages(r, 5)
+
+
+def test_broadcast_to_tokens():
+    offs = np.array([0, 3, 3, 7])
+    adv = O.broadcast_to_tokens(np.array([1.0, 2.0, -1.0]), offs, 9)
+    assert adv.tolist() == [1, 1, 1, -1, -1, -1, -1, 0, 0]
+
+
+# ----------------------------------------------------------------------------- clip / k3 / loss
+def test_clip_branches_constructed():
+    eps_lo, eps_hi = 0.2, 0.28
+    old = np.zeros(6)
+    rho = np.array([1.0, 1.5, 0.5, 1.0, 1.5, 0.5])
+    adv = np.array([2.0, 2.0, 2.0, -2.0, -2.0, -2.0])
+    s, k3, r, active, dlogp = O.per_token_terms(np.log(rho), old, old, adv, eps_lo, eps_hi, 0.0)
+    # A>0: inside -> rho*A; above -> (1+eps_hi)*A clipped; below -> rho*A (unclipped is smaller)
+    # A<0: inside -> rho*A; above -> rho*A (more negative); below -> (1-eps_lo)*A clipped
+    assert np.allclose(s, [2.0, 1.28 * 2, 0.5 * 2, -2.0, -3.0, -0.8 * 2], atol=1e-14)
+    assert active.tolist() == [True, False, True, True, True, False]
+    assert np.allclose(dlogp, -adv * rho * active, atol=1e-14)
+    assert np.all(k3 == 0)
+    # the surrogate as literally printed differs only for A<0
+    s_lit, *_ = O.per_token_terms(np.log(rho), old, old, adv, eps_lo, eps_hi, 0.0, literal_clip=True)
+    assert np.allclose(s_lit[:3], s[:3], atol=1e-14)
+    assert np.allclose(s_lit[3:], [-2.0, -1.28 * 2, -1.0], atol=1e-14)
+
+
+def test_k3_properties():
+    logp = np.array([-1.0, -2.0, -3.0, -0.5])
+    ref = logp + np.array([0.0, 1e-4, -0.7, 1.3])
+    _, k3, _, _, dlogp = O.per_token_terms(logp, logp, ref, np.zeros(4), 0.2, 0.2, 1.0)
+    assert k3[0] == 0 and dlogp[0] == 0
+    assert np.all(k3 >= 0)
+    assert abs(k3[1] - 0.5e-8) < 1e-11                   # Taylor: delta^2/2
+    d = ref - logp
+    assert np.allclose(k3, np.exp(d) - d - 1, atol=1e-15)
+
+
+def _tiny_problem(seed, T=6, d=8, V=16, masked=(4,)):
+    rng = _rng(seed)
+    H = rng.normal(size=(T, d))
+    W = rng.normal(size=(V, d)) * 0.5
+    tokens = rng.integers(0, V, size=T)
+    mask = np.ones(T, dtype=np.uint8)
+    for i in masked:
+        mask[i] = 0
+    logp, _, _ = O.token_logprobs(H, W, tokens)
+    old = logp + rng.normal(size=T) * 0.3
+    ref = logp + rng.normal(size=T) * 0.2
+    adv = rng.normal(size=T)
+    return H, W, tokens, old, ref, adv, mask
+
+
+def test_two_token_worked_example():
+    g = _golden("two_token_worked_example.txt")
+    H = np.array([[1.0]])
+    W = np.array([[0.0], [math.log(3.0)]])
+    tok = np.array([1])
+    m = np.array([1], dtype=np.uint8)
+    old = np.array([math.log(0.5)])
+    ref = np.array([math.log(0.375)])
+    A = O.policy_loss_fwd_bwd(H, W, tok, old, ref, np.array([1.0]), m, 0.2, 0.2, 0.5)
+    assert abs(A["logp"][0] - g["logp"]) < 1e-14 and abs(A["entropy"][0] - g["entropy"]) < 1e-14
+    assert abs(A["rho"][0] - g["rho"]) < 1e-14 and abs(A["kl_mean"] - g["k3"]) < 1e-14
+    assert abs(A["loss"] - g["A_loss"]) < 1e-14
+    assert np.allclose(A["G"][0], [g["A_g0"], g["A_g1"]], atol=1e-14)
+    assert abs(A["dH"][0, 0] - g["A_dH"]) < 1e-14
+    assert np.allclose(A["dW"][:, 0], [g["A_g0"], g["A_g1"]], atol=1e-14)
+    B = O.policy_loss_fwd_bwd(H, W, tok, old, ref, np.array([-1.0]), m, 0.2, 0.2, 0.5)
+    assert abs(B["loss"] - g["B_loss"]) < 1e-14
+    assert np.allclose(B["G"][0], [g["B_g0"], g["B_g1"]], atol=1e-14)
+    Bl = O.policy_loss_fwd_bwd(H, W, tok, old, ref, np.array([-1.0]), m, 0.2, 0.2, 0.5, literal_clip=True)
+    assert abs(Bl["loss"] - g["B_literal_loss"]) < 1e-14
+    C = O.policy_loss_fwd_bwd(H, W, tok, old, ref, np.array([1.0]), m, 0.2, 0.2, 0.5, ent_coef=0.1)
+    assert abs(C["loss"] - g["C_loss"]) < 1e-13
+    assert np.allclose(C["G"][0], [g["C_g0"], g["C_g1"]], atol=1e-13)
+
+
+def test_loss_identities():
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(10)
+    logp, ent, _ = O.token_logprobs(H, W, tokens)
+    w = O.token_weights(mask)
+    assert abs(w.sum() - 1.0) < 1e-15 and w[4] == 0
+    # on-policy (rho = 1), no regulariser: loss = - sum w_t A_t
+    base = O.policy_loss_fwd_bwd(H, W, tokens, logp, None, adv, mask, 0.2, 0.2, 0.0)
+    assert abs(base["loss"] + (w * adv).sum()) < 1e-14
+    # switching beta / ent_coef on moves the loss by exactly beta*sum(w k3) / -c*sum(w Ent)
+    d = ref - logp
+    k3 = np.exp(d) - d - 1
+    withkl = O.policy_loss_fwd_bwd(H, W, tokens, logp, ref, adv, mask, 0.2, 0.2, 0.04)
+    assert abs(withkl["loss"] - base["loss"] - 0.04 * (w * k3).sum()) < 1e-14
+    withent = O.policy_loss_fwd_bwd(H, W, tokens, logp, None, adv, mask, 0.2, 0.2, 0.0, ent_coef=1e-3)
+    assert abs(withent["loss"] - base["loss"] + 1e-3 * (w * ent).sum()) < 1e-14
+    # equal-length unpadded groups: group advantages sum to zero, so the on-policy loss is 0
+    T = 8
+    rng = _rng(11)
+    Hh = rng.normal(size=(T, 4))
+    Ww = rng.normal(size=(5, 4))
+    tk = rng.integers(0, 5, size=T)
+    lp, _, _ = O.token_logprobs(Hh, Ww, tk)
+    a_seq = O.grpo_advantages(np.array([1.0, 0, 0, 1.0]), 4)
+    a_tok = O.broadcast_to_tokens(a_seq, np.array([0, 2, 4, 6, 8]), T)
+    out = O.policy_loss_fwd_bwd(Hh, Ww, tk, lp, None, a_tok, np.ones(T), 0.2, 0.2, 0.0)
+    assert abs(out["loss"]) < 1e-14
+    # empty batch
+    e = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, np.zeros(6), 0.2, 0.2, 0.04)
+    assert e["loss"] == 0 and not e["dH"].any() and not e["dW"].any()
+
+
+# ----------------------------------------------------------------------------- gradients
+def test_gradient_closed_form_on_policy():
+    # Eq. 3: at rho = 1, no clipping, beta = 0 the gradient is the advantage-weighted
+    # score function: g_tj = -w_t A_t (1[j=y_t] - p_tj)
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(12)
+    logp, _, _ = O.token_logprobs(H, W, tokens)
+    out = O.policy_loss_fwd_bwd(H, W, tokens, logp, None, adv, mask, 0.2, 0.2, 0.0)
+    w = O.token_weights(mask)
+    rows = np.nonzero(mask)[0]
+    Z = H[rows] @ W.T
+    P = np.exp(Z) / np.exp(Z).sum(axis=1, keepdims=True)
+    onehot = np.eye(W.shape[0])[tokens[rows]]
+    G = -(w[rows] * adv[rows])[:, None] * (onehot - P)
+    assert np.allclose(out["G"], G, atol=1e-14)
+    dH = np.zeros_like(H)
+    dH[rows] = G @ W
+    assert np.allclose(out["dH"], dH, atol=1e-14)
+    assert np.allclose(out["dW"], G.T @ H[rows], atol=1e-14)
+
+
+@pytest.mark.parametrize("beta,ent_coef,eps", [(0.0, 0.0, (0.2, 0.2)), (0.3, 0.0, (0.2, 0.2)),
+                                               (0.0, 0.05, (0.2, 0.28)), (0.3, 0.05, (0.2, 0.28)),
+                                               (0.3, 0.05, (10.0, 10.0))])
+def test_gradient_finite_differences(beta, ent_coef, eps):
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(13)
+    kw = dict(eps_low=eps[0], eps_high=eps[1], beta=beta, ent_coef=ent_coef)
+    refp = ref if beta != 0 else None
+    out = O.policy_loss_fwd_bwd(H, W, tokens, old, refp, adv, mask, **kw)
+    # the problem must exercise both clipped and unclipped tokens when eps is small
+    if eps[0] < 1:
+        assert out["active"].any() and (~out["active"]).any()
+
+    def loss(Hx, Wx):
+        return O.policy_loss_fwd_bwd(Hx, Wx, tokens, old, refp, adv, mask, **kw)["loss"]
+
+    h = 1e-6
+    for (X, dX, which) in ((H, out["dH"], 0), (W, out["dW"], 1)):
+        num = np.zeros_like(X)
+        for idx in np.ndindex(*X.shape):
+            Xp = X.copy(); Xp[idx] += h
+            Xm = X.copy(); Xm[idx] -= h
+            num[idx] = ((loss(Xp, W) - loss(Xm, W)) if which == 0 else (loss(H, Xp) - loss(H, Xm))) / (2 * h)
+        denom = max(np.abs(num).max(), 1e-12)
+        assert np.abs(num - dX).max() / denom < 1e-6
+
+
+def test_gradient_vs_torch_autograd():
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(14, T=10, d=6, V=20, masked=(1, 8))
+    eps_lo, eps_hi, beta, c_ent = 0.2, 0.28, 0.04, 0.01
+    out = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, eps_lo, eps_hi, beta, ent_coef=c_ent)
+    Ht = torch.tensor(H, requires_grad=True)
+    Wt = torch.tensor(W, requires_grad=True)
+    m = torch.tensor(mask.astype(np.float64))
+    lsm = torch.log_softmax(Ht @ Wt.T, dim=1)
+    lp = lsm.gather(1, torch.tensor(tokens)[:, None])[:, 0]
+    ent = -(lsm.exp() * lsm).sum(1)
+    ratio = (lp - torch.tensor(old)).exp()
+    A = torch.tensor(adv)
+    s = torch.minimum(ratio * A, ratio.clamp(1 - eps_lo, 1 + eps_hi) * A)
+    dl = torch.tensor(ref) - lp
+    lt = -s + beta * (dl.exp() - dl - 1) - c_ent * ent
+    L = (lt * m).sum() / m.sum()
+    L.backward()
+    assert abs(L.item() - out["loss"]) < 1e-13
+    assert np.allclose(Ht.grad.numpy(), out["dH"], atol=1e-13)
+    assert np.allclose(Wt.grad.numpy(), out["dW"], atol=1e-13)
+
+
+def test_gradient_identities():
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(15, T=9, d=5, V=13, masked=(0,))
+    out = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, 0.2, 0.2, 0.04, ent_coef=0.02)
+    assert np.allclose(out["G"].sum(axis=1), 0.0, atol=1e-15)        # softmax gradient rows sum to 0
+    assert np.allclose(out["dW"].sum(axis=0), 0.0, atol=1e-14)
+    assert abs((out["dH"] * H).sum() - (out["dW"] * W).sum()) < 1e-13  # both equal sum g_tj z_tj
+    assert not out["dH"][0].any()
+
+
+def test_custom_token_weight_and_sampled_helpers():
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(16, T=9, d=5, V=13, masked=(3,))
+    rng = _rng(17)
+    tw = rng.uniform(size=9)
+    kw = dict(eps_low=0.2, eps_high=0.28, beta=0.04, ent_coef=0.02)
+    out = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, token_weight=tw, **kw)
+    # linearity in the weights: sum over single-token problems
+    acc = 0.0
+    for t in np.nonzero(mask)[0]:
+        one = np.zeros(9); one[t] = 1
+        acc += tw[t] * O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, one, **kw)["loss"]
+    assert abs(acc - out["loss"]) < 1e-13
+    rows = np.nonzero(mask)[0]
+    w = tw * mask
+    sub = rows[[1, 4, 6]]
+    r = O.dH_rows(H[sub], W, tokens[sub], old[sub], ref[sub], adv[sub], w[sub], **kw)
+    assert np.allclose(r["dH"], out["dH"][sub], atol=1e-14)
+    assert np.allclose(r["logp"], out["logp"][sub], atol=1e-14)
+    sel = np.array([0, 5, 12, int(tokens[rows[0]])])
+    _, _, _, _, dlogp = O.per_token_terms(out["logp"][rows], old[rows], ref[rows], adv[rows], 0.2, 0.28, 0.04)
+    dWs = O.dW_rows(H[rows], W[sel], sel, tokens[rows], out["lse"][rows], out["entropy"][rows],
+                    w[rows] * dlogp, w[rows] * 0.02)
+    assert np.allclose(dWs, out["dW"][sel], atol=1e-14)
