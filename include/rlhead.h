@@ -1,0 +1,162 @@
+/* rlhead.h - C ABI of the fused LM-head log-probability + GRPO policy-loss library (sm_100a).
+ *
+ * The library evaluates, for a batch of token positions, the quantities of the policy-update
+ * step of Algorithm 1 ("compute estimating advantages" and "update the policy model by
+ * maximizing the objective", Eq. 6): GRPO group-normalised advantages (section 4.2), the
+ * log-probability of every sampled token under the next-token policy over the vocabulary
+ * (section 2.2), its entropy (section 2.2 "Regularization"), the clipped importance-ratio
+ * surrogate (section 3.1) with a KL-to-reference regulariser, and the gradient of the resulting
+ * loss with respect to the hidden states H and the LM-head weight W.  The [T,V] logits are
+ * never written to memory.
+ *
+ * Conventions
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.
+ *     The library allocates only inside rl_ctx (a few KB of device memory for counters and the
+ *     status word) and otherwise works in the caller-provided workspace.
+ *   - All functions return rl_status; 0 is success.  Nothing throws, traps or aborts.
+ *   - Calls enqueue work on the context's stream and return; argument errors are reported
+ *     synchronously, errors found on the device (token id outside [0,V) on a valid row, a
+ *     bounded wait that ran out) are latched in a device status word read by
+ *     rl_last_device_status().
+ *   - H is [T,d] bf16 row-major with row stride ldH elements, W is [V,d] bf16 row-major with
+ *     row stride ldW elements (the layout of a linear layer's weight).  Row t of H is the hidden
+ *     state whose next-token distribution scores tokens[t].  d must be a multiple of 64; ldH
+ *     and ldW multiples of 8; H and W base addresses 16-byte aligned (TMA requirements).
+ *   - mask is one byte per row (non-zero = the token takes part in the loss); NULL means all
+ *     valid.  Rows with mask 0 are skipped entirely (padding-free execution, section 4.4):
+ *     their outputs are 0 and their token ids are ignored.
+ *   - T = 0 or an all-zero mask is not an error: loss 0, gradients 0.
+ */
+#ifndef RLHEAD_H_
+#define RLHEAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RL_OK = 0,
+  RL_ERR_INVALID_ARG = 1,      /* NULL required pointer, negative size, bad hyper-parameter   */
+  RL_ERR_SHAPE = 2,            /* d not a multiple of 64, group_size does not divide n_seq ... */
+  RL_ERR_ALIGNMENT = 3,        /* base pointer or leading dimension breaks the TMA rules       */
+  RL_ERR_WORKSPACE = 4,        /* workspace missing or smaller than rl_workspace_bytes()       */
+  RL_ERR_CUDA = 5,             /* a CUDA runtime / driver call failed                          */
+  RL_ERR_UNSUPPORTED_ARCH = 6, /* device is not compute capability 10.x                        */
+  RL_ERR_TOKEN_RANGE = 7,      /* device: token id outside [0,V) on a valid row                */
+  RL_ERR_TIMEOUT = 8           /* device: a bounded wait inside a kernel ran out               */
+} rl_status;
+
+typedef struct rl_ctx rl_ctx;  /* opaque; one per device and stream */
+
+/* Context.  rl_create checks that `device` is compute capability 10.x, allocates the context's
+ * small device block and uses the legacy default stream until rl_set_stream is called. */
+rl_status rl_create(rl_ctx** out, int device);
+rl_status rl_destroy(rl_ctx* ctx);
+rl_status rl_set_stream(rl_ctx* ctx, void* cuda_stream);
+const char* rl_status_string(rl_status s);
+
+/* Bytes of scratch needed by any call with at most T rows, hidden size d, vocabulary V.  The
+ * size does not grow with T*V: the gradient with respect to the logits only ever exists for a
+ * bounded slab of rows x vocabulary columns. */
+rl_status rl_workspace_bytes(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_t* bytes);
+/* Caller-owned device scratch, 256-byte aligned; must outlive the calls that use it. */
+rl_status rl_set_workspace(rl_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* Synchronises the context's stream and returns the latched device status (RL_OK,
+ * RL_ERR_TOKEN_RANGE or RL_ERR_TIMEOUT), then clears it.  detail (host, may be NULL) receives a
+ * kernel-specific word describing where the first error was seen. */
+rl_status rl_last_device_status(rl_ctx* ctx, int32_t* detail);
+
+/* GRPO advantages - Algorithm 1 "compute estimating advantages"; section 3.2.2 advantage
+ * estimation stage; section 4.2 "group-based normalization".
+ * rewards[n_seq] holds one scalar per response (section 3.2.2 scoring stage), the group_size
+ * responses of a prompt stored consecutively.  adv_seq[i] = (r_i - mean_g) / (std_g + eps_std);
+ * a group whose rewards are all equal gets exactly 0.  The basic call uses the sample standard
+ * deviation (ddof = 1) and eps_std = 1e-6.  With seq_offsets[n_seq+1] (row range of each
+ * response) and adv_tok[T] non-NULL the per-response value is also broadcast to every row of
+ * the response (rows outside every range get 0); T = seq_offsets[n_seq].
+ * Errors: group_size < 2 or n_seq % group_size != 0 -> RL_ERR_SHAPE; ddof not 0/1, eps_std < 0,
+ * NULL rewards/adv_seq -> RL_ERR_INVALID_ARG. */
+rl_status rl_grpo_advantages(rl_ctx* ctx, const float* rewards, int64_t n_seq, int group_size,
+                             float* adv_seq);
+rl_status rl_grpo_advantages_ex(rl_ctx* ctx, const float* rewards, int64_t n_seq, int group_size,
+                                int ddof, float eps_std, const int32_t* seq_offsets,
+                                int64_t T, float* adv_seq, float* adv_tok);
+
+/* Per-token log-probability of the sampled token, entropy and log-sum-exp of the next-token
+ * distribution softmax(W h_t) - section 2.2 (policy over the vocabulary; importance ratio
+ * numerator) and section 2.2 "Regularization" (entropy).  Natural logarithms.
+ * logp[T] required; entropy[T] and lse[T] may be NULL.  Masked rows get 0. */
+rl_status rl_token_logprobs(rl_ctx* ctx, const void* H, int64_t ldH, const void* W, int64_t ldW,
+                            const int32_t* tokens, const uint8_t* mask,
+                            int64_t T, int64_t d, int64_t V,
+                            float* logp, float* entropy, float* lse);
+
+/* Loss of Eq. 6 (negated, to be minimised) and its gradients.
+ *   rho_t  = exp(logp_t - old_logp_t)                                   (section 2.2)
+ *   s_t    = min(rho_t A_t, clip(rho_t, 1-eps_low, 1+eps_high) A_t)     (section 3.1)
+ *   k3_t   = exp(delta_t) - delta_t - 1, delta_t = ref_logp_t - logp_t  (KL-to-reference)
+ *   loss   = sum_t w_t (-s_t + beta k3_t - ent_coef Ent_t),  w_t = mask_t / sum(mask)
+ * loss[1] is a device scalar.  dH[T,d] (bf16, row stride d; masked rows 0) and dW[V,d] (fp32,
+ * row stride d) are fully overwritten.  adv is per row [T].  ref_logp may be NULL iff beta == 0.
+ * Errors: eps_low outside [0,1), eps_high < 0, beta < 0, NULL required pointer ->
+ * RL_ERR_INVALID_ARG; shape/alignment/workspace as above. */
+rl_status rl_policy_loss_fwd_bwd(rl_ctx* ctx, const void* H, int64_t ldH, const void* W,
+                                 int64_t ldW, const int32_t* tokens, const float* old_logp,
+                                 const float* ref_logp, const float* adv, const uint8_t* mask,
+                                 int64_t T, int64_t d, int64_t V,
+                                 float eps_low, float eps_high, float beta,
+                                 float* loss, void* dH, float* dW);
+
+/* Options of the extended call.  Zero-initialise, set struct_size = sizeof(rl_loss_opts). */
+typedef struct {
+  size_t struct_size;
+  float ent_coef;             /* entropy bonus coefficient (section 2.2), >= 0                 */
+  const float* token_weight;  /* [T] or NULL: replaces w_t = mask_t/sum(mask) by               */
+                              /* token_weight[t]*mask_t ("length normalization with token      */
+                              /* weights", section 2.2)                                        */
+  int accumulate_dW;          /* non-zero: dW += gradient instead of overwrite                 */
+  float* logp_out;            /* [T] or NULL                                                   */
+  float* entropy_out;         /* [T] or NULL                                                   */
+  float* metrics_out;         /* [8] or NULL: pg_loss, kl_mean, entropy_mean, clip_frac,       */
+                              /* ratio_mean, ratio_max, n_valid, reserved                      */
+} rl_loss_opts;
+
+rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* ctx, const void* H, int64_t ldH, const void* W,
+                                    int64_t ldW, const int32_t* tokens, const float* old_logp,
+                                    const float* ref_logp, const float* adv, const uint8_t* mask,
+                                    int64_t T, int64_t d, int64_t V,
+                                    float eps_low, float eps_high, float beta,
+                                    float* loss, void* dH, float* dW, const rl_loss_opts* opts);
+
+/* Same computation with the per-step inputs in HOST memory (pinned memory gives asynchronous
+ * copies): H, tokens, old_logp, ref_logp, adv, mask are host pointers, copied to the device
+ * inside the call; W, dH and dW stay device pointers (weights and gradients live on the
+ * device); loss_host[1] and metrics_host[8] (may be NULL) are written on the host.  The call
+ * synchronises the context's stream before returning.  The workspace must have been sized with
+ * rl_workspace_bytes_host(). */
+rl_status rl_workspace_bytes_host(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_t* bytes);
+rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* ctx, const void* H_host, int64_t ldH, const void* W,
+                                      int64_t ldW, const int32_t* tokens_host,
+                                      const float* old_logp_host, const float* ref_logp_host,
+                                      const float* adv_host, const uint8_t* mask_host,
+                                      int64_t T, int64_t d, int64_t V,
+                                      float eps_low, float eps_high, float beta, float ent_coef,
+                                      float* loss_host, float* metrics_host, void* dH, float* dW);
+
+/* Self-test of the tensor-core GEMM engine the calls above are built from: C[M,N] (fp32,
+ * row-major, ldc = N) = A * B with bf16 operands.  a_mn_major = 0: A is [M,K] row-major;
+ * 1: A is stored [K,M] row-major.  b_mn_major = 0: B is stored [N,K] row-major; 1: B is stored
+ * [K,N] row-major.  M, N multiples of 64, K a multiple of 8.  The paper has no counterpart; this
+ * entry exists so that the operand layouts can be checked against a library product. */
+rl_status rl_selftest_gemm(rl_ctx* ctx, const void* A, const void* B, float* C,
+                           int64_t M, int64_t N, int64_t K, int a_mn_major, int b_mn_major,
+                           int accumulate);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RLHEAD_H_ */

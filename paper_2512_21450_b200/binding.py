@@ -1,0 +1,254 @@
+"""ctypes binding of librlhead.so (C ABI declared in include/rlhead.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch is used for device memory and streams.  There is no CPU
+fallback: if the shared library is missing or the device is not sm_100, the
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librlhead.so")
+
+STATUS_NAMES = {
+    0: "RL_OK", 1: "RL_ERR_INVALID_ARG", 2: "RL_ERR_SHAPE", 3: "RL_ERR_ALIGNMENT", 4: "RL_ERR_WORKSPACE",
+    5: "RL_ERR_CUDA", 6: "RL_ERR_UNSUPPORTED_ARCH", 7: "RL_ERR_TOKEN_RANGE", 8: "RL_ERR_TIMEOUT",
+}
+
+
+class RLHeadError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class rl_loss_opts(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", c_size_t),
+        ("ent_coef", c_float),
+        ("token_weight", c_void_p),
+        ("accumulate_dW", c_int),
+        ("logp_out", c_void_p),
+        ("entropy_out", c_void_p),
+        ("metrics_out", c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load_library():
+    """Load librlhead.so; raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2512_21450_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    P = c_void_p
+    lib.rl_status_string.restype = c_char_p
+    lib.rl_status_string.argtypes = [c_int]
+    lib.rl_create.argtypes = [POINTER(c_void_p), c_int]
+    lib.rl_destroy.argtypes = [P]
+    lib.rl_set_stream.argtypes = [P, P]
+    lib.rl_workspace_bytes.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
+    lib.rl_workspace_bytes_host.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
+    lib.rl_set_workspace.argtypes = [P, P, c_size_t]
+    lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
+    lib.rl_grpo_advantages.argtypes = [P, P, c_int64, c_int, P]
+    lib.rl_grpo_advantages_ex.argtypes = [P, P, c_int64, c_int, c_int, c_float, P, c_int64, P, P]
+    lib.rl_token_logprobs.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P]
+    loss_args = [P, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int64, c_int64,
+                 c_float, c_float, c_float, P, P, P]
+    lib.rl_policy_loss_fwd_bwd.argtypes = loss_args
+    lib.rl_policy_loss_fwd_bwd_ex.argtypes = loss_args + [POINTER(rl_loss_opts)]
+    lib.rl_policy_loss_fwd_bwd_host.argtypes = [P, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int64, c_int64,
+                                                c_float, c_float, c_float, c_float, P, P, P, P]
+    lib.rl_selftest_gemm.argtypes = [P, P, P, P, c_int64, c_int64, c_int64, c_int, c_int, c_int]
+    for name in ("rl_create", "rl_destroy", "rl_set_stream", "rl_workspace_bytes", "rl_workspace_bytes_host",
+                 "rl_set_workspace", "rl_last_device_status", "rl_grpo_advantages", "rl_grpo_advantages_ex",
+                 "rl_token_logprobs", "rl_policy_loss_fwd_bwd", "rl_policy_loss_fwd_bwd_ex",
+                 "rl_policy_loss_fwd_bwd_host", "rl_selftest_gemm"):
+        getattr(lib, name).restype = c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    return c_void_p(t.data_ptr()) if t is not None else c_void_p(0)
+
+
+def _check(status, where):
+    if status != 0:
+        raise RLHeadError(status, where)
+
+
+class Context:
+    """One library context on one device; owns a torch-allocated workspace."""
+
+    def __init__(self, device=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("rlhead needs a CUDA device (sm_100a); there is no CPU path")
+        self.lib = load_library()
+        self.device = torch.device("cuda", device)
+        self.handle = c_void_p()
+        _check(self.lib.rl_create(byref(self.handle), device), "rl_create")
+        self._ws = None
+        self._ws_key = None
+
+    def close(self):
+        if self.handle:
+            self.lib.rl_destroy(self.handle)
+            self.handle = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _bind_stream(self):
+        _check(self.lib.rl_set_stream(self.handle, c_void_p(torch.cuda.current_stream(self.device).cuda_stream)),
+               "rl_set_stream")
+
+    def workspace_bytes(self, T, d, V, host=False):
+        n = c_size_t()
+        fn = self.lib.rl_workspace_bytes_host if host else self.lib.rl_workspace_bytes
+        _check(fn(self.handle, T, d, V, byref(n)), "rl_workspace_bytes")
+        return n.value
+
+    def ensure_workspace(self, T, d, V, host=False):
+        need = self.workspace_bytes(T, d, V, host)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = None
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        _check(self.lib.rl_set_workspace(self.handle, _ptr(self._ws), self._ws.numel()), "rl_set_workspace")
+
+    def last_device_status(self):
+        detail = c_int32()
+        return self.lib.rl_last_device_status(self.handle, byref(detail)), detail.value
+
+    # ------------------------------------------------------------------ calls
+    def rl_grpo_advantages(self, rewards, group_size, ddof=1, eps_std=1e-6, seq_offsets=None, T=None):
+        self._bind_stream()
+        assert rewards.dtype == torch.float32 and rewards.is_cuda and rewards.is_contiguous()
+        adv_seq = torch.empty_like(rewards)
+        if seq_offsets is None:
+            if ddof == 1 and eps_std == 1e-6:
+                _check(self.lib.rl_grpo_advantages(self.handle, _ptr(rewards), rewards.numel(), group_size,
+                                                   _ptr(adv_seq)), "rl_grpo_advantages")
+            else:
+                _check(self.lib.rl_grpo_advantages_ex(self.handle, _ptr(rewards), rewards.numel(), group_size, ddof,
+                                                      eps_std, None, 0, _ptr(adv_seq), None),
+                       "rl_grpo_advantages_ex")
+            return adv_seq
+        assert seq_offsets.dtype == torch.int32 and seq_offsets.is_cuda
+        adv_tok = torch.empty(T, dtype=torch.float32, device=rewards.device)
+        _check(self.lib.rl_grpo_advantages_ex(self.handle, _ptr(rewards), rewards.numel(), group_size, ddof, eps_std,
+                                              _ptr(seq_offsets), T, _ptr(adv_seq), _ptr(adv_tok)),
+               "rl_grpo_advantages_ex")
+        return adv_seq, adv_tok
+
+    def rl_token_logprobs(self, H, W, tokens, mask=None):
+        self._bind_stream()
+        T, d = H.shape
+        V = W.shape[0]
+        assert H.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and tokens.dtype == torch.int32
+        assert H.stride(1) == 1 and W.stride(1) == 1
+        self.ensure_workspace(T, d, V)
+        logp = torch.empty(T, dtype=torch.float32, device=H.device)
+        ent = torch.empty_like(logp)
+        lse = torch.empty_like(logp)
+        _check(self.lib.rl_token_logprobs(self.handle, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0),
+                                          _ptr(tokens), _ptr(mask), T, d, V, _ptr(logp), _ptr(ent), _ptr(lse)),
+               "rl_token_logprobs")
+        return logp, ent, lse
+
+    def rl_policy_loss_fwd_bwd(self, H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta,
+                               ent_coef=0.0, token_weight=None, accumulate_dW=False, dW=None, want_aux=True,
+                               dH=None, loss=None):
+        self._bind_stream()
+        T, d = H.shape
+        V = W.shape[0]
+        assert H.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and tokens.dtype == torch.int32
+        assert H.stride(1) == 1 and W.stride(1) == 1
+        self.ensure_workspace(T, d, V)
+        dev = W.device
+        loss = torch.empty(1, dtype=torch.float32, device=dev) if loss is None else loss
+        dH = torch.empty(T, d, dtype=torch.bfloat16, device=dev) if dH is None else dH
+        if dW is None:
+            dW = torch.empty(V, d, dtype=torch.float32, device=dev)
+        out = dict(loss=loss, dH=dH, dW=dW)
+        plain = (ent_coef == 0.0 and token_weight is None and not accumulate_dW and not want_aux)
+        args = [self.handle, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0), _ptr(tokens), _ptr(old_logp),
+                _ptr(ref_logp), _ptr(adv), _ptr(mask), T, d, V, eps_low, eps_high, beta, _ptr(loss), _ptr(dH),
+                _ptr(dW)]
+        if plain:
+            _check(self.lib.rl_policy_loss_fwd_bwd(*args), "rl_policy_loss_fwd_bwd")
+            return out
+        opts = rl_loss_opts()
+        opts.struct_size = ctypes.sizeof(rl_loss_opts)
+        opts.ent_coef = ent_coef
+        opts.token_weight = token_weight.data_ptr() if token_weight is not None else None
+        opts.accumulate_dW = int(accumulate_dW)
+        if want_aux:
+            out["logp"] = torch.empty(T, dtype=torch.float32, device=dev)
+            out["entropy"] = torch.empty(T, dtype=torch.float32, device=dev)
+            out["metrics"] = torch.empty(8, dtype=torch.float32, device=dev)
+            opts.logp_out = out["logp"].data_ptr()
+            opts.entropy_out = out["entropy"].data_ptr()
+            opts.metrics_out = out["metrics"].data_ptr()
+        _check(self.lib.rl_policy_loss_fwd_bwd_ex(*args, byref(opts)), "rl_policy_loss_fwd_bwd_ex")
+        return out
+
+    def rl_policy_loss_fwd_bwd_host(self, H_host, W, tokens_host, old_host, ref_host, adv_host, mask_host,
+                                    eps_low, eps_high, beta, ent_coef, dH, dW):
+        """Per-step inputs in (pinned) host memory; W, dH, dW on the device.  Returns (loss, metrics) floats."""
+        self._bind_stream()
+        T, d = H_host.shape
+        V = W.shape[0]
+        self.ensure_workspace(T, d, V, host=True)
+        loss = (c_float * 1)()
+        metrics = (c_float * 8)()
+        _check(self.lib.rl_policy_loss_fwd_bwd_host(
+            self.handle, _ptr(H_host), d, _ptr(W), W.stride(0), _ptr(tokens_host), _ptr(old_host), _ptr(ref_host),
+            _ptr(adv_host), _ptr(mask_host), T, d, V, eps_low, eps_high, beta, ent_coef,
+            ctypes.cast(loss, c_void_p), ctypes.cast(metrics, c_void_p), _ptr(dH), _ptr(dW)),
+            "rl_policy_loss_fwd_bwd_host")
+        return loss[0], list(metrics)
+
+    def rl_selftest_gemm(self, A, B, M, N, K, a_mn_major, b_mn_major, C=None, accumulate=False):
+        self._bind_stream()
+        if C is None:
+            C = torch.empty(M, N, dtype=torch.float32, device=A.device)
+        _check(self.lib.rl_selftest_gemm(self.handle, _ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn_major),
+                                         int(b_mn_major), int(accumulate)), "rl_selftest_gemm")
+        return C
+
+
+_default_ctx = {}
+
+
+def default_context(device=0):
+    if device not in _default_ctx:
+        _default_ctx[device] = Context(device)
+    return _default_ctx[device]
+
+
+def rl_grpo_advantages(rewards, group_size, **kw):
+    return default_context(rewards.device.index or 0).rl_grpo_advantages(rewards, group_size, **kw)
+
+
+def rl_token_logprobs(H, W, tokens, mask=None):
+    return default_context(H.device.index or 0).rl_token_logprobs(H, W, tokens, mask)
+
+
+def rl_policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta, **kw):
+    return default_context(W.device.index or 0).rl_policy_loss_fwd_bwd(
+        H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta, **kw)

@@ -1,0 +1,204 @@
+// Epilogue functors of the GEMM engine.  Each of the 128 epilogue threads owns one row of the
+// 128x256 accumulator tile and receives it in chunks of 32 consecutive columns.
+#pragma once
+#include <math_constants.h>
+
+#include "gemm_engine.cuh"
+
+namespace rlh {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ---------------------------------------------------------------------------------------------
+// Forward statistics (policy over the vocabulary, section 2.2): for its row and the vocabulary
+// range of the work unit, keeps the running maximum M, S = sum exp(z-M), A = sum exp(z-M) z and
+// the logit of the sampled token.  Logits never leave the chip; one float4 per (range, row) does.
+struct EpiStats {
+  struct Params {
+    const int* tokens_c;   // [rows] compact sampled-token ids
+    float4* partials;      // [n_ranges][part_stride]
+    int part_stride;
+    int V;
+  };
+  struct State {
+    float m, s, a, zy;
+    int y;
+  };
+  __device__ static __forceinline__ void begin_unit(const Params& p, State& st, int m_tile, int, int row_in_tile,
+                                                    int m_rows) {
+    st.m = -CUDART_INF_F;
+    st.s = 0.f;
+    st.a = 0.f;
+    st.zy = 0.f;
+    const int row = m_tile * BM + row_in_tile;
+    st.y = row < m_rows ? p.tokens_c[row] : -1;
+  }
+  __device__ static __forceinline__ void chunk(const Params& p, State& st, int, int n_tile, int c, int, int,
+                                               const float (&v)[32]) {
+    const int col0 = n_tile * BN + c * 32;
+    const int nvalid = p.V - col0;
+    if (nvalid <= 0) return;
+    float cmax = -CUDART_INF_F;
+    if (nvalid >= 32) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) cmax = i < nvalid ? fmaxf(cmax, v[i]) : cmax;
+    }
+    const float newm = fmaxf(st.m, cmax);
+    const float scale = exp2f((st.m - newm) * kLog2e);
+    const float mL = newm * kLog2e;
+    float cs = 0.f, ca = 0.f;
+    if (nvalid >= 32) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float e = exp2f(fmaf(v[i], kLog2e, -mL));
+        cs += e;
+        ca = fmaf(e, v[i], ca);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float e = i < nvalid ? exp2f(fmaf(v[i], kLog2e, -mL)) : 0.f;
+        cs += e;
+        ca = fmaf(e, v[i], ca);
+      }
+    }
+    st.s = fmaf(st.s, scale, cs);
+    st.a = fmaf(st.a, scale, ca);
+    st.m = newm;
+    const unsigned rel = (unsigned)(st.y - col0);
+    if (rel < 32u && (int)rel < nvalid) {
+      float z = 0.f;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) z = (rel == (unsigned)i) ? v[i] : z;
+      st.zy = z;
+    }
+  }
+  __device__ static __forceinline__ void end_unit(const Params& p, State& st, int m_tile, int nr, int row_in_tile,
+                                                  int m_rows) {
+    const int row = m_tile * BM + row_in_tile;
+    if (row < m_rows) p.partials[(size_t)nr * p.part_stride + row] = make_float4(st.m, st.s, st.a, st.zy);
+  }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Gradient with respect to the logits for one slab of rows x vocabulary columns, rounded to
+// bf16 and written to the slab scratch (row-major, ldG):
+//   g_tj = cp_t (p_tj - 1[j = y_t]) + ce_t p_tj (log p_tj + Ent_t),  p_tj = exp(z_tj - lse_t)
+// cp_t = -w_t dloss_t/dlogp_t and ce_t = w_t ent_coef come from the per-token loss kernel.
+// Rows past the valid rows of the slab and columns past V are written as zero.
+struct EpiGrad {
+  struct Params {
+    const int* tokens_c;
+    const float* lse;
+    const float* ent;
+    const float* cp;
+    const float* ce;
+    __nv_bfloat16* G;
+    int ldG;
+    int V;
+    int vocab_base;  // global column of the slab's column 0
+    int row_base;    // compact row of the slab's row 0
+  };
+  struct State {
+    float lse, ent, cp, ce;
+    int y;
+    bool valid;
+  };
+  __device__ static __forceinline__ void begin_unit(const Params& p, State& st, int m_tile, int, int row_in_tile,
+                                                    int m_rows) {
+    const int rl = m_tile * BM + row_in_tile;
+    st.valid = rl < m_rows;
+    const int gr = p.row_base + rl;
+    st.lse = st.valid ? p.lse[gr] : 0.f;
+    st.ent = st.valid ? p.ent[gr] : 0.f;
+    st.cp = st.valid ? p.cp[gr] : 0.f;
+    st.ce = st.valid ? p.ce[gr] : 0.f;
+    st.y = st.valid ? p.tokens_c[gr] : -1;
+  }
+  __device__ static __forceinline__ void chunk(const Params& p, State& st, int m_tile, int n_tile, int c,
+                                               int row_in_tile, int, const float (&v)[32]) {
+    const int col_l = n_tile * BN + c * 32;
+    const int col_g = p.vocab_base + col_l;
+    const int nvalid = p.V - col_g;
+    float g[32];
+    if (!st.valid || nvalid <= 0) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) g[i] = 0.f;
+    } else {
+      if (st.ce == 0.f) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) g[i] = st.cp * exp2f((v[i] - st.lse) * kLog2e);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float lp = v[i] - st.lse;
+          g[i] = exp2f(lp * kLog2e) * fmaf(st.ce, lp + st.ent, st.cp);
+        }
+      }
+      const unsigned rel = (unsigned)(st.y - col_g);
+      if (rel < 32u) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) g[i] = (rel == (unsigned)i) ? g[i] - st.cp : g[i];
+      }
+      if (nvalid < 32) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) g[i] = i < nvalid ? g[i] : 0.f;
+      }
+    }
+    const int rl = m_tile * BM + row_in_tile;
+    uint4* dst = reinterpret_cast<uint4*>(p.G + (size_t)rl * p.ldG + col_l);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint4 o;
+      __nv_bfloat162 b0 = __floats2bfloat162_rn(g[8 * j + 0], g[8 * j + 1]);
+      __nv_bfloat162 b1 = __floats2bfloat162_rn(g[8 * j + 2], g[8 * j + 3]);
+      __nv_bfloat162 b2 = __floats2bfloat162_rn(g[8 * j + 4], g[8 * j + 5]);
+      __nv_bfloat162 b3 = __floats2bfloat162_rn(g[8 * j + 6], g[8 * j + 7]);
+      o.x = *reinterpret_cast<uint32_t*>(&b0);
+      o.y = *reinterpret_cast<uint32_t*>(&b1);
+      o.z = *reinterpret_cast<uint32_t*>(&b2);
+      o.w = *reinterpret_cast<uint32_t*>(&b3);
+      dst[j] = o;
+    }
+  }
+  __device__ static __forceinline__ void end_unit(const Params&, State&, int, int, int, int) {}
+};
+
+// ---------------------------------------------------------------------------------------------
+// Plain fp32 output tile: C[row_base + row, col] = acc (+ previous value when accumulating).
+struct EpiAcc {
+  struct Params {
+    float* C;
+    long long ldc;
+    int n_cols;
+    int accumulate;
+    int row_base;
+  };
+  struct State {};
+  __device__ static __forceinline__ void begin_unit(const Params&, State&, int, int, int, int) {}
+  __device__ static __forceinline__ void chunk(const Params& p, State&, int m_tile, int n_tile, int c,
+                                               int row_in_tile, int m_rows, const float (&v)[32]) {
+    const int rl = m_tile * BM + row_in_tile;
+    const int col0 = n_tile * BN + c * 32;
+    if (rl >= m_rows || col0 >= p.n_cols) return;
+    float4* dst = reinterpret_cast<float4*>(p.C + (size_t)(p.row_base + rl) * p.ldc + col0);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (col0 + 4 * j < p.n_cols) {
+        float4 x = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        if (p.accumulate) {
+          const float4 o = dst[j];
+          x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w;
+        }
+        dst[j] = x;
+      }
+    }
+  }
+  __device__ static __forceinline__ void end_unit(const Params&, State&, int, int, int, int) {}
+};
+
+}  // namespace rlh

@@ -1,0 +1,546 @@
+// C ABI of the fused LM-head log-probability + GRPO policy-loss library: argument checks,
+// workspace layout, tensor-map construction and the launch sequences.  All arithmetic of the
+// path runs in the kernels of gemm_engine.cuh / epilogues.cuh / small_kernels.cuh.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "rlhead.h"
+#include "small_kernels.cuh"
+
+using namespace rlh;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct rl_ctx {
+  int device;
+  int n_sm;
+  cudaStream_t stream;
+  DevStatus* dstatus;  // device
+  void* ws;
+  size_t ws_bytes;
+  EncodeTiledFn encode;
+};
+
+namespace {
+
+constexpr int kSlabRowsMax = 32768;        // rows of one gradient slab
+constexpr int kSlabColsMax = 74 * 128;     // vocabulary columns of one gradient slab (37 tiles of 256)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+  int Tpad, Ts, Vs;
+  size_t row_map, tokens_c, lse_c, ent_c, cp_c, ce_c, partials, block_sums, Hc, G, dH_acc, staging, total;
+};
+
+// staging_T > 0 adds room for host-call inputs (H, tokens, old, ref, adv, mask).
+WsLayout ws_layout(int64_t T, int64_t d, int64_t V, bool host_staging) {
+  WsLayout L;
+  L.Tpad = (int)align_up((size_t)(T > 0 ? T : 1), 128);
+  L.Ts = L.Tpad < kSlabRowsMax ? L.Tpad : kSlabRowsMax;
+  const int Vpad = (int)align_up((size_t)V, 256);
+  L.Vs = Vpad < kSlabColsMax ? Vpad : kSlabColsMax;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 1024); return at; };
+  L.row_map = take((size_t)L.Tpad * 4);
+  L.tokens_c = take((size_t)L.Tpad * 4);
+  L.lse_c = take((size_t)L.Tpad * 4);
+  L.ent_c = take((size_t)L.Tpad * 4);
+  L.cp_c = take((size_t)L.Tpad * 4);
+  L.ce_c = take((size_t)L.Tpad * 4);
+  L.partials = take((size_t)kMaxSplit * L.Tpad * sizeof(float4));
+  L.block_sums = take((size_t)1024 * kLossSums * sizeof(double));
+  L.Hc = take((size_t)L.Tpad * d * 2);
+  L.G = take((size_t)L.Ts * L.Vs * 2);
+  L.dH_acc = take((size_t)L.Ts * d * 4);
+  L.staging = o;
+  if (host_staging) {
+    take((size_t)T * d * 2);  // H
+    take((size_t)T * 4);      // tokens
+    take((size_t)T * 4);      // old
+    take((size_t)T * 4);      // ref
+    take((size_t)T * 4);      // adv
+    take((size_t)T);          // mask
+    take(64);                 // loss + metrics
+  }
+  L.total = o;
+  return L;
+}
+
+// K-major operand: global tensor [rows, k] with k contiguous, row stride ld elements.
+bool map_kmajor(rl_ctx* c, CUtensorMap* m, const void* base, uint64_t rows, uint64_t k, uint64_t ld,
+                uint32_t box_rows) {
+  cuuint64_t dims[2] = {k, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t es[2] = {1, 1};
+  return c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// MN-major operand: global tensor [k, mn] with mn contiguous (a multiple of 64), row stride ld.
+// Seen by TMA as {64, k, mn/64} so that one box {64, 64, chunks} fetches `chunks` 64-wide panels.
+bool map_mnmajor(rl_ctx* c, CUtensorMap* m, const void* base, uint64_t k_rows, uint64_t mn, uint64_t ld,
+                 uint32_t chunks) {
+  cuuint64_t dims[3] = {64, k_rows, mn / 64};
+  cuuint64_t strides[2] = {ld * 2, 128};
+  cuuint32_t box[3] = {64, 64, chunks};
+  cuuint32_t es[3] = {1, 1, 1};
+  return c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <class Epi, int A_MN, int B_MN>
+cudaError_t set_smem_attr() {
+  return cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kGemmSmemBytes);
+}
+
+template <class Epi, int A_MN, int B_MN>
+void launch_gemm(rl_ctx* c, const CUtensorMap& a, const CUtensorMap& b, const GemmShape& sh,
+                 const typename Epi::Params& ep) {
+  gemm_kernel<Epi, A_MN, B_MN><<<c->n_sm, kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, sh, ep, c->dstatus);
+}
+
+rl_status check_hw(const void* H, int64_t ldH, const void* W, int64_t ldW, int64_t T, int64_t d, int64_t V) {
+  if (T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
+  if (T > 0 && (!H || !W)) return RL_ERR_INVALID_ARG;
+  if (d % 64 != 0) return RL_ERR_SHAPE;
+  if (T >= (int64_t(1) << 30) || V >= (int64_t(1) << 30)) return RL_ERR_SHAPE;
+  if (ldH < d || ldW < d) return RL_ERR_SHAPE;
+  if (ldH % 8 != 0 || ldW % 8 != 0) return RL_ERR_ALIGNMENT;
+  if ((reinterpret_cast<uintptr_t>(H) & 15) || (reinterpret_cast<uintptr_t>(W) & 15)) return RL_ERR_ALIGNMENT;
+  return RL_OK;
+}
+
+rl_status check_ws(rl_ctx* c, const WsLayout& L) {
+  if (!c->ws || c->ws_bytes < L.total) return RL_ERR_WORKSPACE;
+  return RL_OK;
+}
+
+inline rl_status cuda_ok() { return cudaGetLastError() == cudaSuccess ? RL_OK : RL_ERR_CUDA; }
+
+// Mask scan + row compaction + forward statistics.  Leaves per-range partials in the workspace.
+rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, const void* W, int64_t ldW,
+                      const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d, int64_t V, int* n_tiles_out) {
+  char* ws = static_cast<char*>(c->ws);
+  int* row_map = reinterpret_cast<int*>(ws + L.row_map);
+  int* tokens_c = reinterpret_cast<int*>(ws + L.tokens_c);
+  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + L.Hc);
+  mask_scan_kernel<<<1, kScanThreads, 0, c->stream>>>(mask, (int)T, row_map, c->dstatus);
+  gather_rows_kernel<<<c->n_sm * 4, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16*>(H), ldH, (int)d, row_map,
+                                                         tokens, (int)V, Hc, tokens_c, c->dstatus);
+  CUtensorMap tmA, tmB;
+  if (!map_kmajor(c, &tmA, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM)) return RL_ERR_CUDA;
+  if (!map_kmajor(c, &tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, BN)) return RL_ERR_CUDA;
+  GemmShape sh;
+  memset(&sh, 0, sizeof(sh));
+  sh.n_valid = &c->dstatus->n_valid;
+  sh.m_rows_cap = L.Tpad;
+  sh.m_dyn = 1;
+  sh.k_cap = (int)d;
+  sh.n_tiles = (int)((V + BN - 1) / BN);
+  sh.n_range = 0;  // split chosen on the device from the number of valid rows
+  EpiStats::Params ep;
+  ep.tokens_c = tokens_c;
+  ep.partials = reinterpret_cast<float4*>(ws + L.partials);
+  ep.part_stride = L.Tpad;
+  ep.V = (int)V;
+  launch_gemm<EpiStats, 0, 0>(c, tmA, tmB, sh, ep);
+  *n_tiles_out = sh.n_tiles;
+  return cuda_ok();
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rl_status_string(rl_status s) {
+  switch (s) {
+    case RL_OK: return "ok";
+    case RL_ERR_INVALID_ARG: return "invalid argument";
+    case RL_ERR_SHAPE: return "unsupported shape";
+    case RL_ERR_ALIGNMENT: return "pointer or leading dimension not aligned for TMA";
+    case RL_ERR_WORKSPACE: return "workspace missing or too small";
+    case RL_ERR_CUDA: return "CUDA call failed";
+    case RL_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
+    case RL_ERR_TOKEN_RANGE: return "token id outside [0,V) on a valid row";
+    case RL_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
+  }
+  return "unknown status";
+}
+
+rl_status rl_create(rl_ctx** out, int device) {
+  if (!out) return RL_ERR_INVALID_ARG;
+  *out = nullptr;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return RL_ERR_CUDA;
+  if (prop.major != 10) return RL_ERR_UNSUPPORTED_ARCH;
+  if (cudaSetDevice(device) != cudaSuccess) return RL_ERR_CUDA;
+  rl_ctx* c = new (std::nothrow) rl_ctx();
+  if (!c) return RL_ERR_CUDA;
+  c->device = device;
+  c->n_sm = prop.multiProcessorCount;
+  c->stream = nullptr;
+  c->ws = nullptr;
+  c->ws_bytes = 0;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    delete c;
+    return RL_ERR_CUDA;
+  }
+  c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(&c->dstatus, sizeof(DevStatus)) != cudaSuccess) { delete c; return RL_ERR_CUDA; }
+  cudaMemset(c->dstatus, 0, sizeof(DevStatus));
+  bool ok = set_smem_attr<EpiStats, 0, 0>() == cudaSuccess && set_smem_attr<EpiGrad, 0, 0>() == cudaSuccess &&
+            set_smem_attr<EpiAcc, 0, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 0, 1>() == cudaSuccess &&
+            set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess;
+  if (!ok) { cudaFree(c->dstatus); delete c; return RL_ERR_CUDA; }
+  *out = c;
+  return RL_OK;
+}
+
+rl_status rl_destroy(rl_ctx* c) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  cudaFree(c->dstatus);
+  delete c;
+  return RL_OK;
+}
+
+rl_status rl_set_stream(rl_ctx* c, void* s) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  c->stream = static_cast<cudaStream_t>(s);
+  return RL_OK;
+}
+
+rl_status rl_workspace_bytes(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t* bytes) {
+  if (!c || !bytes || T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
+  *bytes = ws_layout(T, d, V, false).total;
+  return RL_OK;
+}
+
+rl_status rl_workspace_bytes_host(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t* bytes) {
+  if (!c || !bytes || T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
+  *bytes = ws_layout(T, d, V, true).total;
+  return RL_OK;
+}
+
+rl_status rl_set_workspace(rl_ctx* c, void* p, size_t bytes) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  if (p && (reinterpret_cast<uintptr_t>(p) & 255)) return RL_ERR_ALIGNMENT;
+  c->ws = p;
+  c->ws_bytes = p ? bytes : 0;
+  return RL_OK;
+}
+
+rl_status rl_last_device_status(rl_ctx* c, int32_t* detail) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  DevStatus h;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return RL_ERR_CUDA;
+  if (cudaMemcpy(&h, c->dstatus, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return RL_ERR_CUDA;
+  if (detail) *detail = h.detail;
+  if (h.code != 0) {
+    int zero[2] = {0, 0};
+    cudaMemcpy(c->dstatus, zero, sizeof(zero), cudaMemcpyHostToDevice);
+  }
+  return static_cast<rl_status>(h.code);
+}
+
+rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, int group_size, int ddof,
+                                float eps_std, const int32_t* seq_offsets, int64_t T, float* adv_seq,
+                                float* adv_tok) {
+  if (!c || n_seq < 0 || (n_seq > 0 && (!rewards || !adv_seq))) return RL_ERR_INVALID_ARG;
+  if ((ddof != 0 && ddof != 1) || !(eps_std >= 0.f)) return RL_ERR_INVALID_ARG;
+  if ((adv_tok != nullptr) != (seq_offsets != nullptr) || T < 0) return RL_ERR_INVALID_ARG;
+  if (group_size < 2 || n_seq % group_size != 0 || n_seq >= (int64_t(1) << 31)) return RL_ERR_SHAPE;
+  if (n_seq == 0) return RL_OK;
+  const int n_groups = (int)(n_seq / group_size);
+  const int warps = 8;
+  grpo_adv_kernel<<<(n_groups + warps - 1) / warps, warps * 32, 0, c->stream>>>(rewards, n_groups, group_size, ddof,
+                                                                                eps_std, adv_seq);
+  if (adv_tok) {
+    if (T > 0 && cudaMemsetAsync(adv_tok, 0, (size_t)T * 4, c->stream) != cudaSuccess) return RL_ERR_CUDA;
+    int blocks = (int)(n_seq < 4096 ? n_seq : 4096);
+    broadcast_adv_kernel<<<blocks, 256, 0, c->stream>>>(adv_seq, seq_offsets, (int)n_seq, adv_tok);
+  }
+  return cuda_ok();
+}
+
+rl_status rl_grpo_advantages(rl_ctx* c, const float* rewards, int64_t n_seq, int group_size, float* adv_seq) {
+  return rl_grpo_advantages_ex(c, rewards, n_seq, group_size, 1, 1e-6f, nullptr, 0, adv_seq, nullptr);
+}
+
+rl_status rl_token_logprobs(rl_ctx* c, const void* H, int64_t ldH, const void* W, int64_t ldW, const int32_t* tokens,
+                            const uint8_t* mask, int64_t T, int64_t d, int64_t V, float* logp, float* entropy,
+                            float* lse) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  rl_status s = check_hw(H, ldH, W, ldW, T, d, V);
+  if (s != RL_OK) return s;
+  if (T == 0) return RL_OK;
+  if (!tokens || !logp) return RL_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(T, d, V, false);
+  if ((s = check_ws(c, L)) != RL_OK) return s;
+  char* ws = static_cast<char*>(c->ws);
+  cudaMemsetAsync(logp, 0, (size_t)T * 4, c->stream);
+  if (entropy) cudaMemsetAsync(entropy, 0, (size_t)T * 4, c->stream);
+  if (lse) cudaMemsetAsync(lse, 0, (size_t)T * 4, c->stream);
+  int n_tiles = 0;
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &n_tiles)) != RL_OK) return s;
+  LossParams p;
+  memset(&p, 0, sizeof(p));
+  p.partials = reinterpret_cast<const float4*>(ws + L.partials);
+  p.part_stride = L.Tpad;
+  p.n_tiles = n_tiles;
+  p.n_ctas = c->n_sm;
+  p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
+  p.with_loss = 0;
+  p.lse_c = reinterpret_cast<float*>(ws + L.lse_c);
+  p.ent_c = reinterpret_cast<float*>(ws + L.ent_c);
+  p.logp_out = logp;
+  p.ent_out = entropy;
+  p.lse_out = lse;
+  int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
+  if (blocks > 1024) blocks = 1024;
+  combine_loss_kernel<<<blocks, kLossThreads, 0, c->stream>>>(p, c->dstatus);
+  return cuda_ok();
+}
+
+rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const void* W, int64_t ldW,
+                                    const int32_t* tokens, const float* old_logp, const float* ref_logp,
+                                    const float* adv, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
+                                    float eps_low, float eps_high, float beta, float* loss, void* dH, float* dW,
+                                    const rl_loss_opts* opts) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  rl_status s = check_hw(H, ldH, W, ldW, T, d, V);
+  if (s != RL_OK) return s;
+  if (!(eps_low >= 0.f && eps_low < 1.f) || !(eps_high >= 0.f) || !(beta >= 0.f)) return RL_ERR_INVALID_ARG;
+  if (!loss || !dW || !W) return RL_ERR_INVALID_ARG;
+  if (T > 0 && (!tokens || !old_logp || !adv || !dH)) return RL_ERR_INVALID_ARG;
+  if (beta != 0.f && T > 0 && !ref_logp) return RL_ERR_INVALID_ARG;
+  rl_loss_opts o;
+  memset(&o, 0, sizeof(o));
+  if (opts) {
+    if (opts->struct_size < sizeof(size_t) + sizeof(float) || opts->struct_size > sizeof(rl_loss_opts))
+      return RL_ERR_INVALID_ARG;
+    memcpy(&o, opts, opts->struct_size);
+  }
+  if (!(o.ent_coef >= 0.f)) return RL_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dH) & 15) || (reinterpret_cast<uintptr_t>(dW) & 15)) return RL_ERR_ALIGNMENT;
+  const WsLayout L = ws_layout(T, d, V, false);
+  if ((s = check_ws(c, L)) != RL_OK) return s;
+  char* ws = static_cast<char*>(c->ws);
+  cudaStream_t st = c->stream;
+
+  if (T == 0) {
+    cudaMemsetAsync(loss, 0, 4, st);
+    if (!o.accumulate_dW) cudaMemsetAsync(dW, 0, (size_t)V * d * 4, st);
+    if (o.metrics_out) cudaMemsetAsync(o.metrics_out, 0, 32, st);
+    return cuda_ok();
+  }
+  cudaMemsetAsync(dH, 0, (size_t)T * d * 2, st);
+  if (o.logp_out) cudaMemsetAsync(o.logp_out, 0, (size_t)T * 4, st);
+  if (o.entropy_out) cudaMemsetAsync(o.entropy_out, 0, (size_t)T * 4, st);
+
+  // ---- forward: statistics per (row, vocabulary range)
+  int n_tiles = 0;
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &n_tiles)) != RL_OK) return s;
+
+  // ---- merge + per-token loss, coefficients of the backward pass
+  LossParams p;
+  memset(&p, 0, sizeof(p));
+  p.partials = reinterpret_cast<const float4*>(ws + L.partials);
+  p.part_stride = L.Tpad;
+  p.n_tiles = n_tiles;
+  p.n_ctas = c->n_sm;
+  p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
+  p.old_logp = old_logp;
+  p.ref_logp = ref_logp;
+  p.adv = adv;
+  p.token_weight = o.token_weight;
+  p.eps_low = eps_low;
+  p.eps_high = eps_high;
+  p.beta = beta;
+  p.ent_coef = o.ent_coef;
+  p.with_loss = 1;
+  p.lse_c = reinterpret_cast<float*>(ws + L.lse_c);
+  p.ent_c = reinterpret_cast<float*>(ws + L.ent_c);
+  p.cp_c = reinterpret_cast<float*>(ws + L.cp_c);
+  p.ce_c = reinterpret_cast<float*>(ws + L.ce_c);
+  p.logp_out = o.logp_out;
+  p.ent_out = o.entropy_out;
+  p.block_sums = reinterpret_cast<double*>(ws + L.block_sums);
+  int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
+  if (blocks > 1024) blocks = 1024;
+  combine_loss_kernel<<<blocks, kLossThreads, 0, st>>>(p, c->dstatus);
+  finalize_loss_kernel<<<1, 32, 0, st>>>(p.block_sums, blocks, loss, o.metrics_out, c->dstatus);
+
+  // ---- backward, one (row slab x vocabulary slab) at a time
+  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + L.Hc);
+  __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(ws + L.G);
+  float* dH_acc = reinterpret_cast<float*>(ws + L.dH_acc);
+  const int* row_map = reinterpret_cast<const int*>(ws + L.row_map);
+  const int* n_valid = &c->dstatus->n_valid;
+
+  CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn;
+  bool ok = map_kmajor(c, &tmHc_k, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM) &&
+            map_kmajor(c, &tmW_k, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, BN) &&
+            map_kmajor(c, &tmG_k, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM) &&
+            map_mnmajor(c, &tmW_mn, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, BN / 64) &&
+            map_mnmajor(c, &tmG_mn, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM / 64) &&
+            map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BN / 64);
+  if (!ok) return RL_ERR_CUDA;
+
+  const int n_row_slabs = (L.Tpad + L.Ts - 1) / L.Ts;
+  const int n_col_slabs = (int)((V + L.Vs - 1) / L.Vs);
+  const int d_tiles = (int)((d + BN - 1) / BN);
+  for (int r = 0; r < n_row_slabs; ++r) {
+    const int row_base = r * L.Ts;
+    const int rows_cap = (L.Tpad - row_base) < L.Ts ? (L.Tpad - row_base) : L.Ts;
+    for (int cs = 0; cs < n_col_slabs; ++cs) {
+      const int vocab_base = cs * L.Vs;
+      const int cols = (int)((V - vocab_base) < L.Vs ? (V - vocab_base) : L.Vs);
+      // (1) recompute the logits of the slab, write G = dloss/dlogits as bf16
+      {
+        GemmShape sh;
+        memset(&sh, 0, sizeof(sh));
+        sh.n_valid = n_valid;
+        sh.m_rows_cap = rows_cap; sh.m_dyn = 1; sh.m_dyn_off = row_base;
+        sh.k_cap = (int)d;
+        sh.n_tiles = (cols + BN - 1) / BN;
+        sh.n_range = 1;
+        sh.a_mn_off = row_base;
+        sh.b_mn_off = vocab_base;
+        EpiGrad::Params ep;
+        ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
+        ep.lse = p.lse_c; ep.ent = p.ent_c; ep.cp = p.cp_c; ep.ce = p.ce_c;
+        ep.G = G; ep.ldG = L.Vs; ep.V = (int)V; ep.vocab_base = vocab_base; ep.row_base = row_base;
+        launch_gemm<EpiGrad, 0, 0>(c, tmHc_k, tmW_k, sh, ep);
+      }
+      // (2) dH_slab (+)= G * W_slab        [rows x d], K = vocabulary columns of the slab
+      {
+        GemmShape sh;
+        memset(&sh, 0, sizeof(sh));
+        sh.n_valid = n_valid;
+        sh.m_rows_cap = rows_cap; sh.m_dyn = 1; sh.m_dyn_off = row_base;
+        sh.k_cap = cols;
+        sh.n_tiles = d_tiles;
+        sh.n_range = 1;
+        sh.b_k_off = vocab_base;
+        EpiAcc::Params ep;
+        ep.C = dH_acc; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0;
+        launch_gemm<EpiAcc, 0, 1>(c, tmG_k, tmW_mn, sh, ep);
+      }
+      // (3) dW_slab (+)= G^T * H_slab      [vocabulary rows x d], K = valid rows of the slab
+      {
+        GemmShape sh;
+        memset(&sh, 0, sizeof(sh));
+        sh.n_valid = n_valid;
+        sh.m_rows_cap = cols;
+        sh.k_cap = rows_cap; sh.k_dyn = 1; sh.k_dyn_off = row_base;
+        sh.n_tiles = d_tiles;
+        sh.n_range = 1;
+        sh.skip_if_k0 = (r > 0 || o.accumulate_dW) ? 1 : 0;
+        sh.b_k_off = row_base;
+        EpiAcc::Params ep;
+        ep.C = dW; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
+        ep.row_base = vocab_base;
+        launch_gemm<EpiAcc, 1, 1>(c, tmG_mn, tmHc_mn, sh, ep);
+      }
+    }
+    scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
+                                                   static_cast<__nv_bfloat16*>(dH), c->dstatus);
+  }
+  return cuda_ok();
+}
+
+rl_status rl_policy_loss_fwd_bwd(rl_ctx* c, const void* H, int64_t ldH, const void* W, int64_t ldW,
+                                 const int32_t* tokens, const float* old_logp, const float* ref_logp,
+                                 const float* adv, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
+                                 float eps_low, float eps_high, float beta, float* loss, void* dH, float* dW) {
+  return rl_policy_loss_fwd_bwd_ex(c, H, ldH, W, ldW, tokens, old_logp, ref_logp, adv, mask, T, d, V, eps_low,
+                                   eps_high, beta, loss, dH, dW, nullptr);
+}
+
+rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* c, const void* H_host, int64_t ldH, const void* W, int64_t ldW,
+                                      const int32_t* tokens_host, const float* old_host, const float* ref_host,
+                                      const float* adv_host, const uint8_t* mask_host, int64_t T, int64_t d,
+                                      int64_t V, float eps_low, float eps_high, float beta, float ent_coef,
+                                      float* loss_host, float* metrics_host, void* dH, float* dW) {
+  if (!c || !loss_host) return RL_ERR_INVALID_ARG;
+  if (T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
+  if (T > 0 && (!H_host || !tokens_host || !old_host || !adv_host)) return RL_ERR_INVALID_ARG;
+  if (ldH != d) return RL_ERR_SHAPE;  // host rows are copied as one block
+  const WsLayout L = ws_layout(T, d, V, true);
+  rl_status s = check_ws(c, L);
+  if (s != RL_OK) return s;
+  char* ws = static_cast<char*>(c->ws);
+  size_t o = L.staging;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 1024); return ws + at; };
+  void* dH_in = take((size_t)T * d * 2);
+  int32_t* d_tok = reinterpret_cast<int32_t*>(take((size_t)T * 4));
+  float* d_old = reinterpret_cast<float*>(take((size_t)T * 4));
+  float* d_ref = reinterpret_cast<float*>(take((size_t)T * 4));
+  float* d_adv = reinterpret_cast<float*>(take((size_t)T * 4));
+  uint8_t* d_mask = reinterpret_cast<uint8_t*>(take((size_t)T));
+  float* d_out = reinterpret_cast<float*>(take(64));
+  cudaStream_t st = c->stream;
+  if (T > 0) {
+    cudaMemcpyAsync(dH_in, H_host, (size_t)T * d * 2, cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(d_tok, tokens_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(d_old, old_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
+    if (ref_host) cudaMemcpyAsync(d_ref, ref_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(d_adv, adv_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
+    if (mask_host) cudaMemcpyAsync(d_mask, mask_host, (size_t)T, cudaMemcpyHostToDevice, st);
+  }
+  rl_loss_opts opts;
+  memset(&opts, 0, sizeof(opts));
+  opts.struct_size = sizeof(opts);
+  opts.ent_coef = ent_coef;
+  opts.metrics_out = d_out + 8;
+  s = rl_policy_loss_fwd_bwd_ex(c, dH_in, d, W, ldW, d_tok, d_old, ref_host ? d_ref : nullptr, d_adv,
+                                mask_host ? d_mask : nullptr, T, d, V, eps_low, eps_high, beta, d_out, dH, dW,
+                                &opts);
+  if (s != RL_OK) return s;
+  float h_out[16];
+  if (cudaMemcpyAsync(h_out, d_out, sizeof(h_out), cudaMemcpyDeviceToHost, st) != cudaSuccess) return RL_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return RL_ERR_CUDA;
+  loss_host[0] = h_out[0];
+  if (metrics_host) memcpy(metrics_host, h_out + 8, 32);
+  return RL_OK;
+}
+
+rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,
+                           int a_mn, int b_mn, int accumulate) {
+  if (!c || !A || !B || !C || M <= 0 || N <= 0 || K <= 0) return RL_ERR_INVALID_ARG;
+  if (M % 128 != 0 || N % 256 != 0 || K % 8 != 0) return RL_ERR_SHAPE;
+  CUtensorMap ta, tb;
+  bool ok = a_mn ? map_mnmajor(c, &ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)M, BM / 64)
+                 : map_kmajor(c, &ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM);
+  ok = ok && (b_mn ? map_mnmajor(c, &tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)N, BN / 64)
+                   : map_kmajor(c, &tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN));
+  if (!ok) return RL_ERR_CUDA;
+  GemmShape sh;
+  memset(&sh, 0, sizeof(sh));
+  sh.m_rows_cap = (int)M;
+  sh.k_cap = (int)K;
+  sh.n_tiles = (int)(N / BN);
+  sh.n_range = 1;
+  EpiAcc::Params ep;
+  ep.C = C; ep.ldc = N; ep.n_cols = (int)N; ep.accumulate = accumulate; ep.row_base = 0;
+  if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, ta, tb, sh, ep);
+  else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, ta, tb, sh, ep);
+  else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, ta, tb, sh, ep);
+  else launch_gemm<EpiAcc, 1, 1>(c, ta, tb, sh, ep);
+  return cuda_ok();
+}
+
+}  // extern "C"

@@ -1,0 +1,287 @@
+// O(T) and O(B) kernels around the tensor-core passes: mask scan / row compaction
+// (padding-free execution), GRPO advantages, merge of the per-range softmax statistics,
+// per-token loss arithmetic with a deterministic two-stage reduction, and the final
+// conversion of dH.  All of them are bandwidth- or latency-bound; loads are coalesced and
+// vectorised where a row is wide enough to matter.
+#pragma once
+#include "epilogues.cuh"
+
+namespace rlh {
+
+// ------------------------------------------------------------------------------------------
+// Mask scan: row_map[i] = index of the i-th row with mask != 0 (ascending), n_valid = their
+// number.  One block; each thread scans a contiguous piece.
+constexpr int kScanThreads = 1024;
+__global__ void __launch_bounds__(kScanThreads) mask_scan_kernel(const uint8_t* __restrict__ mask, int T,
+                                                                 int* __restrict__ row_map, DevStatus* st) {
+  __shared__ int warp_sums[32];
+  __shared__ int total;
+  const int tid = threadIdx.x;
+  const int per = (T + kScanThreads - 1) / kScanThreads;
+  const int begin = min(tid * per, T), end = min(begin + per, T);
+  int cnt = 0;
+  if (mask) {
+    for (int i = begin; i < end; ++i) cnt += mask[i] != 0;
+  } else {
+    cnt = end - begin;
+  }
+  // block exclusive scan of cnt
+  int incl = cnt;
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums[lane];
+    int wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int v = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += v;
+    }
+    warp_sums[lane] = wi - w;
+    if (lane == 31) total = wi;
+  }
+  __syncthreads();
+  int pos = warp_sums[warp] + incl - cnt;
+  for (int i = begin; i < end; ++i) {
+    if (!mask || mask[i] != 0) row_map[pos++] = i;
+  }
+  if (tid == 0) st->n_valid = total;
+}
+
+// ------------------------------------------------------------------------------------------
+// Row compaction: Hc[i,:] = H[row_map[i],:] for i < n_valid, zero rows up to the next multiple
+// of 128 (so that tensor-core tiles never see stale data), compact token ids, and the
+// token-range check.  One warp per row, 16-byte loads.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* __restrict__ H, long long ldH, int d,
+                                                          const int* __restrict__ row_map,
+                                                          const int* __restrict__ tokens, int V,
+                                                          __nv_bfloat16* __restrict__ Hc,
+                                                          int* __restrict__ tokens_c, DevStatus* st) {
+  const int n = st->n_valid;
+  const int n_pad = (n + 127) / 128 * 128;
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  const int vec_per_row = d / 8;
+  for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < n_pad; i += gridDim.x * warps_per_block) {
+    uint4* dst = reinterpret_cast<uint4*>(Hc + (size_t)i * d);
+    if (i < n) {
+      const int r = row_map[i];
+      const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)r * ldH);
+      for (int v = lane; v < vec_per_row; v += 32) dst[v] = __ldg(src + v);
+      if (lane == 0) {
+        const int y = tokens[r];
+        tokens_c[i] = y;
+        if (y < 0 || y >= V) latch_status(st, kStatusTokenRange, r);
+      }
+    } else {
+      for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+      if (lane == 0) tokens_c[i] = -1;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// GRPO advantages (section 4.2 group-based normalisation): one warp per group of G consecutive
+// rewards, shuffle reductions for mean, centred sum of squares and the all-equal test.
+__global__ void __launch_bounds__(256) grpo_adv_kernel(const float* __restrict__ rewards, int n_groups, int G,
+                                                       int ddof, float eps_std, float* __restrict__ adv_seq) {
+  const int lane = threadIdx.x & 31;
+  const int g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (g >= n_groups) return;
+  const float* r = rewards + (size_t)g * G;
+  float sum = 0.f, mx = -CUDART_INF_F, mn = CUDART_INF_F;
+  for (int i = lane; i < G; i += 32) {
+    const float x = r[i];
+    sum += x;
+    mx = fmaxf(mx, x);
+    mn = fminf(mn, x);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+  }
+  const float mu = sum / (float)G;
+  float ss = 0.f;
+  for (int i = lane; i < G; i += 32) {
+    const float c = r[i] - mu;
+    ss = fmaf(c, c, ss);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float sigma = sqrtf(ss / (float)(G - ddof));
+  const float inv = (mx == mn) ? 0.f : 1.f / (sigma + eps_std);
+  for (int i = lane; i < G; i += 32) adv_seq[(size_t)g * G + i] = (mx == mn) ? 0.f : (r[i] - mu) * inv;
+}
+
+// Broadcast of the per-response advantage to the rows of the response (outcome supervision).
+__global__ void __launch_bounds__(256) broadcast_adv_kernel(const float* __restrict__ adv_seq,
+                                                            const int* __restrict__ seq_offsets, int n_seq,
+                                                            float* __restrict__ adv_tok) {
+  for (int s = blockIdx.x; s < n_seq; s += gridDim.x) {
+    const int b = seq_offsets[s], e = seq_offsets[s + 1];
+    const float a = adv_seq[s];
+    for (int t = b + threadIdx.x; t < e; t += blockDim.x) adv_tok[t] = a;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Merge of the per-range statistics and the per-token loss arithmetic (Eq. 6 with the clipped
+// surrogate of section 3.1 and the k3 KL-to-reference term).
+struct LossParams {
+  // inputs
+  const float4* partials;
+  int part_stride;
+  int n_tiles;        // 256-wide vocabulary tiles of the forward pass
+  int n_ctas;         // grid of the forward pass (fixes the split)
+  const int* row_map;
+  const float* old_logp;   // [T] original rows; NULL in log-prob-only mode
+  const float* ref_logp;   // [T] or NULL
+  const float* adv;        // [T]
+  const float* token_weight;  // [T] or NULL
+  float eps_low, eps_high, beta, ent_coef;
+  int with_loss;
+  // compact outputs
+  float* lse_c;
+  float* ent_c;
+  float* cp_c;
+  float* ce_c;
+  // scattered outputs (original rows), any may be NULL
+  float* logp_out;
+  float* ent_out;
+  float* lse_out;
+  // reduction scratch: [gridDim.x][kLossSums] doubles
+  double* block_sums;
+};
+constexpr int kLossSums = 8;  // loss, pg, kl, ent, clip, ratio, ratio_max, unused
+constexpr int kLossThreads = 256;
+
+__global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossParams p, DevStatus* st) {
+  const int n = st->n_valid;
+  const int m_tiles = (n + BM - 1) / BM;
+  const int split = choose_split(m_tiles, p.n_tiles, p.n_ctas);
+  const int n_range = max((p.n_tiles + split - 1) / max(split, 1), 1);
+  const int n_ranges = (p.n_tiles + n_range - 1) / n_range;
+  double acc[kLossSums];
+#pragma unroll
+  for (int k = 0; k < kLossSums; ++k) acc[k] = 0.0;
+  const float w_mean = n > 0 ? 1.f / (float)n : 0.f;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    float M = -CUDART_INF_F;
+    for (int r = 0; r < n_ranges; ++r) M = fmaxf(M, p.partials[(size_t)r * p.part_stride + i].x);
+    float S = 0.f, A = 0.f, zy = 0.f;
+    for (int r = 0; r < n_ranges; ++r) {
+      const float4 q = p.partials[(size_t)r * p.part_stride + i];
+      const float sc = exp2f((q.x - M) * kLog2e);
+      S = fmaf(q.y, sc, S);
+      A = fmaf(q.z, sc, A);
+      zy += q.w;
+    }
+    const float lse = M + logf(S);
+    const float logp = zy - lse;
+    const float ent = lse - A / S;
+    const int row = p.row_map[i];
+    p.lse_c[i] = lse;
+    p.ent_c[i] = ent;
+    if (p.logp_out) p.logp_out[row] = logp;
+    if (p.ent_out) p.ent_out[row] = ent;
+    if (p.lse_out) p.lse_out[row] = lse;
+    if (p.with_loss) {
+      const float w = p.token_weight ? p.token_weight[row] : w_mean;
+      const float A_t = p.adv[row];
+      const float rho = expf(logp - p.old_logp[row]);
+      const float clipped = fminf(fmaxf(rho, 1.f - p.eps_low), 1.f + p.eps_high);
+      const float su = rho * A_t, sc = clipped * A_t;
+      const bool active = su <= sc;          // unclipped branch is the minimum (ties: unclipped)
+      const float s = active ? su : sc;
+      float k3 = 0.f, dk3 = 0.f;
+      if (p.beta != 0.f) {
+        const float delta = p.ref_logp[row] - logp;
+        const float ed = expf(delta);
+        k3 = ed - delta - 1.f;
+        dk3 = 1.f - ed;
+      }
+      const float dlogp = -(active ? A_t * rho : 0.f) + p.beta * dk3;
+      p.cp_c[i] = -w * dlogp;
+      p.ce_c[i] = w * p.ent_coef;
+      acc[0] += (double)w * (double)(-s + p.beta * k3 - p.ent_coef * ent);
+      acc[1] += (double)w * (double)(-s);
+      acc[2] += (double)w * (double)k3;
+      acc[3] += (double)w * (double)ent;
+      acc[4] += active ? 0.0 : (double)w;
+      acc[5] += (double)w * (double)rho;
+      acc[6] = fmax(acc[6], (double)rho);
+    }
+  }
+  if (!p.with_loss) return;
+  __shared__ double red[kLossThreads / 32][kLossSums];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int k = 0; k < kLossSums; ++k) {
+    double v = acc[k];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double u = __shfl_xor_sync(0xffffffffu, v, o);
+      v = (k == 6) ? fmax(v, u) : v + u;
+    }
+    if (lane == 0) red[warp][k] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < kLossSums) {
+    const int k = threadIdx.x;
+    double v = red[0][k];
+    for (int w = 1; w < kLossThreads / 32; ++w) v = (k == 6) ? fmax(v, red[w][k]) : v + red[w][k];
+    p.block_sums[(size_t)blockIdx.x * kLossSums + k] = v;
+  }
+}
+
+// Second stage: fixed-order sum of the block partials -> loss[1] and metrics[8].
+__global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restrict__ block_sums, int n_blocks,
+                                                           float* __restrict__ loss, float* __restrict__ metrics,
+                                                           const DevStatus* st) {
+  const int k = threadIdx.x;
+  if (k >= kLossSums) return;
+  double v = 0.0;
+  for (int b = 0; b < n_blocks; ++b) {
+    const double u = block_sums[(size_t)b * kLossSums + k];
+    v = (k == 6) ? fmax(v, u) : v + u;
+  }
+  if (k == 0) loss[0] = (float)v;
+  if (metrics) {
+    if (k >= 1 && k <= 6) metrics[k - 1] = (float)v;
+    if (k == 7) { metrics[6] = (float)st->n_valid; metrics[7] = 0.f; }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// dH of one row slab: fp32 accumulator rows -> bf16 rows of the caller's dH at their original
+// positions.  One warp per row.
+__global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict__ acc, int d, int slab_base,
+                                                         int slab_rows, const int* __restrict__ row_map,
+                                                         __nv_bfloat16* __restrict__ dH, const DevStatus* st) {
+  const int n = st->n_valid;
+  const int rows = min(max(n - slab_base, 0), slab_rows);
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
+    const float4* src = reinterpret_cast<const float4*>(acc + (size_t)i * d);
+    uint2* dst = reinterpret_cast<uint2*>(dH + (size_t)row_map[slab_base + i] * d);
+    for (int v = lane; v < d / 4; v += 32) {
+      const float4 x = src[v];
+      __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
+      uint2 o;
+      o.x = *reinterpret_cast<uint32_t*>(&lo);
+      o.y = *reinterpret_cast<uint32_t*>(&hi);
+      dst[v] = o;
+    }
+  }
+}
+
+}  // namespace rlh
