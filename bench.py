@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the fused LM-head log-probability + GRPO loss forward+backward path.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config k] [--impl reference]
+
+One step = one pass of the whole hot path over one synthetic batch: GRPO advantages from the
+rewards, mask scan / row compaction, forward statistics, per-token loss, dH and dW.  The default
+workload is the 3B-class head (d=2048, V=151936, 8 prompts x 8 responses x up to 512 tokens).
+Prints one JSON line (rank 0).  `--impl reference` times the float64 CPU oracle instead.
+"""
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fused LM-head logprob+GRPO loss fwd+bwd tokens/s; % of bf16 tensor peak"
+KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad> (dlogits slab)",
+              "gemm_kernel<EpiAcc,K,MN> (dH)", "gemm_kernel<EpiAcc,MN,MN> (dW)"]
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant
+# kernel from an ncu capture, valid only for the kernel sources whose hash is recorded with it.
+NCU_TRAFFIC = {"sources_sha256": None, "kind": None, "bytes_per_launch": None}
+
+
+def sources_hash():
+    h = hashlib.sha256()
+    cs = os.path.join(ROOT, "paper_2512_21450_b200", "csrc")
+    for f in sorted(os.listdir(cs)):
+        h.update(open(os.path.join(cs, f), "rb").read())
+    return h.hexdigest()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(burst=j["bf16_tflops"], sustained=j.get("bf16_tflops_sustained", j["bf16_tflops"]),
+                    hbm=j["hbm_gbs"], source="measured")
+    return dict(burst=1590.0, sustained=1400.0, hbm=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only)."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                smax = float(r[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=smax, reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+def oracle_sample_time(w, n_rows, repeat=1):
+    """Times the float64 oracle (as it stands) on the first n_rows valid rows of workload w."""
+    import numpy as np
+    import torch
+    from oracle import grpo_oracle as O
+    rows = torch.nonzero(w.mask, as_tuple=False)[:n_rows, 0]
+    f64 = lambda t: t.double().cpu().numpy()  # noqa: E731
+    H = f64(w.H[rows])
+    W = f64(w.W)
+    tok = w.tokens[rows].cpu().numpy()
+    old = f64(w.old_logp[rows])
+    ref = None if w.ref_logp is None else f64(w.ref_logp[rows])
+    adv_seq = O.grpo_advantages(w.rewards.cpu().numpy(), w.G)
+    adv = O.broadcast_to_tokens(adv_seq, w.seq_offsets.cpu().numpy(), w.T)[rows.cpu().numpy()]
+    mask = np.ones(rows.numel(), dtype=np.uint8)
+    best = None
+    for _ in range(repeat):
+        t0 = time.perf_counter()
+        O.grpo_advantages(w.rewards.cpu().numpy(), w.G)
+        O.policy_loss_fwd_bwd(H, W, tok, old, ref, adv, mask, w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return rows.numel(), best
+
+
+def run_reference(args):
+    import torch
+    from paper_2512_21450_b200.workloads import CONFIGS, make_workload
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    cfg = CONFIGS[args.config]
+    # the inputs are the bench workload; only a bounded sample of its valid rows is timed per step
+    small = dict(prompts=1, L_max=min(cfg["L_max"], 64)) if dev == "cpu" else {}
+    w = make_workload(args.config, device=dev, **small)
+    n_rows = args.reference_rows
+    cores = len(os.sched_getaffinity(0))
+    for _ in range(args.warmup):
+        oracle_sample_time(w, min(n_rows, 32))
+    t_total, n_tok = 0.0, 0
+    for _ in range(args.steps):
+        n, dt = oracle_sample_time(w, n_rows)
+        t_total += dt
+        n_tok += n
+    value = n_tok / t_total
+    sample = f"{n_tok // max(args.steps, 1)} valid rows per step of workload {w.name} (full d, V), float64 numpy"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"config {args.config}: {w.name} d={w.d} V={w.V}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--reference-rows", type=int, default=256)
+    ap.add_argument("--cpu-baseline-rows", type=int, default=512)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200 import parallel as par
+    from paper_2512_21450_b200.workloads import SEED_BASE, make_workload
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    # weak scaling: every rank owns a full batch of the configuration, with its own seed
+    w = make_workload(args.config, device=dev, seed=SEED_BASE + args.config + 1000 * rank)
+    ctx = Context(local)
+    ctx.ensure_workspace(w.T, w.d, w.V, host=True)
+    dH = torch.empty(w.T, w.d, dtype=torch.bfloat16, device=dev)
+    dW = torch.empty(w.V, w.d, dtype=torch.float32, device=dev)
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+
+    def step():
+        _, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+        tw = par.global_token_weight(w.mask) if world > 1 else None
+        ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, w.eps_low,
+                                   w.eps_high, w.beta, ent_coef=w.ent_coef, token_weight=tw, dW=dW, dH=dH,
+                                   loss=loss, want_aux=False)
+        if world > 1:
+            par.allreduce_gradients(dW, loss)
+
+    def fence():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    fence()
+    status, detail = ctx.last_device_status()
+    assert status == 0, f"device status {status} detail {detail:#x}"
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ctx.set_profiling(True)
+    launches0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fence()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    fence()
+    ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count() - launches0
+    kind_ms, kind_n = ctx.profile_read()
+    ctx.set_profiling(False)
+    clocks = sampler.stop()
+    status, detail = ctx.last_device_status()
+    assert status == 0, f"device status {status} detail {detail:#x}"
+
+    t = torch.tensor([ms, float(w.n_valid)], dtype=torch.float64, device=dev)
+    if world > 1:
+        tmax = t.clone()
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone()
+        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        ms, n_tok = float(tmax[0].item()), float(tsum[1].item())
+    else:
+        n_tok = float(w.n_valid)
+    value = n_tok * args.steps / (ms / 1e3)
+
+    # ---- end to end through the host-buffer entry point: per-step inputs start in pinned host memory
+    pin = lambda x: None if x is None else x.cpu().pin_memory()  # noqa: E731
+    hH, htok, hold, href, hmask = pin(w.H), pin(w.tokens), pin(w.old_logp), pin(w.ref_logp), pin(w.mask)
+    hrew, hoff = pin(w.rewards), pin(w.seq_offsets)
+    h2d = sum(x.numel() * x.element_size() for x in (hH, htok, hold, href, hmask, hrew, hoff) if x is not None)
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        return ctx.rl_policy_loss_fwd_bwd_host(hH, w.W, htok, hold, href, None, hmask, w.eps_low, w.eps_high, w.beta,
+                                               w.ent_coef, dH, dW, rewards_host=hrew, group_size=w.G,
+                                               seq_offsets_host=hoff)
+    e2e_val = None
+    if world == 1:
+        for _ in range(2):
+            e2e_step()
+        fence()
+        e0.record()
+        for _ in range(e2e_steps):
+            host_loss, _ = e2e_step()
+        e1.record()
+        fence()
+        e2e_ms = e0.elapsed_time(e1)
+        e2e_val = n_tok * e2e_steps / (e2e_ms / 1e3)
+        assert abs(host_loss - loss.item()) <= 1e-5 * abs(loss.item()) + 1e-7
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    flops_pass = 2.0 * w.d * w.V * w.n_valid * args.steps       # one GEMM pass over the valid tokens
+    kinds = []
+    for k in range(4):
+        if kind_n[k]:
+            kinds.append(dict(kernel=KIND_NAMES[k], launches=kind_n[k], ms_total=kind_ms[k],
+                              tflops=flops_pass / (kind_ms[k] / 1e3) / 1e12))
+    dom = max(range(4), key=lambda k: kind_ms[k])
+    achieved = flops_pass / (kind_ms[dom] / 1e3) / 1e12
+    traffic = None
+    if NCU_TRAFFIC["sources_sha256"] == sources_hash() and NCU_TRAFFIC["kind"] == dom:
+        traffic = NCU_TRAFFIC["bytes_per_launch"]
+    roofline = {
+        "bound": "tensor", "kernel": KIND_NAMES[dom], "achieved": achieved, "peak": peaks["sustained"],
+        "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "peak_source": f"of {peaks['source']} (sustained)",
+        "traffic": traffic, "flops_per_launch": flops_pass / max(kind_n[dom], 1),
+        "avg_launch_ms": kind_ms[dom] / max(kind_n[dom], 1), "kernels": kinds,
+    }
+    exec_tflops = 8.0 * w.d * w.V * n_tok * args.steps / (ms / 1e3) / 1e12
+    out = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"config {args.config}: {w.name} d={w.d} V={w.V} rows={w.T} valid_tokens={w.n_valid} "
+                               f"G={w.G} eps=({w.eps_low},{w.eps_high}) beta={w.beta} ent_coef={w.ent_coef}",
+                   "l2": "inputs larger than L2 (W alone is %.0f MB; L2 126 MB)" % (w.V * w.d * 2 / 1e6),
+                   "parallelism": f"dp{world}" if world > 1 else "single GPU",
+                   "masked_rows": "skipped (row compaction)"},
+        "pct_of_bf16_peak": {"executed_8dV_of_burst": 100 * exec_tflops / world / peaks["burst"],
+                             "executed_8dV_of_sustained": 100 * exec_tflops / world / peaks["sustained"],
+                             "useful_6dV_of_burst": 75 * exec_tflops / world / peaks["burst"],
+                             "executed_tflops_per_gpu": exec_tflops / world, "peaks": peaks["source"]},
+        "clocks": clocks, "gpu_launches": launches, "roofline": roofline,
+    }
+    if e2e_val is not None:
+        out["e2e"] = {"value": e2e_val, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 64,
+                      "steps": e2e_steps, "call": "rl_policy_loss_fwd_bwd_host (pinned host inputs, W resident)"}
+    if world == 1 and not args.no_cpu_baseline:
+        n, dt = oracle_sample_time(w, args.cpu_baseline_rows)
+        out["cpu_baseline"] = {"value": n / dt, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)),
+                               "kind": "oracle", "sample": f"first {n} valid rows of the same workload, full d and V, "
+                                                           f"float64 numpy, one pass ({dt:.1f} s)"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -62,6 +62,12 @@ const char* rl_status_string(rl_status s);
  * size does not grow with T*V: the gradient with respect to the logits only ever exists for a
  * bounded slab of rows x vocabulary columns. */
 rl_status rl_workspace_bytes(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_t* bytes);
+/* Size of the slab the backward pass works in: at most max_rows token rows x max_cols vocabulary
+ * columns of the gradient with respect to the logits exist at a time (bf16, in the workspace).
+ * max_rows a multiple of 128, max_cols a multiple of 256; 0 restores a default (32768 x 9472,
+ * chosen so that the tile counts of the three backward passes are multiples of 148 SMs for
+ * d = 2048, 2560 and 3584).  Changes what rl_workspace_bytes() returns: call it first. */
+rl_status rl_set_slab_limits(rl_ctx* ctx, int max_rows, int max_cols);
 /* Caller-owned device scratch, 256-byte aligned; must outlive the calls that use it. */
 rl_status rl_set_workspace(rl_ctx* ctx, void* dev_ptr, size_t bytes);
 
@@ -132,20 +138,35 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* ctx, const void* H, int64_t ldH, con
                                     float eps_low, float eps_high, float beta,
                                     float* loss, void* dH, float* dW, const rl_loss_opts* opts);
 
-/* Same computation with the per-step inputs in HOST memory (pinned memory gives asynchronous
- * copies): H, tokens, old_logp, ref_logp, adv, mask are host pointers, copied to the device
- * inside the call; W, dH and dW stay device pointers (weights and gradients live on the
- * device); loss_host[1] and metrics_host[8] (may be NULL) are written on the host.  The call
- * synchronises the context's stream before returning.  The workspace must have been sized with
- * rl_workspace_bytes_host(). */
+/* One whole step with the per-step inputs in HOST memory (pinned memory gives asynchronous
+ * copies): H, tokens, old_logp, ref_logp, mask and either adv (per row) or rewards[n_seq] +
+ * seq_offsets[n_seq+1] are host pointers, copied to the device inside the call; when adv_host is
+ * NULL the advantages are computed on the device from the rewards as rl_grpo_advantages does and
+ * broadcast over seq_offsets.  W, dH and dW stay device pointers (weights and gradients live on
+ * the device); loss_host[1] and metrics_host[8] (may be NULL) are written on the host.  ldH must
+ * equal d.  The call synchronises the context's stream before returning.  The workspace must
+ * have been sized with rl_workspace_bytes_host(). */
 rl_status rl_workspace_bytes_host(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_t* bytes);
 rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* ctx, const void* H_host, int64_t ldH, const void* W,
                                       int64_t ldW, const int32_t* tokens_host,
                                       const float* old_logp_host, const float* ref_logp_host,
-                                      const float* adv_host, const uint8_t* mask_host,
+                                      const float* adv_host, const float* rewards_host,
+                                      int64_t n_seq, int group_size,
+                                      const int32_t* seq_offsets_host, const uint8_t* mask_host,
                                       int64_t T, int64_t d, int64_t V,
                                       float eps_low, float eps_high, float beta, float ent_coef,
                                       float* loss_host, float* metrics_host, void* dH, float* dW);
+
+/* Instrumentation.  rl_launch_count: kernels this context has launched so far.
+ * rl_set_profiling(on): when on, every tensor-core launch is bracketed by a pair of CUDA events
+ * on the context's stream (at most 2048 launches are kept between two reads).
+ * rl_profile_read: synchronises the stream and returns, per kernel kind (0 forward statistics,
+ * 1 gradient-of-logits slab, 2 dH, 3 dW), the summed device time in milliseconds ms[4] (host)
+ * and the number of launches launches[4] (host) since the previous read.  The paper has no
+ * counterpart; these exist so that a benchmark can report per-kernel roofline figures. */
+rl_status rl_launch_count(rl_ctx* ctx, int64_t* n);
+rl_status rl_set_profiling(rl_ctx* ctx, int on);
+rl_status rl_profile_read(rl_ctx* ctx, double* ms, int64_t* launches);
 
 /* Self-test of the tensor-core GEMM engine the calls above are built from: C[M,N] (fp32,
  * row-major, ldc = N) = A * B with bf16 operands.  a_mn_major = 0: A is [M,K] row-major;

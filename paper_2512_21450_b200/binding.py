@@ -60,6 +60,7 @@ def load_library():
     lib.rl_workspace_bytes.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
     lib.rl_workspace_bytes_host.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
     lib.rl_set_workspace.argtypes = [P, P, c_size_t]
+    lib.rl_set_slab_limits.argtypes = [P, c_int, c_int]
     lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
     lib.rl_grpo_advantages.argtypes = [P, P, c_int64, c_int, P]
     lib.rl_grpo_advantages_ex.argtypes = [P, P, c_int64, c_int, c_int, c_float, P, c_int64, P, P]
@@ -68,13 +69,18 @@ def load_library():
                  c_float, c_float, c_float, P, P, P]
     lib.rl_policy_loss_fwd_bwd.argtypes = loss_args
     lib.rl_policy_loss_fwd_bwd_ex.argtypes = loss_args + [POINTER(rl_loss_opts)]
-    lib.rl_policy_loss_fwd_bwd_host.argtypes = [P, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int64, c_int64,
+    lib.rl_policy_loss_fwd_bwd_host.argtypes = [P, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int, P, P,
+                                                c_int64, c_int64, c_int64,
                                                 c_float, c_float, c_float, c_float, P, P, P, P]
+    lib.rl_launch_count.argtypes = [P, POINTER(c_int64)]
+    lib.rl_set_profiling.argtypes = [P, c_int]
+    lib.rl_profile_read.argtypes = [P, POINTER(ctypes.c_double), POINTER(c_int64)]
     lib.rl_selftest_gemm.argtypes = [P, P, P, P, c_int64, c_int64, c_int64, c_int, c_int, c_int]
     for name in ("rl_create", "rl_destroy", "rl_set_stream", "rl_workspace_bytes", "rl_workspace_bytes_host",
-                 "rl_set_workspace", "rl_last_device_status", "rl_grpo_advantages", "rl_grpo_advantages_ex",
+                 "rl_set_workspace", "rl_set_slab_limits", "rl_last_device_status", "rl_grpo_advantages", "rl_grpo_advantages_ex",
                  "rl_token_logprobs", "rl_policy_loss_fwd_bwd", "rl_policy_loss_fwd_bwd_ex",
-                 "rl_policy_loss_fwd_bwd_host", "rl_selftest_gemm"):
+                 "rl_policy_loss_fwd_bwd_host", "rl_selftest_gemm", "rl_launch_count", "rl_set_profiling",
+                 "rl_profile_read"):
         getattr(lib, name).restype = c_int
     _lib = lib
     return lib
@@ -129,6 +135,9 @@ class Context:
             self._ws = None
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         _check(self.lib.rl_set_workspace(self.handle, _ptr(self._ws), self._ws.numel()), "rl_set_workspace")
+
+    def set_slab_limits(self, max_rows=0, max_cols=0):
+        _check(self.lib.rl_set_slab_limits(self.handle, max_rows, max_cols), "rl_set_slab_limits")
 
     def last_device_status(self):
         detail = c_int32()
@@ -207,8 +216,23 @@ class Context:
         _check(self.lib.rl_policy_loss_fwd_bwd_ex(*args, byref(opts)), "rl_policy_loss_fwd_bwd_ex")
         return out
 
+    def launch_count(self):
+        n = c_int64()
+        _check(self.lib.rl_launch_count(self.handle, byref(n)), "rl_launch_count")
+        return n.value
+
+    def set_profiling(self, on):
+        _check(self.lib.rl_set_profiling(self.handle, int(on)), "rl_set_profiling")
+
+    def profile_read(self):
+        ms = (ctypes.c_double * 4)()
+        n = (c_int64 * 4)()
+        _check(self.lib.rl_profile_read(self.handle, ms, n), "rl_profile_read")
+        return list(ms), list(n)
+
     def rl_policy_loss_fwd_bwd_host(self, H_host, W, tokens_host, old_host, ref_host, adv_host, mask_host,
-                                    eps_low, eps_high, beta, ent_coef, dH, dW):
+                                    eps_low, eps_high, beta, ent_coef, dH, dW, rewards_host=None, group_size=0,
+                                    seq_offsets_host=None):
         """Per-step inputs in (pinned) host memory; W, dH, dW on the device.  Returns (loss, metrics) floats."""
         self._bind_stream()
         T, d = H_host.shape
@@ -218,7 +242,8 @@ class Context:
         metrics = (c_float * 8)()
         _check(self.lib.rl_policy_loss_fwd_bwd_host(
             self.handle, _ptr(H_host), d, _ptr(W), W.stride(0), _ptr(tokens_host), _ptr(old_host), _ptr(ref_host),
-            _ptr(adv_host), _ptr(mask_host), T, d, V, eps_low, eps_high, beta, ent_coef,
+            _ptr(adv_host), _ptr(rewards_host), rewards_host.numel() if rewards_host is not None else 0, group_size,
+            _ptr(seq_offsets_host), _ptr(mask_host), T, d, V, eps_low, eps_high, beta, ent_coef,
             ctypes.cast(loss, c_void_p), ctypes.cast(metrics, c_void_p), _ptr(dH), _ptr(dW)),
             "rl_policy_loss_fwd_bwd_host")
         return loss[0], list(metrics)

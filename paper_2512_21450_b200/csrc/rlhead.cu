@@ -17,6 +17,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+constexpr int kProfMax = 2048;   // timed launches kept between two rl_profile_read calls
+constexpr int kProfKinds = 4;    // 0 forward statistics, 1 dlogits, 2 dH, 3 dW
+
 struct rl_ctx {
   int device;
   int n_sm;
@@ -25,6 +28,14 @@ struct rl_ctx {
   void* ws;
   size_t ws_bytes;
   EncodeTiledFn encode;
+  int slab_rows;  // rows of one gradient slab (multiple of 128)
+  int slab_cols;  // vocabulary columns of one gradient slab (multiple of 256)
+  long long launches;  // kernels launched by this context so far
+  // optional per-kernel timing: event pairs around every tensor-core launch, by kernel kind
+  int prof_on;
+  int prof_used;
+  int prof_kind[kProfMax];
+  cudaEvent_t prof_ev[kProfMax][2];
 };
 
 namespace {
@@ -40,12 +51,12 @@ struct WsLayout {
 };
 
 // staging_T > 0 adds room for host-call inputs (H, tokens, old, ref, adv, mask).
-WsLayout ws_layout(int64_t T, int64_t d, int64_t V, bool host_staging) {
+WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_staging) {
   WsLayout L;
   L.Tpad = (int)align_up((size_t)(T > 0 ? T : 1), 128);
-  L.Ts = L.Tpad < kSlabRowsMax ? L.Tpad : kSlabRowsMax;
+  L.Ts = L.Tpad < c->slab_rows ? L.Tpad : c->slab_rows;
   const int Vpad = (int)align_up((size_t)V, 256);
-  L.Vs = Vpad < kSlabColsMax ? Vpad : kSlabColsMax;
+  L.Vs = Vpad < c->slab_cols ? Vpad : c->slab_cols;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 1024); return at; };
   L.row_map = take((size_t)L.Tpad * 4);
@@ -68,6 +79,9 @@ WsLayout ws_layout(int64_t T, int64_t d, int64_t V, bool host_staging) {
     take((size_t)T * 4);      // adv
     take((size_t)T);          // mask
     take(64);                 // loss + metrics
+    take((size_t)T * 4);      // rewards
+    take((size_t)T * 4);      // per-response advantages
+    take((size_t)(T + 1) * 4);  // seq_offsets
   }
   L.total = o;
   return L;
@@ -104,9 +118,20 @@ cudaError_t set_smem_attr() {
 }
 
 template <class Epi, int A_MN, int B_MN>
-void launch_gemm(rl_ctx* c, const CUtensorMap& a, const CUtensorMap& b, const GemmShape& sh,
+void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const GemmShape& sh,
                  const typename Epi::Params& ep) {
+  const bool timed = c->prof_on && kind >= 0 && kind < kProfKinds && c->prof_used < kProfMax;
+  if (timed) {
+    for (int e = 0; e < 2; ++e)
+      if (!c->prof_ev[c->prof_used][e]) cudaEventCreate(&c->prof_ev[c->prof_used][e]);
+    cudaEventRecord(c->prof_ev[c->prof_used][0], c->stream);
+  }
   gemm_kernel<Epi, A_MN, B_MN><<<c->n_sm, kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, sh, ep, c->dstatus);
+  c->launches++;
+  if (timed) {
+    cudaEventRecord(c->prof_ev[c->prof_used][1], c->stream);
+    c->prof_kind[c->prof_used++] = kind;
+  }
 }
 
 rl_status check_hw(const void* H, int64_t ldH, const void* W, int64_t ldW, int64_t T, int64_t d, int64_t V) {
@@ -137,6 +162,7 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   mask_scan_kernel<<<1, kScanThreads, 0, c->stream>>>(mask, (int)T, row_map, c->dstatus);
   gather_rows_kernel<<<c->n_sm * 4, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16*>(H), ldH, (int)d, row_map,
                                                          tokens, (int)V, Hc, tokens_c, c->dstatus);
+  c->launches += 2;
   CUtensorMap tmA, tmB;
   if (!map_kmajor(c, &tmA, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM)) return RL_ERR_CUDA;
   if (!map_kmajor(c, &tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, BN)) return RL_ERR_CUDA;
@@ -153,7 +179,7 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   ep.partials = reinterpret_cast<float4*>(ws + L.partials);
   ep.part_stride = L.Tpad;
   ep.V = (int)V;
-  launch_gemm<EpiStats, 0, 0>(c, tmA, tmB, sh, ep);
+  launch_gemm<EpiStats, 0, 0>(c, 0, tmA, tmB, sh, ep);
   *n_tiles_out = sh.n_tiles;
   return cuda_ok();
 }
@@ -191,6 +217,12 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->stream = nullptr;
   c->ws = nullptr;
   c->ws_bytes = 0;
+  c->slab_rows = kSlabRowsMax;
+  c->slab_cols = kSlabColsMax;
+  c->launches = 0;
+  c->prof_on = 0;
+  c->prof_used = 0;
+  memset(c->prof_ev, 0, sizeof(c->prof_ev));
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -211,6 +243,9 @@ rl_status rl_create(rl_ctx** out, int device) {
 
 rl_status rl_destroy(rl_ctx* c) {
   if (!c) return RL_ERR_INVALID_ARG;
+  for (int i = 0; i < kProfMax; ++i)
+    for (int e = 0; e < 2; ++e)
+      if (c->prof_ev[i][e]) cudaEventDestroy(c->prof_ev[i][e]);
   cudaFree(c->dstatus);
   delete c;
   return RL_OK;
@@ -224,13 +259,51 @@ rl_status rl_set_stream(rl_ctx* c, void* s) {
 
 rl_status rl_workspace_bytes(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t* bytes) {
   if (!c || !bytes || T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
-  *bytes = ws_layout(T, d, V, false).total;
+  *bytes = ws_layout(c, T, d, V, false).total;
   return RL_OK;
 }
 
 rl_status rl_workspace_bytes_host(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t* bytes) {
   if (!c || !bytes || T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
-  *bytes = ws_layout(T, d, V, true).total;
+  *bytes = ws_layout(c, T, d, V, true).total;
+  return RL_OK;
+}
+
+rl_status rl_launch_count(rl_ctx* c, int64_t* n) {
+  if (!c || !n) return RL_ERR_INVALID_ARG;
+  *n = c->launches;
+  return RL_OK;
+}
+
+rl_status rl_set_profiling(rl_ctx* c, int on) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  c->prof_on = on ? 1 : 0;
+  c->prof_used = 0;
+  return RL_OK;
+}
+
+rl_status rl_profile_read(rl_ctx* c, double* ms, int64_t* launches) {
+  if (!c || !ms || !launches) return RL_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return RL_ERR_CUDA;
+  for (int k = 0; k < kProfKinds; ++k) { ms[k] = 0.0; launches[k] = 0; }
+  for (int i = 0; i < c->prof_used; ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, c->prof_ev[i][0], c->prof_ev[i][1]) != cudaSuccess) return RL_ERR_CUDA;
+    ms[c->prof_kind[i]] += t;
+    launches[c->prof_kind[i]]++;
+  }
+  c->prof_used = 0;
+  return RL_OK;
+}
+
+rl_status rl_set_slab_limits(rl_ctx* c, int max_rows, int max_cols) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  if (max_rows == 0) max_rows = kSlabRowsMax;
+  if (max_cols == 0) max_cols = kSlabColsMax;
+  if (max_rows < 128 || max_rows % 128 != 0 || max_cols < 256 || max_cols % 256 != 0) return RL_ERR_SHAPE;
+  if ((int64_t)max_rows * max_cols > (int64_t(1) << 31)) return RL_ERR_SHAPE;
+  c->slab_rows = max_rows;
+  c->slab_cols = max_cols;
   return RL_OK;
 }
 
@@ -267,10 +340,12 @@ rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, 
   const int warps = 8;
   grpo_adv_kernel<<<(n_groups + warps - 1) / warps, warps * 32, 0, c->stream>>>(rewards, n_groups, group_size, ddof,
                                                                                 eps_std, adv_seq);
+  c->launches++;
   if (adv_tok) {
     if (T > 0 && cudaMemsetAsync(adv_tok, 0, (size_t)T * 4, c->stream) != cudaSuccess) return RL_ERR_CUDA;
     int blocks = (int)(n_seq < 4096 ? n_seq : 4096);
     broadcast_adv_kernel<<<blocks, 256, 0, c->stream>>>(adv_seq, seq_offsets, (int)n_seq, adv_tok);
+    c->launches++;
   }
   return cuda_ok();
 }
@@ -287,7 +362,7 @@ rl_status rl_token_logprobs(rl_ctx* c, const void* H, int64_t ldH, const void* W
   if (s != RL_OK) return s;
   if (T == 0) return RL_OK;
   if (!tokens || !logp) return RL_ERR_INVALID_ARG;
-  const WsLayout L = ws_layout(T, d, V, false);
+  const WsLayout L = ws_layout(c, T, d, V, false);
   if ((s = check_ws(c, L)) != RL_OK) return s;
   char* ws = static_cast<char*>(c->ws);
   cudaMemsetAsync(logp, 0, (size_t)T * 4, c->stream);
@@ -311,6 +386,7 @@ rl_status rl_token_logprobs(rl_ctx* c, const void* H, int64_t ldH, const void* W
   int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
   if (blocks > 1024) blocks = 1024;
   combine_loss_kernel<<<blocks, kLossThreads, 0, c->stream>>>(p, c->dstatus);
+  c->launches++;
   return cuda_ok();
 }
 
@@ -335,7 +411,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   }
   if (!(o.ent_coef >= 0.f)) return RL_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(dH) & 15) || (reinterpret_cast<uintptr_t>(dW) & 15)) return RL_ERR_ALIGNMENT;
-  const WsLayout L = ws_layout(T, d, V, false);
+  const WsLayout L = ws_layout(c, T, d, V, false);
   if ((s = check_ws(c, L)) != RL_OK) return s;
   char* ws = static_cast<char*>(c->ws);
   cudaStream_t st = c->stream;
@@ -382,6 +458,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   if (blocks > 1024) blocks = 1024;
   combine_loss_kernel<<<blocks, kLossThreads, 0, st>>>(p, c->dstatus);
   finalize_loss_kernel<<<1, 32, 0, st>>>(p.block_sums, blocks, loss, o.metrics_out, c->dstatus);
+  c->launches += 2;
 
   // ---- backward, one (row slab x vocabulary slab) at a time
   __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + L.Hc);
@@ -423,7 +500,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
         ep.lse = p.lse_c; ep.ent = p.ent_c; ep.cp = p.cp_c; ep.ce = p.ce_c;
         ep.G = G; ep.ldG = L.Vs; ep.V = (int)V; ep.vocab_base = vocab_base; ep.row_base = row_base;
-        launch_gemm<EpiGrad, 0, 0>(c, tmHc_k, tmW_k, sh, ep);
+        launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, sh, ep);
       }
       // (2) dH_slab (+)= G * W_slab        [rows x d], K = vocabulary columns of the slab
       {
@@ -437,7 +514,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         sh.b_k_off = vocab_base;
         EpiAcc::Params ep;
         ep.C = dH_acc; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0;
-        launch_gemm<EpiAcc, 0, 1>(c, tmG_k, tmW_mn, sh, ep);
+        launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, sh, ep);
       }
       // (3) dW_slab (+)= G^T * H_slab      [vocabulary rows x d], K = valid rows of the slab
       {
@@ -453,11 +530,12 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         EpiAcc::Params ep;
         ep.C = dW; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
         ep.row_base = vocab_base;
-        launch_gemm<EpiAcc, 1, 1>(c, tmG_mn, tmHc_mn, sh, ep);
+        launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, sh, ep);
       }
     }
     scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
                                                    static_cast<__nv_bfloat16*>(dH), c->dstatus);
+    c->launches++;
   }
   return cuda_ok();
 }
@@ -472,14 +550,17 @@ rl_status rl_policy_loss_fwd_bwd(rl_ctx* c, const void* H, int64_t ldH, const vo
 
 rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* c, const void* H_host, int64_t ldH, const void* W, int64_t ldW,
                                       const int32_t* tokens_host, const float* old_host, const float* ref_host,
-                                      const float* adv_host, const uint8_t* mask_host, int64_t T, int64_t d,
+                                      const float* adv_host, const float* rewards_host, int64_t n_seq,
+                                      int group_size, const int32_t* seq_offsets_host,
+                                      const uint8_t* mask_host, int64_t T, int64_t d,
                                       int64_t V, float eps_low, float eps_high, float beta, float ent_coef,
                                       float* loss_host, float* metrics_host, void* dH, float* dW) {
   if (!c || !loss_host) return RL_ERR_INVALID_ARG;
   if (T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
-  if (T > 0 && (!H_host || !tokens_host || !old_host || !adv_host)) return RL_ERR_INVALID_ARG;
+  if (T > 0 && (!H_host || !tokens_host || !old_host)) return RL_ERR_INVALID_ARG;
+  if (T > 0 && !adv_host && (!rewards_host || !seq_offsets_host || n_seq <= 0 || n_seq > T)) return RL_ERR_INVALID_ARG;
   if (ldH != d) return RL_ERR_SHAPE;  // host rows are copied as one block
-  const WsLayout L = ws_layout(T, d, V, true);
+  const WsLayout L = ws_layout(c, T, d, V, true);
   rl_status s = check_ws(c, L);
   if (s != RL_OK) return s;
   char* ws = static_cast<char*>(c->ws);
@@ -492,13 +573,23 @@ rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* c, const void* H_host, int64_t ldH
   float* d_adv = reinterpret_cast<float*>(take((size_t)T * 4));
   uint8_t* d_mask = reinterpret_cast<uint8_t*>(take((size_t)T));
   float* d_out = reinterpret_cast<float*>(take(64));
+  float* d_rew = reinterpret_cast<float*>(take((size_t)T * 4));
+  float* d_advseq = reinterpret_cast<float*>(take((size_t)T * 4));
+  int32_t* d_off = reinterpret_cast<int32_t*>(take((size_t)(T + 1) * 4));
   cudaStream_t st = c->stream;
   if (T > 0) {
     cudaMemcpyAsync(dH_in, H_host, (size_t)T * d * 2, cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(d_tok, tokens_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(d_old, old_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
     if (ref_host) cudaMemcpyAsync(d_ref, ref_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
-    cudaMemcpyAsync(d_adv, adv_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
+    if (adv_host) {
+      cudaMemcpyAsync(d_adv, adv_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
+    } else {
+      cudaMemcpyAsync(d_rew, rewards_host, (size_t)n_seq * 4, cudaMemcpyHostToDevice, st);
+      cudaMemcpyAsync(d_off, seq_offsets_host, (size_t)(n_seq + 1) * 4, cudaMemcpyHostToDevice, st);
+      rl_status sa = rl_grpo_advantages_ex(c, d_rew, n_seq, group_size, 1, 1e-6f, d_off, T, d_advseq, d_adv);
+      if (sa != RL_OK) return sa;
+    }
     if (mask_host) cudaMemcpyAsync(d_mask, mask_host, (size_t)T, cudaMemcpyHostToDevice, st);
   }
   rl_loss_opts opts;
@@ -536,10 +627,10 @@ rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, in
   sh.n_range = 1;
   EpiAcc::Params ep;
   ep.C = C; ep.ldc = N; ep.n_cols = (int)N; ep.accumulate = accumulate; ep.row_base = 0;
-  if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, ta, tb, sh, ep);
-  else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, ta, tb, sh, ep);
-  else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, ta, tb, sh, ep);
-  else launch_gemm<EpiAcc, 1, 1>(c, ta, tb, sh, ep);
+  if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, -1, ta, tb, sh, ep);
+  else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, -1, ta, tb, sh, ep);
+  else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, -1, ta, tb, sh, ep);
+  else launch_gemm<EpiAcc, 1, 1>(c, -1, ta, tb, sh, ep);
   return cuda_ok();
 }
 

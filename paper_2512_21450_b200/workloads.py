@@ -65,7 +65,10 @@ class Workload:
 
 def _lengths_and_mask(cfg, n_seq, L_max, rng):
     lo, hi = cfg["len_range"]
-    lo, hi = min(lo, L_max), min(hi, L_max)
+    if L_max != cfg["L_max"]:
+        # shrunk parity case: keep the shape of the length distribution
+        lo = max(1, lo * L_max // cfg["L_max"])
+        hi = max(lo, hi * L_max // cfg["L_max"])
     lens = rng.integers(lo, hi + 1, size=n_seq)
     mask = np.zeros((n_seq, L_max), dtype=np.uint8)
     for i, n in enumerate(lens):
@@ -73,11 +76,13 @@ def _lengths_and_mask(cfg, n_seq, L_max, rng):
     frac = cfg.get("span_mask")
     if frac:
         # multi-turn rollouts: observation / tool-output spans are excluded from the loss
+        s_lo = max(2, 32 * L_max // cfg["L_max"])
+        s_hi = max(s_lo + 1, 256 * L_max // cfg["L_max"])
         for i in range(n_seq):
             target = int(frac * lens[i])
             guard = 0
             while (lens[i] - mask[i].sum()) < target and guard < 10000:
-                span = int(rng.integers(32, 257))
+                span = int(rng.integers(s_lo, s_hi + 1))
                 start = int(rng.integers(1, max(2, lens[i] - span)))
                 mask[i, start:start + span] = 0
                 guard += 1

@@ -1,0 +1,83 @@
+"""CPU-only checks of the boundary and the host logic: the shared library builds, loads and
+exports every symbol the header declares; the binding refuses to run without a GPU; the
+synthetic workloads have the structure the configurations ask for."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "rlhead.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rl_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    from paper_2512_21450_b200 import build
+    path = build.build()
+    assert os.path.exists(path)
+    lib = ctypes.CDLL(path)
+    names = _declared_symbols()
+    assert {"rl_grpo_advantages", "rl_token_logprobs", "rl_policy_loss_fwd_bwd"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in rlhead.h but not exported"
+    lib.rl_status_string.restype = ctypes.c_char_p
+    assert lib.rl_status_string(0) == b"ok"
+    assert b"token" in lib.rl_status_string(7)
+
+
+def test_binding_declares_every_symbol_and_has_no_cpu_path():
+    from paper_2512_21450_b200 import binding
+    lib = binding.load_library()
+    for n in _declared_symbols():
+        assert getattr(lib, n).argtypes is not None or n == "rl_status_string"
+    if not torch.cuda.is_available():
+        with pytest.raises(RuntimeError):
+            binding.Context(0)
+
+
+def test_product_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2512_21450_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert not re.search(r"^\s*(from|import)\s+oracle\b", src, flags=re.M), f
+                assert "grpo_oracle" not in src and "oracle/" not in src and "oracle." not in src, f
+    osrc = open(os.path.join(ROOT, "oracle", "grpo_oracle.py")).read()
+    assert "paper_2512_21450_b200" not in osrc and "import torch" not in osrc
+
+
+def test_workload_structure_cpu():
+    from paper_2512_21450_b200.workloads import CONFIGS, make_workload
+    w = make_workload(0, device="cpu")
+    assert (w.T, w.d, w.V, w.G, w.n_seq, w.n_valid) == (256, 256, 4096, 4, 16, 256)
+    assert w.H.dtype == torch.bfloat16 and w.W.dtype == torch.bfloat16 and w.tokens.dtype == torch.int32
+    assert int(w.tokens.min()) >= 0 and int(w.tokens.max()) < w.V
+    w2 = make_workload(0, device="cpu")
+    assert torch.equal(w.H, w2.H) and torch.equal(w.tokens, w2.tokens) and torch.equal(w.old_logp, w2.old_logp)
+    # perturbation scale of the behaviour / reference log-probabilities
+    z = w.H.float() @ w.W.float().T
+    lp = torch.log_softmax(z, 1).gather(1, w.tokens.long()[:, None])[:, 0]
+    assert 0.03 < (w.old_logp - lp).std().item() < 0.07
+    assert 0.07 < (w.ref_logp - lp).std().item() < 0.13
+    # small-shape stand-ins of the other configurations keep their mask / reward structure
+    w1 = make_workload(1, device="cpu", d=64, V=512)
+    lens = w1.mask.view(w1.n_seq, w1.L_max).sum(1)
+    assert w1.T == 64 * 512 and int(lens.min()) >= 64 and int(lens.max()) <= 512
+    m = w1.mask.view(w1.n_seq, w1.L_max)
+    assert all(bool((row[:n] == 1).all()) and not bool(row[n:].any()) for row, n in zip(m, lens))  # right-padded
+    w3 = make_workload(3, device="cpu", prompts=1, d=64, V=512)
+    frac = 1 - w3.n_valid / w3.T
+    assert 0.28 < frac < 0.36 and bool(w3.mask.view(w3.n_seq, -1)[:, 0].all())
+    w4 = make_workload(4, device="cpu", L_max=8, d=64, V=512)
+    r = w4.rewards.view(-1, w4.G)
+    zero_var = (r.max(1).values == r.min(1).values).float().mean().item()
+    assert 0.1 < zero_var < 0.45 and w4.ref_logp is None and w4.ent_coef == 1e-3 and w4.eps_high == 0.28
+    assert CONFIGS[2]["V"] == 152064 and CONFIGS[2]["d"] == 3584

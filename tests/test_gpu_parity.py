@@ -1,0 +1,297 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle on the same
+seeded inputs.  Tolerances are the stated ones for bf16 inputs with fp32 accumulation:
+|dlogp| <= 2e-3, |dentropy| <= 2e-3, loss relative error <= 1e-3, dH and dW relative Frobenius
+error <= 1e-2, advantages within 1e-6."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import grpo_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+TOL_LOGP = 2e-3
+TOL_ENT = 2e-3
+TOL_LOSS_REL = 1e-3
+TOL_GRAD_REL = 1e-2
+TOL_ADV = 1e-6
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2512_21450_b200 import Context
+    c = Context(0)
+    yield c
+    c.close()
+
+
+def _np64(t):
+    return t.detach().double().cpu().numpy()
+
+
+def _assert_status_ok(ctx):
+    s, detail = ctx.last_device_status()
+    assert s == 0, f"device status {s} detail {detail:#x}"
+
+
+def _rel(a, b):
+    nb = np.linalg.norm(b)
+    return np.linalg.norm(a - b) / nb if nb > 0 else np.linalg.norm(a)
+
+
+def _oracle_case(w, adv_tok_np, **kw):
+    return O.policy_loss_fwd_bwd(
+        _np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), _np64(w.old_logp),
+        None if w.ref_logp is None else _np64(w.ref_logp), adv_tok_np, w.mask.cpu().numpy(),
+        w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef, **kw)
+
+
+def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5):
+    from paper_2512_21450_b200.workloads import Workload  # noqa: F401
+    adv_seq, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+    o_adv = O.grpo_advantages(w.rewards.cpu().numpy(), w.G)
+    assert np.abs(_np64(adv_seq) - o_adv).max() <= TOL_ADV
+    o_adv_tok = O.broadcast_to_tokens(o_adv, w.seq_offsets.cpu().numpy(), w.T)
+    assert np.abs(_np64(adv_tok) - o_adv_tok).max() <= TOL_ADV
+
+    out = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask,
+                                     w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef,
+                                     token_weight=token_weight)
+    _assert_status_ok(ctx)
+    # the oracle gets the advantages the GPU loss saw (their own parity is checked above)
+    oo = _oracle_case(w, _np64(adv_tok), token_weight=None if token_weight is None else _np64(token_weight))
+    m = w.mask.cpu().numpy().astype(bool)
+    assert np.abs(_np64(out["logp"]) - oo["logp"]).max() <= TOL_LOGP
+    assert np.abs(_np64(out["entropy"]) - oo["entropy"]).max() <= TOL_ENT
+    assert np.all(_np64(out["logp"])[~m] == 0) and np.all(_np64(out["entropy"])[~m] == 0)
+    # the clip decision is taken in fp32 on the GPU: tokens whose ratio sits on a clip boundary
+    # within rounding may legitimately fall on either side; the seeds used here have none
+    rho = oo["rho"]
+    if rho.size:
+        dist = np.minimum(np.abs(rho - (1 - w.eps_low)), np.abs(rho - (1 + w.eps_high)))
+        assert dist.min() > boundary_margin, "a token sits on the clip boundary; pick another seed"
+    loss = float(out["loss"].item())
+    assert abs(loss - oo["loss"]) <= TOL_LOSS_REL * abs(oo["loss"]) + 1e-7
+    dH = _np64(out["dH"])
+    assert not dH[~m].any()
+    assert _rel(dH, oo["dH"]) <= TOL_GRAD_REL
+    assert _rel(_np64(out["dW"]), oo["dW"]) <= TOL_GRAD_REL
+    met = _np64(out["metrics"])
+    assert abs(met[0] - oo["pg_loss"]) <= 1e-3 * abs(oo["pg_loss"]) + 1e-7
+    assert abs(met[1] - oo["kl_mean"]) <= 1e-3 * abs(oo["kl_mean"]) + 1e-7
+    assert abs(met[2] - oo["entropy_mean"]) <= 2e-3
+    assert abs(met[3] - oo["clip_frac"]) <= 1e-6
+    assert met[6] == m.sum()
+    return out, oo
+
+
+# ------------------------------------------------------------------------------------------------
+def test_gemm_engine_layouts(ctx):
+    # operand layouts of the tensor-core engine against a library product
+    g = torch.Generator(device="cuda").manual_seed(1)
+    for (M, N, K) in [(128, 256, 64), (256, 512, 200), (384, 768, 2048)]:
+        A = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+        B = torch.randn(N, K, generator=g, device="cuda").to(torch.bfloat16)
+        ref = A.float() @ B.float().T
+        for a_mn in (0, 1):
+            for b_mn in (0, 1):
+                C = ctx.rl_selftest_gemm(A.T.contiguous() if a_mn else A, B.T.contiguous() if b_mn else B,
+                                         M, N, K, a_mn, b_mn)
+                _assert_status_ok(ctx)
+                assert (C - ref).abs().max().item() <= 1e-4 * ref.abs().max().item()
+                C2 = ctx.rl_selftest_gemm(A.T.contiguous() if a_mn else A, B.T.contiguous() if b_mn else B,
+                                          M, N, K, a_mn, b_mn, C=C.clone(), accumulate=True)
+                assert (C2 - 2 * ref).abs().max().item() <= 2e-4 * ref.abs().max().item()
+
+
+@pytest.mark.parametrize("n_groups,G", [(4, 4), (8, 8), (64, 16), (7, 5), (3, 40), (1024, 8)])
+def test_advantages(ctx, n_groups, G):
+    rng = np.random.default_rng(100 + G)
+    for kind in ("bernoulli", "uniform", "zero_var"):
+        if kind == "bernoulli":
+            r = (rng.uniform(size=n_groups * G) < 0.4).astype(np.float32)
+        elif kind == "uniform":
+            r = rng.uniform(size=n_groups * G).astype(np.float32)
+        else:
+            r = np.repeat(rng.uniform(size=n_groups).astype(np.float32), G)
+        rt = torch.from_numpy(r).cuda()
+        for ddof in (0, 1):
+            a = ctx.rl_grpo_advantages(rt, G, ddof=ddof, eps_std=1e-6)
+            o = O.grpo_advantages(r, G, ddof=ddof, eps_std=1e-6)
+            assert np.abs(_np64(a) - o).max() <= TOL_ADV
+            if kind == "zero_var":
+                assert not _np64(a).any()
+
+
+def test_config0_full(ctx):
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0)
+    assert w.T == 256 and w.n_valid == 256
+    lp, ent, lse = ctx.rl_token_logprobs(w.H, w.W, w.tokens, w.mask)
+    _assert_status_ok(ctx)
+    olp, oent, olse = O.token_logprobs(_np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), w.mask.cpu().numpy())
+    assert np.abs(_np64(lp) - olp).max() <= TOL_LOGP
+    assert np.abs(_np64(ent) - oent).max() <= TOL_ENT
+    assert np.abs(_np64(lse) - olse).max() <= TOL_LOGP
+    _check_against_oracle(ctx, w)
+
+
+@pytest.mark.parametrize("cfg_id,prompts,L_max", [(1, 1, 96), (2, 1, 64), (3, 2, 64), (4, 4, 24)])
+def test_reduced_configs(ctx, cfg_id, prompts, L_max):
+    # same d, V, distributions and masks as the full configuration, fewer prompts / shorter rows
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(cfg_id, prompts=prompts, L_max=L_max)
+    assert w.n_valid > 128 and w.n_valid % 128 != 0      # several row tiles and a ragged tail
+    if cfg_id == 4:
+        r = w.rewards.cpu().numpy().reshape(-1, w.G)
+        assert (r.max(axis=1) == r.min(axis=1)).any()     # a zero-variance group is present
+        assert w.ref_logp is None and w.ent_coef > 0
+    _check_against_oracle(ctx, w)
+
+
+def test_clip_exercised_and_peaked_rows(ctx):
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, sigma_old=0.3, peaked_frac=0.05, seed=77)
+    out, oo = _check_against_oracle(ctx, w)
+    assert 0.05 < oo["clip_frac"] < 0.6                   # the clip is active on a real share of tokens
+    assert oo["entropy"][w.mask.cpu().numpy().astype(bool)].min() < 1.0   # peaked rows present
+    w = make_workload(4, prompts=2, L_max=16, sigma_old=0.3, seed=78, d=256, V=5000)
+    _check_against_oracle(ctx, w)
+
+
+@pytest.mark.parametrize("V,L_max", [(4096, 13), (4000, 16), (4100, 16), (300, 9), (9472 + 256 + 40, 11)])
+def test_ragged_shapes(ctx, V, L_max):
+    # rows not a multiple of 128, vocabulary not a multiple of 256 / 32, more than one vocabulary slab
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, L_max=L_max, V=V, seed=500 + V)
+    _check_against_oracle(ctx, w)
+
+
+def test_multiple_slabs(ctx):
+    # force several row slabs and several vocabulary slabs on a small case
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    c2 = Context(0)
+    try:
+        c2.set_slab_limits(128, 512)
+        w = make_workload(1, prompts=1, L_max=64, d=128, V=1500, seed=9)
+        assert w.n_valid > 256
+        _check_against_oracle(c2, w)
+    finally:
+        c2.close()
+
+
+def test_token_weight_accumulate_and_strides(ctx):
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, seed=31)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    tw = torch.rand(w.T, generator=g, device="cuda") / w.T
+    _check_against_oracle(ctx, w, token_weight=tw)
+    # accumulate_dW adds to what is there; strided H (ldH > d) is read correctly
+    adv_seq, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+    base = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask,
+                                      w.eps_low, w.eps_high, w.beta)
+    dW0 = base["dW"].clone()
+    Hwide = torch.zeros(w.T, w.d + 64, dtype=torch.bfloat16, device="cuda")
+    Hwide[:, :w.d] = w.H
+    acc = ctx.rl_policy_loss_fwd_bwd(Hwide[:, :w.d], w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask,
+                                     w.eps_low, w.eps_high, w.beta, accumulate_dW=True, dW=dW0.clone())
+    _assert_status_ok(ctx)
+    assert torch.allclose(acc["dW"], 2 * dW0, rtol=1e-5, atol=1e-12)
+    assert torch.equal(acc["dH"], base["dH"])
+    assert acc["loss"].item() == base["loss"].item()     # deterministic reductions
+
+
+def test_degenerate_batches(ctx):
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, seed=41)
+    adv = torch.ones(w.T, device="cuda")
+    # all rows masked: loss 0, gradients 0, no error
+    zero_mask = torch.zeros_like(w.mask)
+    out = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv, zero_mask,
+                                     w.eps_low, w.eps_high, w.beta)
+    _assert_status_ok(ctx)
+    assert out["loss"].item() == 0 and not out["dH"].any() and not out["dW"].any()
+    assert not out["logp"].any()
+    # a single valid row
+    one = torch.zeros_like(w.mask)
+    one[37] = 1
+    out = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv, one,
+                                     w.eps_low, w.eps_high, w.beta)
+    oo = O.policy_loss_fwd_bwd(_np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), _np64(w.old_logp),
+                               _np64(w.ref_logp), _np64(adv), one.cpu().numpy(), w.eps_low, w.eps_high, w.beta)
+    assert abs(out["loss"].item() - oo["loss"]) <= TOL_LOSS_REL * abs(oo["loss"]) + 1e-7
+    assert _rel(_np64(out["dH"]), oo["dH"]) <= TOL_GRAD_REL and _rel(_np64(out["dW"]), oo["dW"]) <= TOL_GRAD_REL
+    # mask = NULL means all valid
+    lp_all, _, _ = ctx.rl_token_logprobs(w.H, w.W, w.tokens, None)
+    lp_m, _, _ = ctx.rl_token_logprobs(w.H, w.W, w.tokens, torch.ones_like(w.mask))
+    assert torch.equal(lp_all, lp_m)
+    # T = 0
+    e = torch.empty(0, w.d, dtype=torch.bfloat16, device="cuda")
+    ei = torch.empty(0, dtype=torch.int32, device="cuda")
+    ef = torch.empty(0, dtype=torch.float32, device="cuda")
+    out = ctx.rl_policy_loss_fwd_bwd(e, w.W, ei, ef, ef, ef, None, 0.2, 0.2, 0.04, want_aux=False)
+    assert out["loss"].item() == 0 and not out["dW"].any()
+    _assert_status_ok(ctx)
+
+
+def test_error_reporting(ctx):
+    from paper_2512_21450_b200 import Context, RLHeadError
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, seed=51)
+    adv = torch.ones(w.T, device="cuda")
+
+    def status_of(fn):
+        with pytest.raises(RLHeadError) as e:
+            fn()
+        return e.value.status
+
+    args = (w.tokens, w.old_logp, w.ref_logp, adv, w.mask)
+    assert status_of(lambda: ctx.rl_policy_loss_fwd_bwd(w.H, w.W, *args, 1.5, 0.2, 0.04)) == 1     # eps_low
+    assert status_of(lambda: ctx.rl_policy_loss_fwd_bwd(w.H, w.W, *args, 0.2, -1.0, 0.04)) == 1    # eps_high
+    assert status_of(lambda: ctx.rl_policy_loss_fwd_bwd(w.H, w.W, *args, 0.2, 0.2, -0.1)) == 1     # beta
+    assert status_of(lambda: ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, None, adv, w.mask,
+                                                        0.2, 0.2, 0.04)) == 1                       # ref missing
+    H_bad = torch.zeros(w.T, 96, dtype=torch.bfloat16, device="cuda")
+    W_bad = torch.zeros(w.V, 96, dtype=torch.bfloat16, device="cuda")
+    assert status_of(lambda: ctx.rl_token_logprobs(H_bad, W_bad, w.tokens, w.mask)) == 2           # d % 64
+    H_off = torch.zeros(w.T * w.d + 8, dtype=torch.bfloat16, device="cuda")[4:4 + w.T * w.d].view(w.T, w.d)
+    assert status_of(lambda: ctx.rl_token_logprobs(H_off, w.W, w.tokens, w.mask)) == 3             # 8-byte offset
+    assert status_of(lambda: ctx.rl_grpo_advantages(w.rewards, 1)) == 2
+    assert status_of(lambda: ctx.rl_grpo_advantages(w.rewards, 5)) == 2
+    assert status_of(lambda: ctx.rl_grpo_advantages(w.rewards, 4, ddof=2, eps_std=1e-6)) == 1
+    # no workspace bound
+    c2 = Context(0)
+    try:
+        lib = c2.lib
+        import ctypes
+        s = lib.rl_token_logprobs(c2.handle, ctypes.c_void_p(w.H.data_ptr()), w.d, ctypes.c_void_p(w.W.data_ptr()),
+                                  w.d, ctypes.c_void_p(w.tokens.data_ptr()), None, w.T, w.d, w.V,
+                                  ctypes.c_void_p(adv.data_ptr()), None, None)
+        assert s == 4
+    finally:
+        c2.close()
+    # token id outside the vocabulary on a valid row -> latched device status, context still usable
+    bad = w.tokens.clone()
+    bad[5] = w.V + 3
+    ctx.rl_token_logprobs(w.H, w.W, bad, w.mask)
+    s, detail = ctx.last_device_status()
+    assert s == 7 and detail == 5
+    masked = w.mask.clone()
+    masked[5] = 0
+    ctx.rl_token_logprobs(w.H, w.W, bad, masked)           # ignored on a masked row
+    _assert_status_ok(ctx)
+    lp, _, _ = ctx.rl_token_logprobs(w.H, w.W, w.tokens, w.mask)
+    _assert_status_ok(ctx)
+    assert torch.isfinite(lp).all()
+
+
+def test_run_to_run_determinism(ctx):
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(1, prompts=1, L_max=40, seed=61)
+    adv_seq, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+    a = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, 0.2, 0.2, 0.04)
+    a = {k: v.clone() for k, v in a.items()}
+    b = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, 0.2, 0.2, 0.04)
+    for k in ("loss", "dH", "dW", "logp", "entropy"):
+        assert torch.equal(a[k], b[k]), k
