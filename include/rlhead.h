@@ -157,6 +157,33 @@ rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* ctx, const void* H_host, int64_t l
                                       float eps_low, float eps_high, float beta, float ent_coef,
                                       float* loss_host, float* metrics_host, void* dH, float* dW);
 
+/* rl_token_logprobs without any device allocation and without a context (the paper has no
+ * counterpart).  It is meant for callers that cannot allocate GPU memory when they need
+ * log-probabilities: a scoring pass that shares the GPU with a rollout engine which has already
+ * reserved almost all of its memory (the co-located setup of section 4.4 leaves no room for
+ * cudaMalloc to succeed), or code that must not pay the device-wide synchronisation cudaMalloc /
+ * cudaFree imply.  Inputs and outputs are the caller's device buffers exactly as in
+ * rl_token_logprobs; everything in between (compacted rows, row map, per-range softmax
+ * statistics, the status word) lives in a fixed 16 MiB device array that is part of the library
+ * image, so every GPU on which the library is loaded holds those 16 MiB until the process exits.
+ *   Limit: the forward scratch, about Tpad*(2*d + 280) + 70 KB bytes with Tpad = T rounded up to
+ *   128, must fit in 16 MiB - 256 B (e.g. T <= 3712 at d = 2048, T <= 1920 at d = 4096); larger
+ *   sizes are rejected with RL_ERR_WORKSPACE before anything is enqueued.
+ *   The call runs on the CURRENT device (device ordinal < 16) and enqueues on cuda_stream.  The
+ *   first call on each device looks up the array's device address and configures the kernel; make
+ *   that first call before any stream capture begins.  No cudaMalloc, cudaFree or other allocating
+ *   routine is called, on the first call or later.
+ *   All calls on a device share the one array and it keeps the previous call's contents; the call
+ *   clears what has to start at zero (status word, valid-row count) itself.  Two calls whose GPU
+ *   work overlaps (different streams, or different host threads on different streams) race on the
+ *   array: serialise them on one stream or with events.  Host-side the call is thread-safe.
+ *   dev_status (device, int32[2], may be NULL) receives {status, detail} as rl_last_device_status
+ *   would report them (RL_ERR_TOKEN_RANGE / RL_ERR_TIMEOUT), written in stream order. */
+rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH, const void* W,
+                                   int64_t ldW, const int32_t* tokens, const uint8_t* mask,
+                                   int64_t T, int64_t d, int64_t V,
+                                   float* logp, float* entropy, float* lse, int32_t* dev_status);
+
 /* Instrumentation.  rl_launch_count: kernels this context has launched so far.
  * rl_set_profiling(on): when on, every tensor-core launch is bracketed by a pair of CUDA events
  * on the context's stream (at most 2048 launches are kept between two reads).

@@ -76,6 +76,8 @@ def load_library():
     lib.rl_set_profiling.argtypes = [P, c_int]
     lib.rl_profile_read.argtypes = [P, POINTER(ctypes.c_double), POINTER(c_int64)]
     lib.rl_selftest_gemm.argtypes = [P, P, P, P, c_int64, c_int64, c_int64, c_int, c_int, c_int]
+    lib.rl_token_logprobs_static.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P, P]
+    lib.rl_token_logprobs_static.restype = c_int
     for name in ("rl_create", "rl_destroy", "rl_set_stream", "rl_workspace_bytes", "rl_workspace_bytes_host",
                  "rl_set_workspace", "rl_set_slab_limits", "rl_last_device_status", "rl_grpo_advantages", "rl_grpo_advantages_ex",
                  "rl_token_logprobs", "rl_policy_loss_fwd_bwd", "rl_policy_loss_fwd_bwd_ex",
@@ -277,3 +279,22 @@ def rl_token_logprobs(H, W, tokens, mask=None):
 def rl_policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta, **kw):
     return default_context(W.device.index or 0).rl_policy_loss_fwd_bwd(
         H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta, **kw)
+
+
+def rl_token_logprobs_static(H, W, tokens, mask, logp, entropy=None, lse=None, dev_status=None):
+    """Allocation-free log-probabilities: no context, no workspace, outputs preallocated by the caller.
+
+    For callers that cannot allocate device memory at call time (see include/rlhead.h).  Runs on
+    the current device and the current torch stream; scratch is the library's fixed 16 MiB device
+    array, so overlapping calls race and sizes beyond the limit raise RL_ERR_WORKSPACE.
+    """
+    lib = load_library()
+    T, d = H.shape
+    V = W.shape[0]
+    assert H.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and tokens.dtype == torch.int32
+    assert logp.dtype == torch.float32 and logp.numel() == T
+    stream = c_void_p(torch.cuda.current_stream(H.device).cuda_stream)
+    _check(lib.rl_token_logprobs_static(stream, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0), _ptr(tokens),
+                                        _ptr(mask), T, d, V, _ptr(logp), _ptr(entropy), _ptr(lse), _ptr(dev_status)),
+           "rl_token_logprobs_static")
+    return logp

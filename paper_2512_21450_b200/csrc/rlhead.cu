@@ -6,6 +6,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "rlhead.h"
@@ -631,6 +632,97 @@ rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, in
   else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, -1, ta, tb, sh, ep);
   else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, -1, ta, tb, sh, ep);
   else launch_gemm<EpiAcc, 1, 1>(c, -1, ta, tb, sh, ep);
+  return cuda_ok();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of rl_token_logprobs.  Its scratch (compacted rows, row map, per-range
+// softmax statistics, status word) lives in one file-scope device array instead of a caller
+// workspace, so the call path contains no device allocation at all.
+namespace {
+constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // 16 MiB per GPU that loads the library
+constexpr size_t kStaticHeaderBytes = 256;                  // status word, then the workspace proper
+constexpr int kStaticMaxDevices = 16;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+struct StaticSlot {
+  bool ready;
+  rl_ctx ctx;
+};
+StaticSlot g_static_slot[kStaticMaxDevices];
+std::mutex g_static_mutex;
+}  // namespace
+
+rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH, const void* W, int64_t ldW,
+                                   const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
+                                   float* logp, float* entropy, float* lse, int32_t* dev_status) {
+  rl_status s = check_hw(H, ldH, W, ldW, T, d, V);
+  if (s != RL_OK) return s;
+  if (T > 0 && (!tokens || !logp)) return RL_ERR_INVALID_ARG;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) return RL_ERR_CUDA;
+  if (device < 0 || device >= kStaticMaxDevices) return RL_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticSlot& slot = g_static_slot[device];
+  if (!slot.ready) {
+    // once per device, with that device current: the array's name is only a host-side handle;
+    // the address kernels and memsets can use comes from cudaGetSymbolAddress
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return RL_ERR_CUDA;
+    if (prop.major != 10) return RL_ERR_UNSUPPORTED_ARCH;
+    unsigned char* base = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&base), g_static_scratch) != cudaSuccess || !base)
+      return RL_ERR_CUDA;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+      return RL_ERR_CUDA;
+    if (set_smem_attr<EpiStats, 0, 0>() != cudaSuccess) return RL_ERR_CUDA;
+    rl_ctx& c = slot.ctx;
+    memset(&c, 0, sizeof(c));
+    c.device = device;
+    c.n_sm = prop.multiProcessorCount;
+    c.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    c.dstatus = reinterpret_cast<DevStatus*>(base);
+    c.ws = base + kStaticHeaderBytes;
+    c.ws_bytes = kStaticScratchBytes - kStaticHeaderBytes;
+    c.slab_rows = kSlabRowsMax;
+    c.slab_cols = kSlabColsMax;
+    slot.ready = true;
+  }
+  rl_ctx* c = &slot.ctx;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  if (T == 0) return RL_OK;
+  // only the forward part of the workspace layout is needed: everything before the gradient slab
+  const WsLayout L = ws_layout(c, T, d, V, false);
+  if (L.G > c->ws_bytes) return RL_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(c->ws);
+  // the array keeps the previous call's contents: the status word and the valid-row count start at zero
+  if (cudaMemsetAsync(c->dstatus, 0, sizeof(DevStatus), c->stream) != cudaSuccess) return RL_ERR_CUDA;
+  cudaMemsetAsync(logp, 0, (size_t)T * 4, c->stream);
+  if (entropy) cudaMemsetAsync(entropy, 0, (size_t)T * 4, c->stream);
+  if (lse) cudaMemsetAsync(lse, 0, (size_t)T * 4, c->stream);
+  int n_tiles = 0;
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &n_tiles)) != RL_OK) return s;
+  LossParams p;
+  memset(&p, 0, sizeof(p));
+  p.partials = reinterpret_cast<const float4*>(ws + L.partials);
+  p.part_stride = L.Tpad;
+  p.n_tiles = n_tiles;
+  p.n_ctas = c->n_sm;
+  p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
+  p.with_loss = 0;
+  p.lse_c = reinterpret_cast<float*>(ws + L.lse_c);
+  p.ent_c = reinterpret_cast<float*>(ws + L.ent_c);
+  p.logp_out = logp;
+  p.ent_out = entropy;
+  p.lse_out = lse;
+  int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
+  if (blocks > 1024) blocks = 1024;
+  combine_loss_kernel<<<blocks, kLossThreads, 0, c->stream>>>(p, c->dstatus);
+  if (dev_status &&
+      cudaMemcpyAsync(dev_status, c->dstatus, 2 * sizeof(int32_t), cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
+    return RL_ERR_CUDA;
   return cuda_ok();
 }
 
