@@ -68,6 +68,11 @@ rl_status rl_workspace_bytes(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_
  * chosen so that the tile counts of the three backward passes are multiples of 148 SMs for
  * d = 2048, 2560 and 3584).  Changes what rl_workspace_bytes() returns: call it first. */
 rl_status rl_set_slab_limits(rl_ctx* ctx, int max_rows, int max_cols);
+/* Tile shape of the tensor-core passes: 1 = one CTA per 128x256 output tile, 2 = CTA pairs
+ * (clusters of two SMs, tcgen05 cta_group::2) on 256x256 tiles, which halves the shared-memory
+ * and L2 traffic of the B operand.  2 is the default when the device can co-schedule CTA pairs;
+ * asking for 2 when it cannot returns RL_ERR_UNSUPPORTED_ARCH.  Results are identical up to fp32 summation order inside the tensor core. */
+rl_status rl_set_cta_group(rl_ctx* ctx, int cta_group);
 /* Caller-owned device scratch, 256-byte aligned; must outlive the calls that use it. */
 rl_status rl_set_workspace(rl_ctx* ctx, void* dev_ptr, size_t bytes);
 

@@ -61,6 +61,8 @@ def load_library():
     lib.rl_workspace_bytes_host.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
     lib.rl_set_workspace.argtypes = [P, P, c_size_t]
     lib.rl_set_slab_limits.argtypes = [P, c_int, c_int]
+    lib.rl_set_cta_group.argtypes = [P, c_int]
+    lib.rl_set_cta_group.restype = c_int
     lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
     lib.rl_grpo_advantages.argtypes = [P, P, c_int64, c_int, P]
     lib.rl_grpo_advantages_ex.argtypes = [P, P, c_int64, c_int, c_int, c_float, P, c_int64, P, P]
@@ -140,6 +142,9 @@ class Context:
 
     def set_slab_limits(self, max_rows=0, max_cols=0):
         _check(self.lib.rl_set_slab_limits(self.handle, max_rows, max_cols), "rl_set_slab_limits")
+
+    def set_cta_group(self, cta_group):
+        _check(self.lib.rl_set_cta_group(self.handle, cta_group), "rl_set_cta_group")
 
     def last_device_status(self):
         detail = c_int32()

@@ -120,7 +120,9 @@ struct EpiGrad {
     st.y = st.valid ? p.tokens_c[gr] : -1;
   }
   __device__ static __forceinline__ void chunk(const Params& p, State& st, int m_tile, int n_tile, int c,
-                                               int row_in_tile, int, const float (&v)[32]) {
+                                               int row_in_tile, int m_rows, const float (&v)[32]) {
+    // a CTA pair may own a 128-row tile that lies wholly past the slab's rows: nothing to write
+    if (m_tile * BM >= ((m_rows + BM - 1) / BM) * BM) return;
     const int col_l = n_tile * BN + c * 32;
     const int col_g = p.vocab_base + col_l;
     const int nvalid = p.V - col_g;

@@ -1,18 +1,28 @@
 // Persistent, warp-specialised bf16 GEMM main loop for sm_100a with pluggable epilogues.
 //
-//   warp 0      : TMA producer (one lane) - streams 128x64 A tiles and 256x64 B tiles into a
-//                 4-stage shared-memory ring, 128-byte swizzled.
-//   warp 1      : allocates tensor memory; one lane issues tcgen05.mma (128x256x16 per
-//                 instruction) into one of two 256-column fp32 accumulators.
+//   warp 0      : TMA producer (one lane) - streams A and B k-slices (64 elements of K) into a
+//                 shared-memory ring, 128-byte swizzled.
+//   warp 1      : allocates tensor memory; one lane issues tcgen05.mma into one of two
+//                 256-column fp32 accumulators.
 //   warps 2..5  : epilogue - each warp owns the 32 tensor-memory lanes (tile rows) that its
 //                 rank modulo 4 may read, pulls the accumulator out in 32-column chunks and
 //                 hands them to the epilogue functor.  While they drain accumulator a, the MMA
 //                 warp already fills accumulator a^1.
 //
+// CG = 1: one CTA per 128x256 output tile (4 stages of 16 KB A + 32 KB B).
+// CG = 2: a cluster of two CTAs (one SM pair) per 256x256 output tile.  Each CTA stages its own
+//         128 rows of A and 128 of the 256 columns of B (6 stages of 16 KB + 16 KB), the even
+//         CTA issues tcgen05.mma.cta_group::2 (M = 256) which reads both halves of B and writes
+//         128 accumulator rows into each CTA's tensor memory; both CTAs run their own epilogue.
+//         All TMA completions of a stage are counted on the even CTA's barrier; stage-free and
+//         accumulator-ready signals are multicast to both CTAs by tcgen05.commit; the odd CTA's
+//         epilogue reports "accumulator drained" to the even CTA with a remote mbarrier arrive.
+//         No TMA load is multicast.
+//
 // Either operand may be K-major (its global tensor is [rows, K], K contiguous) or MN-major
 // (its global tensor is [K, rows], rows contiguous).  A K-major tile is one 2-D TMA box
 // {64 k, rows}; an MN-major tile is one 3-D box {64 rows, 64 k, rows/64}, which lands in shared
-// memory as rows/64 chunks of 8 KB, each chunk 64 k-lines of 128 bytes.
+// memory as rows/64 panels of 8 KB, each panel 64 k-lines of 128 bytes.
 //
 // Every wait is bounded: when one runs out the block raises a shared abort flag, every role
 // leaves its loop, the status word is latched and the block still frees its tensor memory.
@@ -23,17 +33,24 @@
 
 namespace rlh {
 
-constexpr int BM = 128;
-constexpr int BN = 256;
+constexpr int BM = 128;   // accumulator rows per CTA
+constexpr int BN = 256;   // accumulator columns
 constexpr int BK = 64;
-constexpr int kStages = 4;
 constexpr int kAStageBytes = BM * BK * 2;
-constexpr int kBStageBytes = BN * BK * 2;
-constexpr int kStageBytes = kAStageBytes + kBStageBytes;
 constexpr int kGemmThreads = 192;
-constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024;  // + slack for 1024-byte alignment
+constexpr int kGemmSmemBytes = 192 * 1024 + 1024;  // ring + slack for 1024-byte alignment
 constexpr int kTmemCols = 512;
 constexpr int kMaxSplit = 16;
+
+template <int CG>
+struct StageCfg {
+  static constexpr int kBRows = BN / CG;                    // B rows (output columns) staged per CTA
+  static constexpr int kBBytes = kBRows * BK * 2;
+  static constexpr int kStageBytes = kAStageBytes + kBBytes;
+  static constexpr int kStages = (192 * 1024) / kStageBytes;  // 4 (CG = 1) or 6 (CG = 2)
+  static constexpr uint32_t kTxBytes = uint32_t(kStageBytes) * CG;  // bytes counted on the issuing CTA's barrier
+};
+constexpr int kMaxStages = 6;
 
 // Device status word shared by all kernels of a context.
 struct DevStatus {
@@ -58,18 +75,20 @@ struct GemmShape {
   int n_tiles;      // number of 256-wide column tiles
   int n_range;      // consecutive column tiles per work unit; 0 = choose so that units fill the SMs
   int skip_if_k0;   // nothing to do at all when K is empty (otherwise the epilogue sees zeros)
+  int n_fastest;    // 1: consecutive units walk the column ranges of one row tile first
   // coordinate offsets into the operands' global tensors
   int a_mn_off, a_k_off, b_mn_off, b_k_off;
 };
 
-// Number of vocabulary ranges each 128-row tile is split into so that (row tiles x ranges) fills
-// the machine: minimises waves * tiles-per-range, preferring fewer ranges on ties.
-__host__ __device__ inline int choose_split(int m_tiles, int n_tiles, int n_ctas) {
+// Number of vocabulary ranges each row tile is split into so that (row tiles x ranges) fills the
+// machine: minimises waves * tiles-per-range, preferring fewer ranges on ties.  m_units = row
+// tiles of 128*CG rows, n_workers = CTAs (CG = 1) or CTA pairs (CG = 2).
+__host__ __device__ inline int choose_split(int m_units, int n_tiles, int n_workers) {
   int best = 1;
   long best_cost = -1;
   for (int s = 1; s <= kMaxSplit && s <= n_tiles; ++s) {
-    long units = (long)m_tiles * s;
-    long waves = (units + n_ctas - 1) / n_ctas;
+    long units = (long)m_units * s;
+    long waves = (units + n_workers - 1) / n_workers;
     long cost = waves * ((n_tiles + s - 1) / s);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
   }
@@ -77,23 +96,32 @@ __host__ __device__ inline int choose_split(int m_tiles, int n_tiles, int n_ctas
 }
 
 struct GemmExtents {
-  int m_rows, m_tiles, k_blocks, n_range, n_ranges, n_units;
+  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units;
 };
 
-__device__ __forceinline__ GemmExtents gemm_extents(const GemmShape& sh) {
+// cg = CTAs per output row tile, n_workers = gridDim.x / cg.
+__host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_valid, int cg, int n_workers) {
   GemmExtents e;
-  int nv = sh.n_valid ? *sh.n_valid : 0;
-  e.m_rows = sh.m_dyn ? min(max(nv - sh.m_dyn_off, 0), sh.m_rows_cap) : sh.m_rows_cap;
-  int k_len = sh.k_dyn ? min(max(nv - sh.k_dyn_off, 0), sh.k_cap) : sh.k_cap;
-  e.m_tiles = (e.m_rows + BM - 1) / BM;
+  int m = n_valid - sh.m_dyn_off;
+  m = m < 0 ? 0 : (m > sh.m_rows_cap ? sh.m_rows_cap : m);
+  e.m_rows = sh.m_dyn ? m : sh.m_rows_cap;
+  int k = n_valid - sh.k_dyn_off;
+  k = k < 0 ? 0 : (k > sh.k_cap ? sh.k_cap : k);
+  const int k_len = sh.k_dyn ? k : sh.k_cap;
+  e.m_units = (e.m_rows + BM * cg - 1) / (BM * cg);
   e.k_blocks = (k_len + BK - 1) / BK;
-  int split = sh.n_range > 0 ? 0 : choose_split(e.m_tiles, sh.n_tiles, (int)gridDim.x);
-  e.n_range = sh.n_range > 0 ? sh.n_range : (sh.n_tiles + split - 1) / max(split, 1);
-  e.n_range = max(e.n_range, 1);
+  const int split = sh.n_range > 0 ? 1 : choose_split(e.m_units, sh.n_tiles, n_workers);
+  e.n_range = sh.n_range > 0 ? sh.n_range : (sh.n_tiles + split - 1) / split;
+  if (e.n_range < 1) e.n_range = 1;
   e.n_ranges = (sh.n_tiles + e.n_range - 1) / e.n_range;
-  e.n_units = e.m_tiles * e.n_ranges;
+  e.n_units = e.m_units * e.n_ranges;
   if (sh.skip_if_k0 && e.k_blocks == 0) e.n_units = 0;
   return e;
+}
+
+__device__ __forceinline__ void unit_coords(const GemmShape& sh, const GemmExtents& ex, int u, int& mu, int& nr) {
+  if (sh.n_fastest) { nr = u % ex.n_ranges; mu = u / ex.n_ranges; }
+  else              { mu = u % ex.m_units;  nr = u / ex.m_units; }
 }
 
 // Epilogue functor contract (all methods run in the 128 epilogue threads, one tile row each):
@@ -101,13 +129,16 @@ __device__ __forceinline__ GemmExtents gemm_extents(const GemmShape& sh) {
 //     static void begin_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows);
 //     static void chunk(const Params&, State&, int m_tile, int n_tile, int chunk, int row_in_tile, int m_rows, const float (&v)[32]);
 //     static void end_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows); };
-template <class Epi, int A_MN, int B_MN>
+// m_tile counts 128-row tiles.
+template <class Epi, int A_MN, int B_MN, int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const GemmShape sh, const typename Epi::Params ep, DevStatus* status) {
+  using Cfg = StageCfg<CG>;
+  constexpr int kStages = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_full[kStages];
-  __shared__ __align__(8) uint64_t bar_empty[kStages];
+  __shared__ __align__(8) uint64_t bar_full[kMaxStages];
+  __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
   __shared__ __align__(8) uint64_t bar_acc_full[2];
   __shared__ __align__(8) uint64_t bar_acc_empty[2];
   __shared__ __align__(8) uint64_t bar_drain;
@@ -117,10 +148,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;   // position in the CTA pair
+  const int worker = blockIdx.x / CG;
+  const int n_workers = gridDim.x / CG;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&bar_acc_full[a]), 1); mbar_init(smem_u32(&bar_acc_empty[a]), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&bar_acc_full[a]), 1); mbar_init(smem_u32(&bar_acc_empty[a]), 4 * CG); }
     mbar_init(smem_u32(&bar_drain), 1);
     abort_flag = 0;
     fence_mbar_init();
@@ -128,25 +162,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     prefetch_tmap(&tmB);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_smem), kTmemCols);
-    tmem_relinquish();
+    if (CG == 2) { tmem_alloc_pair(smem_u32(&tmem_base_smem), kTmemCols); tmem_relinquish_pair(); }
+    else         { tmem_alloc(smem_u32(&tmem_base_smem), kTmemCols);      tmem_relinquish(); }
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();   // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_smem;
   volatile int* abort_p = &abort_flag;
 
-  const GemmExtents ex = gemm_extents(sh);
+  const GemmExtents ex = gemm_extents(sh, sh.n_valid ? *sh.n_valid : 0, CG, n_workers);
 
   if (warp == 0) {
-    // ------------------------------------------------------------- TMA producer
+    // ------------------------------------------------------------- TMA producer (both CTAs)
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < ex.n_units && ok; u += gridDim.x) {
-        const int m = u % ex.m_tiles, nr = u / ex.m_tiles;
+      for (int u = worker; u < ex.n_units && ok; u += n_workers) {
+        int mu, nr;
+        unit_coords(sh, ex, u, mu, nr);
+        const int m = mu * CG + (int)rank;
         const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
         for (int n = n0; n < n1 && ok; ++n) {
           for (int kb = 0; kb < ex.k_blocks; ++kb) {
@@ -155,19 +192,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               ok = false;
               break;
             }
-            const uint32_t full = smem_u32(&bar_full[stage]);
-            const uint32_t a_dst = tiles_base + stage * kAStageBytes;
-            const uint32_t b_dst = tiles_base + kStages * kAStageBytes + stage * kBStageBytes;
-            mbar_arrive_expect_tx(full, kStageBytes);
-            if (A_MN) tma_load_3d(a_dst, &tmA, full, 0, sh.a_k_off + kb * BK, (sh.a_mn_off + m * BM) / 64);
-            else      tma_load_2d(a_dst, &tmA, full, sh.a_k_off + kb * BK, sh.a_mn_off + m * BM);
-            if (B_MN) tma_load_3d(b_dst, &tmB, full, 0, sh.b_k_off + kb * BK, (sh.b_mn_off + n * BN) / 64);
-            else      tma_load_2d(b_dst, &tmB, full, sh.b_k_off + kb * BK, sh.b_mn_off + n * BN);
+            const uint32_t full_local = smem_u32(&bar_full[stage]);
+            const uint32_t a_dst = tiles_base + stage * Cfg::kStageBytes;
+            const uint32_t b_dst = a_dst + kAStageBytes;
+            const int a_row = sh.a_mn_off + m * BM;
+            const int b_row = sh.b_mn_off + n * BN + (int)rank * Cfg::kBRows;
+            if (CG == 1) {
+              mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
+              if (A_MN) tma_load_3d(a_dst, &tmA, full_local, 0, sh.a_k_off + kb * BK, a_row / 64);
+              else      tma_load_2d(a_dst, &tmA, full_local, sh.a_k_off + kb * BK, a_row);
+              if (B_MN) tma_load_3d(b_dst, &tmB, full_local, 0, sh.b_k_off + kb * BK, b_row / 64);
+              else      tma_load_2d(b_dst, &tmB, full_local, sh.b_k_off + kb * BK, b_row);
+            } else {
+              // the even CTA's barrier counts the bytes of both CTAs' copies
+              if (rank == 0) mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
+              const uint32_t full = mapa_cluster(full_local, 0);
+              if (A_MN) tma_load_3d_pair(a_dst, &tmA, full, 0, sh.a_k_off + kb * BK, a_row / 64);
+              else      tma_load_2d_pair(a_dst, &tmA, full, sh.a_k_off + kb * BK, a_row);
+              if (B_MN) tma_load_3d_pair(b_dst, &tmB, full, 0, sh.b_k_off + kb * BK, b_row / 64);
+              else      tma_load_2d_pair(b_dst, &tmB, full, sh.b_k_off + kb * BK, b_row);
+            }
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
       }
-      if (!ok) {
+      if (!ok && (CG == 1 || rank == 0)) {
         // let copies that were already issued land before the block's shared memory goes away
         for (int s = 0; s < kStages; ++s) {
           uint32_t p = (s < stage) ? phase : (phase ^ 1u);
@@ -176,11 +225,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(BM, BN, A_MN, B_MN);
+    // ------------------------------------------------------------- MMA issuer (even CTA of a pair)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(BM * CG, BN, A_MN, B_MN);
       // K-major: 8-row groups 1024 B apart, 32 bytes per 16-element k step.
-      // MN-major: 64-row chunks 8192 B apart, 8-k-line groups 1024 B apart, 2048 B per k step.
+      // MN-major: 64-row panels 8192 B apart, 8-k-line groups 1024 B apart, 2048 B per k step.
       constexpr uint64_t a_hi = A_MN ? make_smem_desc_hi(8192, 1024) : make_smem_desc_hi(16, 1024);
       constexpr uint64_t b_hi = B_MN ? make_smem_desc_hi(8192, 1024) : make_smem_desc_hi(16, 1024);
       constexpr uint32_t a_kstep = A_MN ? 2048 : 32;
@@ -190,12 +239,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t t = 0;
       bool ok = true;
       if (ex.k_blocks > 0) {
-        for (int u = blockIdx.x; u < ex.n_units && ok; u += gridDim.x) {
-          const int nr = u / ex.m_tiles;
+        for (int u = worker; u < ex.n_units && ok; u += n_workers) {
+          int mu, nr;
+          unit_coords(sh, ex, u, mu, nr);
           const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
           for (int n = n0; n < n1 && ok; ++n, ++t) {
             const uint32_t a = t & 1u, round = t >> 1;
-            if (!mbar_wait_bounded(smem_u32(&bar_acc_empty[a]), (round & 1u) ^ 1u, abort_p)) {
+            if (!mbar_wait_bounded_cluster(smem_u32(&bar_acc_empty[a]), (round & 1u) ^ 1u, abort_p)) {
               latch_status(status, kStatusTimeout, (2 << 28) | (blockIdx.x << 8) | a);
               ok = false;
               break;
@@ -203,47 +253,55 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + a * BN;
             for (int kb = 0; kb < ex.k_blocks; ++kb) {
-              if (!mbar_wait_bounded(smem_u32(&bar_full[stage]), phase, abort_p)) {
+              if (!mbar_wait_bounded_cluster(smem_u32(&bar_full[stage]), phase, abort_p)) {
                 latch_status(status, kStatusTimeout, (3 << 28) | (blockIdx.x << 8) | stage);
                 ok = false;
                 break;
               }
               tc_fence_after();
-              const uint32_t a_src = tiles_base + stage * kAStageBytes;
-              const uint32_t b_src = tiles_base + kStages * kAStageBytes + stage * kBStageBytes;
+              const uint32_t a_src = tiles_base + stage * Cfg::kStageBytes;
+              const uint32_t b_src = a_src + kAStageBytes;
 #pragma unroll
               for (int k = 0; k < BK / 16; ++k) {
-                umma_bf16(d_tmem, smem_desc(a_hi, a_src + k * a_kstep), smem_desc(b_hi, b_src + k * b_kstep),
-                          idesc, (kb | k) != 0 ? 1u : 0u);
+                const uint64_t da = smem_desc(a_hi, a_src + k * a_kstep), db = smem_desc(b_hi, b_src + k * b_kstep);
+                if (CG == 2) umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                else         umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
               }
-              umma_commit(smem_u32(&bar_empty[stage]));
+              if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_empty[stage]), 3);
+              else         umma_commit(smem_u32(&bar_empty[stage]));
               if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
-            if (ok) umma_commit(smem_u32(&bar_acc_full[a]));
+            if (ok) {
+              if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_acc_full[a]), 3);
+              else         umma_commit(smem_u32(&bar_acc_full[a]));
+            }
           }
         }
       }
       // every UMMA issued above has to retire before tensor memory is released
-      umma_commit(smem_u32(&bar_drain));
+      if (CG == 2) umma_commit_pair(smem_u32(&bar_drain));
+      else         umma_commit(smem_u32(&bar_drain));
       bool drained = false;
       for (int it = 0; it < (1 << 22) && !drained; ++it) drained = mbar_try_wait(smem_u32(&bar_drain), 0) != 0;
       if (!drained) latch_status(status, kStatusTimeout, (4 << 28) | (blockIdx.x << 8));
     }
   } else {
-    // ------------------------------------------------------------- epilogue warps
+    // ------------------------------------------------------------- epilogue warps (both CTAs)
     const int q = warp & 3;
     const int row_in_tile = q * 32 + lane;
     typename Epi::State st;
     uint32_t t = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < ex.n_units && ok; u += gridDim.x) {
-      const int m = u % ex.m_tiles, nr = u / ex.m_tiles;
+    for (int u = worker; u < ex.n_units && ok; u += n_workers) {
+      int mu, nr;
+      unit_coords(sh, ex, u, mu, nr);
+      const int m = mu * CG + (int)rank;
       const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
       Epi::begin_unit(ep, st, m, nr, row_in_tile, ex.m_rows);
       for (int n = n0; n < n1 && ok; ++n, ++t) {
         const uint32_t a = t & 1u, round = t >> 1;
         if (ex.k_blocks > 0) {
-          if (!mbar_wait_bounded(smem_u32(&bar_acc_full[a]), round & 1u, abort_p)) {
+          if (!mbar_wait_bounded_cluster(smem_u32(&bar_acc_full[a]), round & 1u, abort_p)) {
             latch_status(status, kStatusTimeout, (5 << 28) | (blockIdx.x << 8) | a);
             ok = false;
           }
@@ -270,7 +328,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (ex.k_blocks > 0) {
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[a]));
+          if (lane == 0) {
+            if (CG == 2 && rank != 0) mbar_arrive_cluster(mapa_cluster(smem_u32(&bar_acc_empty[a]), 0));
+            else                      mbar_arrive(smem_u32(&bar_acc_empty[a]));
+          }
         }
       }
       if (ok) Epi::end_unit(ep, st, m, nr, row_in_tile, ex.m_rows);
@@ -279,10 +340,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();   // the pair's UMMAs have retired and both epilogues are done
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (CG == 2) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else         tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 

@@ -31,6 +31,8 @@ struct rl_ctx {
   EncodeTiledFn encode;
   int slab_rows;  // rows of one gradient slab (multiple of 128)
   int slab_cols;  // vocabulary columns of one gradient slab (multiple of 256)
+  int cta_group;  // 1: one CTA per 128x256 tile; 2: CTA pairs on 256x256 tiles
+  int grid[3];    // persistent grid for cta_group 1 and 2 (index = cta_group)
   long long launches;  // kernels launched by this context so far
   // optional per-kernel timing: event pairs around every tensor-core launch, by kernel kind
   int prof_on;
@@ -114,9 +116,17 @@ bool map_mnmajor(rl_ctx* c, CUtensorMap* m, const void* base, uint64_t k_rows, u
 
 template <class Epi, int A_MN, int B_MN>
 cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kGemmSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               kGemmSmemBytes);
 }
+
+// Rows of B that one CTA stages per k-slice (box height of a K-major B map) and the number of
+// 64-wide panels of an MN-major B map, for the context's CTA grouping.
+inline uint32_t b_box_rows(const rl_ctx* c) { return BN / c->cta_group; }
+inline uint32_t b_box_panels(const rl_ctx* c) { return BN / 64 / c->cta_group; }
 
 template <class Epi, int A_MN, int B_MN>
 void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const GemmShape& sh,
@@ -127,7 +137,25 @@ void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b
       if (!c->prof_ev[c->prof_used][e]) cudaEventCreate(&c->prof_ev[c->prof_used][e]);
     cudaEventRecord(c->prof_ev[c->prof_used][0], c->stream);
   }
-  gemm_kernel<Epi, A_MN, B_MN><<<c->n_sm, kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, sh, ep, c->dstatus);
+  if (c->cta_group == 2) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->grid[2]);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = kGemmSmemBytes;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, gemm_kernel<Epi, A_MN, B_MN, 2>, a, b, sh, ep, c->dstatus);
+  } else {
+    gemm_kernel<Epi, A_MN, B_MN, 1><<<c->grid[1], kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, sh, ep,
+                                                                                            c->dstatus);
+  }
   c->launches++;
   if (timed) {
     cudaEventRecord(c->prof_ev[c->prof_used][1], c->stream);
@@ -155,7 +183,8 @@ inline rl_status cuda_ok() { return cudaGetLastError() == cudaSuccess ? RL_OK : 
 
 // Mask scan + row compaction + forward statistics.  Leaves per-range partials in the workspace.
 rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, const void* W, int64_t ldW,
-                      const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d, int64_t V, int* n_tiles_out) {
+                      const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
+                      GemmShape* shape_out) {
   char* ws = static_cast<char*>(c->ws);
   int* row_map = reinterpret_cast<int*>(ws + L.row_map);
   int* tokens_c = reinterpret_cast<int*>(ws + L.tokens_c);
@@ -166,7 +195,7 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   c->launches += 2;
   CUtensorMap tmA, tmB;
   if (!map_kmajor(c, &tmA, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM)) return RL_ERR_CUDA;
-  if (!map_kmajor(c, &tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, BN)) return RL_ERR_CUDA;
+  if (!map_kmajor(c, &tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_rows(c))) return RL_ERR_CUDA;
   GemmShape sh;
   memset(&sh, 0, sizeof(sh));
   sh.n_valid = &c->dstatus->n_valid;
@@ -181,7 +210,7 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   ep.part_stride = L.Tpad;
   ep.V = (int)V;
   launch_gemm<EpiStats, 0, 0>(c, 0, tmA, tmB, sh, ep);
-  *n_tiles_out = sh.n_tiles;
+  *shape_out = sh;
   return cuda_ok();
 }
 
@@ -220,6 +249,10 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->ws_bytes = 0;
   c->slab_rows = kSlabRowsMax;
   c->slab_cols = kSlabColsMax;
+  c->cta_group = 1;
+  c->grid[0] = 0;
+  c->grid[1] = c->n_sm;
+  c->grid[2] = c->n_sm / 2 * 2;
   c->launches = 0;
   c->prof_on = 0;
   c->prof_used = 0;
@@ -238,6 +271,31 @@ rl_status rl_create(rl_ctx** out, int device) {
             set_smem_attr<EpiAcc, 0, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 0, 1>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess;
   if (!ok) { cudaFree(c->dstatus); delete c; return RL_ERR_CUDA; }
+  {
+    // how many CTA pairs can be resident at once (pairs must share a TPC): the persistent grid
+    // of the paired kernels must not exceed it
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->grid[2]);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = kGemmSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, gemm_kernel<EpiAcc, 0, 0, 2>, &cfg) == cudaSuccess &&
+        n_clusters > 0) {
+      if (2 * n_clusters < c->grid[2]) c->grid[2] = 2 * n_clusters;
+    } else {
+      cudaGetLastError();
+      c->grid[2] = 0;   // paired kernels unavailable
+    }
+    if (c->grid[2] >= 2) c->cta_group = 2;   // default: CTA pairs
+  }
   *out = c;
   return RL_OK;
 }
@@ -267,6 +325,14 @@ rl_status rl_workspace_bytes(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t*
 rl_status rl_workspace_bytes_host(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t* bytes) {
   if (!c || !bytes || T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
   *bytes = ws_layout(c, T, d, V, true).total;
+  return RL_OK;
+}
+
+rl_status rl_set_cta_group(rl_ctx* c, int cta_group) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  if (cta_group != 1 && cta_group != 2) return RL_ERR_INVALID_ARG;
+  if (cta_group == 2 && c->grid[2] < 2) return RL_ERR_UNSUPPORTED_ARCH;
+  c->cta_group = cta_group;
   return RL_OK;
 }
 
@@ -369,14 +435,15 @@ rl_status rl_token_logprobs(rl_ctx* c, const void* H, int64_t ldH, const void* W
   cudaMemsetAsync(logp, 0, (size_t)T * 4, c->stream);
   if (entropy) cudaMemsetAsync(entropy, 0, (size_t)T * 4, c->stream);
   if (lse) cudaMemsetAsync(lse, 0, (size_t)T * 4, c->stream);
-  int n_tiles = 0;
-  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &n_tiles)) != RL_OK) return s;
+  GemmShape fwd_shape;
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &fwd_shape)) != RL_OK) return s;
   LossParams p;
   memset(&p, 0, sizeof(p));
   p.partials = reinterpret_cast<const float4*>(ws + L.partials);
   p.part_stride = L.Tpad;
-  p.n_tiles = n_tiles;
-  p.n_ctas = c->n_sm;
+  p.fwd_shape = fwd_shape;
+  p.fwd_cg = c->cta_group;
+  p.fwd_workers = c->grid[c->cta_group] / c->cta_group;
   p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
   p.with_loss = 0;
   p.lse_c = reinterpret_cast<float*>(ws + L.lse_c);
@@ -428,16 +495,17 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   if (o.entropy_out) cudaMemsetAsync(o.entropy_out, 0, (size_t)T * 4, st);
 
   // ---- forward: statistics per (row, vocabulary range)
-  int n_tiles = 0;
-  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &n_tiles)) != RL_OK) return s;
+  GemmShape fwd_shape;
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &fwd_shape)) != RL_OK) return s;
 
   // ---- merge + per-token loss, coefficients of the backward pass
   LossParams p;
   memset(&p, 0, sizeof(p));
   p.partials = reinterpret_cast<const float4*>(ws + L.partials);
   p.part_stride = L.Tpad;
-  p.n_tiles = n_tiles;
-  p.n_ctas = c->n_sm;
+  p.fwd_shape = fwd_shape;
+  p.fwd_cg = c->cta_group;
+  p.fwd_workers = c->grid[c->cta_group] / c->cta_group;
   p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
   p.old_logp = old_logp;
   p.ref_logp = ref_logp;
@@ -470,11 +538,11 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
 
   CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn;
   bool ok = map_kmajor(c, &tmHc_k, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM) &&
-            map_kmajor(c, &tmW_k, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, BN) &&
+            map_kmajor(c, &tmW_k, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_rows(c)) &&
             map_kmajor(c, &tmG_k, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM) &&
-            map_mnmajor(c, &tmW_mn, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, BN / 64) &&
+            map_mnmajor(c, &tmW_mn, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_panels(c)) &&
             map_mnmajor(c, &tmG_mn, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM / 64) &&
-            map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BN / 64);
+            map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, b_box_panels(c));
   if (!ok) return RL_ERR_CUDA;
 
   const int n_row_slabs = (L.Tpad + L.Ts - 1) / L.Ts;
@@ -513,6 +581,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         sh.n_tiles = d_tiles;
         sh.n_range = 1;
         sh.b_k_off = vocab_base;
+        sh.n_fastest = 1;   // the CTAs that share a panel of G rows run together
         EpiAcc::Params ep;
         ep.C = dH_acc; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0;
         launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, sh, ep);
@@ -528,6 +597,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         sh.n_range = 1;
         sh.skip_if_k0 = (r > 0 || o.accumulate_dW) ? 1 : 0;
         sh.b_k_off = row_base;
+        sh.n_fastest = 1;
         EpiAcc::Params ep;
         ep.C = dW; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
         ep.row_base = vocab_base;
@@ -617,8 +687,8 @@ rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, in
   CUtensorMap ta, tb;
   bool ok = a_mn ? map_mnmajor(c, &ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)M, BM / 64)
                  : map_kmajor(c, &ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM);
-  ok = ok && (b_mn ? map_mnmajor(c, &tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)N, BN / 64)
-                   : map_kmajor(c, &tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN));
+  ok = ok && (b_mn ? map_mnmajor(c, &tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)N, b_box_panels(c))
+                   : map_kmajor(c, &tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)K, b_box_rows(c)));
   if (!ok) return RL_ERR_CUDA;
   GemmShape sh;
   memset(&sh, 0, sizeof(sh));
@@ -688,6 +758,8 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
     c.ws_bytes = kStaticScratchBytes - kStaticHeaderBytes;
     c.slab_rows = kSlabRowsMax;
     c.slab_cols = kSlabColsMax;
+    c.cta_group = 1;
+    c.grid[1] = c.n_sm;
     slot.ready = true;
   }
   rl_ctx* c = &slot.ctx;
@@ -702,14 +774,15 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
   cudaMemsetAsync(logp, 0, (size_t)T * 4, c->stream);
   if (entropy) cudaMemsetAsync(entropy, 0, (size_t)T * 4, c->stream);
   if (lse) cudaMemsetAsync(lse, 0, (size_t)T * 4, c->stream);
-  int n_tiles = 0;
-  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &n_tiles)) != RL_OK) return s;
+  GemmShape fwd_shape;
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &fwd_shape)) != RL_OK) return s;
   LossParams p;
   memset(&p, 0, sizeof(p));
   p.partials = reinterpret_cast<const float4*>(ws + L.partials);
   p.part_stride = L.Tpad;
-  p.n_tiles = n_tiles;
-  p.n_ctas = c->n_sm;
+  p.fwd_shape = fwd_shape;
+  p.fwd_cg = c->cta_group;
+  p.fwd_workers = c->grid[c->cta_group] / c->cta_group;
   p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
   p.with_loss = 0;
   p.lse_c = reinterpret_cast<float*>(ws + L.lse_c);

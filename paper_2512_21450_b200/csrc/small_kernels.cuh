@@ -139,8 +139,9 @@ struct LossParams {
   // inputs
   const float4* partials;
   int part_stride;
-  int n_tiles;        // 256-wide vocabulary tiles of the forward pass
-  int n_ctas;         // grid of the forward pass (fixes the split)
+  GemmShape fwd_shape;  // shape of the forward pass: together with its grid it fixes the vocabulary split
+  int fwd_cg;           // CTAs per row tile of the forward pass
+  int fwd_workers;      // grid of the forward pass / fwd_cg
   const int* row_map;
   const float* old_logp;   // [T] original rows; NULL in log-prob-only mode
   const float* ref_logp;   // [T] or NULL
@@ -165,10 +166,7 @@ constexpr int kLossThreads = 256;
 
 __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossParams p, DevStatus* st) {
   const int n = st->n_valid;
-  const int m_tiles = (n + BM - 1) / BM;
-  const int split = choose_split(m_tiles, p.n_tiles, p.n_ctas);
-  const int n_range = max((p.n_tiles + split - 1) / max(split, 1), 1);
-  const int n_ranges = (p.n_tiles + n_range - 1) / n_range;
+  const int n_ranges = gemm_extents(p.fwd_shape, n, p.fwd_cg, p.fwd_workers).n_ranges;
   double acc[kLossSums];
 #pragma unroll
   for (int k = 0; k < kLossSums; ++k) acc[k] = 0.0;

@@ -58,8 +58,8 @@ def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5):
                                      w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef,
                                      token_weight=token_weight)
     _assert_status_ok(ctx)
-    # the oracle gets the advantages the GPU loss saw (their own parity is checked above)
-    oo = _oracle_case(w, _np64(adv_tok), token_weight=None if token_weight is None else _np64(token_weight))
+    # the oracle works from its own advantages; nothing it sees comes from the CUDA path
+    oo = _oracle_case(w, o_adv_tok, token_weight=None if token_weight is None else _np64(token_weight))
     m = w.mask.cpu().numpy().astype(bool)
     assert np.abs(_np64(out["logp"]) - oo["logp"]).max() <= TOL_LOGP
     assert np.abs(_np64(out["entropy"]) - oo["entropy"]).max() <= TOL_ENT
@@ -86,10 +86,14 @@ def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5):
 
 
 # ------------------------------------------------------------------------------------------------
-def test_gemm_engine_layouts(ctx):
-    # operand layouts of the tensor-core engine against a library product
+@pytest.mark.parametrize("cta_group", [1, 2])
+def test_gemm_engine_layouts(cta_group):
+    # operand layouts of the tensor-core engine (single CTAs and CTA pairs) against a library product
+    from paper_2512_21450_b200 import Context
+    ctx = Context(0)
+    ctx.set_cta_group(cta_group)
     g = torch.Generator(device="cuda").manual_seed(1)
-    for (M, N, K) in [(128, 256, 64), (256, 512, 200), (384, 768, 2048)]:
+    for (M, N, K) in [(128, 256, 64), (256, 512, 200), (384, 768, 2048), (1280, 256, 72)]:
         A = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
         B = torch.randn(N, K, generator=g, device="cuda").to(torch.bfloat16)
         ref = A.float() @ B.float().T
@@ -102,6 +106,20 @@ def test_gemm_engine_layouts(ctx):
                 C2 = ctx.rl_selftest_gemm(A.T.contiguous() if a_mn else A, B.T.contiguous() if b_mn else B,
                                           M, N, K, a_mn, b_mn, C=C.clone(), accumulate=True)
                 assert (C2 - 2 * ref).abs().max().item() <= 2e-4 * ref.abs().max().item()
+    ctx.close()
+
+
+def test_single_cta_tiles_match_oracle():
+    # the default context runs CTA pairs; the single-CTA tile shape must give the same results
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    c1 = Context(0)
+    try:
+        c1.set_cta_group(1)
+        _check_against_oracle(c1, make_workload(0, L_max=13, V=4100, seed=700))
+        _check_against_oracle(c1, make_workload(1, prompts=1, L_max=40, seed=701))
+    finally:
+        c1.close()
 
 
 @pytest.mark.parametrize("n_groups,G", [(4, 4), (8, 8), (64, 16), (7, 5), (3, 40), (1024, 8)])
