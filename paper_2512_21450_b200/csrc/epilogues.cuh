@@ -10,6 +10,14 @@ namespace rlh {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
+// One MUFU instruction: 2^x, denormal results flushed to zero (arguments here are <= 0 up to
+// rounding, results in [0, 1]); -inf gives 0.
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Forward statistics (policy over the vocabulary, section 2.2): for its row and the vocabulary
 // range of the work unit, keeps the running maximum M, S = sum exp(z-M), A = sum exp(z-M) z and
@@ -42,26 +50,33 @@ struct EpiStats {
     float cmax = -CUDART_INF_F;
     if (nvalid >= 32) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
+      for (int i = 0; i < 32; i += 2) cmax = fmaxf(cmax, fmaxf(v[i], v[i + 1]));
     } else {
 #pragma unroll
       for (int i = 0; i < 32; ++i) cmax = i < nvalid ? fmaxf(cmax, v[i]) : cmax;
     }
     const float newm = fmaxf(st.m, cmax);
-    const float scale = exp2f((st.m - newm) * kLog2e);
+    const float scale = ex2_approx((st.m - newm) * kLog2e);
     const float mL = newm * kLog2e;
     float cs = 0.f, ca = 0.f;
     if (nvalid >= 32) {
+      // two columns per instruction (packed fp32 pairs): e = 2^(z*log2e - M*log2e), S += e, A += e*z
+      const float2 l2 = make_float2(kLog2e, kLog2e), nm2 = make_float2(-mL, -mL);
+      float2 cs2 = make_float2(0.f, 0.f), ca2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float e = exp2f(fmaf(v[i], kLog2e, -mL));
-        cs += e;
-        ca = fmaf(e, v[i], ca);
+      for (int i = 0; i < 32; i += 2) {
+        const float2 z2 = make_float2(v[i], v[i + 1]);
+        const float2 t2 = __ffma2_rn(z2, l2, nm2);
+        const float2 e2 = make_float2(ex2_approx(t2.x), ex2_approx(t2.y));
+        cs2 = __fadd2_rn(cs2, e2);
+        ca2 = __ffma2_rn(e2, z2, ca2);
       }
+      cs = cs2.x + cs2.y;
+      ca = ca2.x + ca2.y;
     } else {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        const float e = i < nvalid ? exp2f(fmaf(v[i], kLog2e, -mL)) : 0.f;
+        const float e = i < nvalid ? ex2_approx(fmaf(v[i], kLog2e, -mL)) : 0.f;
         cs += e;
         ca = fmaf(e, v[i], ca);
       }
@@ -132,13 +147,21 @@ struct EpiGrad {
       for (int i = 0; i < 32; ++i) g[i] = 0.f;
     } else {
       if (st.ce == 0.f) {
+        // packed fp32 pairs: p = 2^(z*log2e - lse*log2e), g = cp * p
+        const float2 l2 = make_float2(kLog2e, kLog2e), nl2 = make_float2(-st.lse * kLog2e, -st.lse * kLog2e);
+        const float2 cp2 = make_float2(st.cp, st.cp);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) g[i] = st.cp * exp2f((v[i] - st.lse) * kLog2e);
+        for (int i = 0; i < 32; i += 2) {
+          const float2 t2 = __ffma2_rn(make_float2(v[i], v[i + 1]), l2, nl2);
+          const float2 g2 = __fmul2_rn(make_float2(ex2_approx(t2.x), ex2_approx(t2.y)), cp2);
+          g[i] = g2.x;
+          g[i + 1] = g2.y;
+        }
       } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const float lp = v[i] - st.lse;
-          g[i] = exp2f(lp * kLog2e) * fmaf(st.ce, lp + st.ent, st.cp);
+          g[i] = ex2_approx(lp * kLog2e) * fmaf(st.ce, lp + st.ent, st.cp);
         }
       }
       const unsigned rel = (unsigned)(st.y - col_g);

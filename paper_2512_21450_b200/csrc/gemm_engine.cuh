@@ -11,7 +11,7 @@
 //
 // CG = 1: one CTA per 128x256 output tile (4 stages of 16 KB A + 32 KB B).
 // CG = 2: a cluster of two CTAs (one SM pair) per 256x256 output tile.  Each CTA stages its own
-//         128 rows of A and 128 of the 256 columns of B (6 stages of 16 KB + 16 KB), the even
+//         128 rows of A and 128 of the 256 columns of B (7 stages of 16 KB + 16 KB), the even
 //         CTA issues tcgen05.mma.cta_group::2 (M = 256) which reads both halves of B and writes
 //         128 accumulator rows into each CTA's tensor memory; both CTAs run their own epilogue.
 //         All TMA completions of a stage are counted on the even CTA's barrier; stage-free and
@@ -38,7 +38,8 @@ constexpr int BN = 256;   // accumulator columns
 constexpr int BK = 64;
 constexpr int kAStageBytes = BM * BK * 2;
 constexpr int kGemmThreads = 192;
-constexpr int kGemmSmemBytes = 192 * 1024 + 1024;  // ring + slack for 1024-byte alignment
+constexpr int kRingBytes = 224 * 1024;             // shared-memory ring of operand stages
+constexpr int kGemmSmemBytes = kRingBytes + 1024;  // + slack for 1024-byte alignment
 constexpr int kTmemCols = 512;
 constexpr int kMaxSplit = 16;
 
@@ -47,10 +48,10 @@ struct StageCfg {
   static constexpr int kBRows = BN / CG;                    // B rows (output columns) staged per CTA
   static constexpr int kBBytes = kBRows * BK * 2;
   static constexpr int kStageBytes = kAStageBytes + kBBytes;
-  static constexpr int kStages = (192 * 1024) / kStageBytes;  // 4 (CG = 1) or 6 (CG = 2)
+  static constexpr int kStages = kRingBytes / kStageBytes;  // 4 (CG = 1) or 7 (CG = 2)
   static constexpr uint32_t kTxBytes = uint32_t(kStageBytes) * CG;  // bytes counted on the issuing CTA's barrier
 };
-constexpr int kMaxStages = 6;
+constexpr int kMaxStages = 7;
 
 // Device status word shared by all kernels of a context.
 struct DevStatus {

@@ -44,7 +44,7 @@ struct rl_ctx {
 namespace {
 
 constexpr int kSlabRowsMax = 32768;        // rows of one gradient slab
-constexpr int kSlabColsMax = 74 * 128;     // vocabulary columns of one gradient slab (37 tiles of 256)
+constexpr int kSlabColsMax = 148 * 128;    // vocabulary columns of one gradient slab (74 tiles of 256)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
