@@ -293,6 +293,25 @@ def main():
         "traffic": traffic, "flops_per_launch": flops_pass / max(kind_n[dom], 1),
         "avg_launch_ms": kind_ms[dom] / max(kind_n[dom], 1), "kernels": kinds,
     }
+    # HBM-bound helpers: algorithmic bytes per step against their event time
+    N, Npad = w.n_valid, (w.n_valid + 127) // 128 * 128
+    n_tiles = (w.V + 255) // 256
+    m_units, workers = (N + 255) // 256, 74
+    split = min(range(1, min(16, n_tiles) + 1),
+                key=lambda sp: (-(-m_units * sp // workers) * -(-n_tiles // sp), sp))
+    small_bytes = {
+        4: ("mask scan (3 launches)", w.T + 4 * N),
+        5: ("row gather", 2 * N * w.d + 2 * Npad * w.d + 12 * N),
+        6: ("merge + per-token loss", N * (16 * split + 32)),
+        7: ("dH scatter", 6 * N * w.d + 4 * N),
+        8: ("GRPO advantages + broadcast", 12 * w.n_seq + 4 * w.T),
+    }
+    small = []
+    for k, (name, nbytes) in small_bytes.items():
+        if kind_n[k]:
+            t_ms = kind_ms[k] / args.steps
+            small.append(dict(kernel=name, ms_per_step=t_ms, bytes_per_step=nbytes,
+                              gbs=nbytes / (t_ms / 1e3) / 1e9, frac_of_hbm_peak=nbytes / (t_ms / 1e3) / 1e9 / peaks["hbm"]))
     exec_tflops = 8.0 * w.d * w.V * n_tok * args.steps / (ms / 1e3) / 1e12
     out = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -308,6 +327,7 @@ def main():
                              "useful_6dV_of_burst": 75 * exec_tflops / world / peaks["burst"],
                              "executed_tflops_per_gpu": exec_tflops / world, "peaks": peaks["source"]},
         "clocks": clocks, "gpu_launches": launches, "roofline": roofline,
+        "small_kernels": {"bound": "hbm", "peak_gbs": peaks["hbm"], "kernels": small},
     }
     if e2e_val is not None:
         out["e2e"] = {"value": e2e_val, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 64,

@@ -190,11 +190,12 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
                                    float* logp, float* entropy, float* lse, int32_t* dev_status);
 
 /* Instrumentation.  rl_launch_count: kernels this context has launched so far.
- * rl_set_profiling(on): when on, every tensor-core launch is bracketed by a pair of CUDA events
+ * rl_set_profiling(on): when on, every kernel (or group of small kernels) is bracketed by a pair of CUDA events
  * on the context's stream (at most 2048 launches are kept between two reads).
  * rl_profile_read: synchronises the stream and returns, per kernel kind (0 forward statistics,
- * 1 gradient-of-logits slab, 2 dH, 3 dW), the summed device time in milliseconds ms[4] (host)
- * and the number of launches launches[4] (host) since the previous read.  The paper has no
+ * 1 gradient-of-logits slab, 2 dH, 3 dW, 4 mask scan, 5 row gather, 6 merge + per-token loss,
+ * 7 dH scatter, 8 advantages), the summed device time in milliseconds ms[9] (host) and the number
+ * of timed launch groups launches[9] (host) since the previous read.  The paper has no
  * counterpart; these exist so that a benchmark can report per-kernel roofline figures. */
 rl_status rl_launch_count(rl_ctx* ctx, int64_t* n);
 rl_status rl_set_profiling(rl_ctx* ctx, int on);

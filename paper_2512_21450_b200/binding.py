@@ -232,8 +232,8 @@ class Context:
         _check(self.lib.rl_set_profiling(self.handle, int(on)), "rl_set_profiling")
 
     def profile_read(self):
-        ms = (ctypes.c_double * 4)()
-        n = (c_int64 * 4)()
+        ms = (ctypes.c_double * 9)()
+        n = (c_int64 * 9)()
         _check(self.lib.rl_profile_read(self.handle, ms, n), "rl_profile_read")
         return list(ms), list(n)
 

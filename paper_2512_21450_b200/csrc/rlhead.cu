@@ -19,7 +19,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kProfMax = 2048;   // timed launches kept between two rl_profile_read calls
-constexpr int kProfKinds = 4;    // 0 forward statistics, 1 dlogits, 2 dH, 3 dW
+constexpr int kProfKinds = 9;    // 0 forward statistics, 1 dlogits, 2 dH, 3 dW, 4 mask scan, 5 row gather,
+                                 // 6 merge + loss, 7 dH scatter, 8 advantages
 
 struct rl_ctx {
   int device;
@@ -50,7 +51,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
   int Tpad, Ts, Vs;
-  size_t row_map, tokens_c, lse_c, ent_c, cp_c, ce_c, partials, block_sums, Hc, G, dH_acc, staging, total;
+  size_t scan_counts, row_map, tokens_c, lse_c, ent_c, cp_c, ce_c, partials, block_sums, Hc, G, dH_acc, staging, total;
 };
 
 // staging_T > 0 adds room for host-call inputs (H, tokens, old, ref, adv, mask).
@@ -62,6 +63,7 @@ WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_s
   L.Vs = Vpad < c->slab_cols ? Vpad : c->slab_cols;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 1024); return at; };
+  L.scan_counts = take(((size_t)L.Tpad / 4096 + 2) * 4);
   L.row_map = take((size_t)L.Tpad * 4);
   L.tokens_c = take((size_t)L.Tpad * 4);
   L.lse_c = take((size_t)L.Tpad * 4);
@@ -128,15 +130,26 @@ cudaError_t set_smem_attr() {
 inline uint32_t b_box_rows(const rl_ctx* c) { return BN / c->cta_group; }
 inline uint32_t b_box_panels(const rl_ctx* c) { return BN / 64 / c->cta_group; }
 
+// Optional timing of a group of launches: event pair on the context's stream, tagged with a kind.
+int prof_begin(rl_ctx* c, int kind) {
+  if (!(c->prof_on && kind >= 0 && kind < kProfKinds && c->prof_used < kProfMax)) return -1;
+  const int i = c->prof_used;
+  for (int e = 0; e < 2; ++e)
+    if (!c->prof_ev[i][e]) cudaEventCreate(&c->prof_ev[i][e]);
+  cudaEventRecord(c->prof_ev[i][0], c->stream);
+  return i;
+}
+void prof_end(rl_ctx* c, int i, int kind) {
+  if (i < 0) return;
+  cudaEventRecord(c->prof_ev[i][1], c->stream);
+  c->prof_kind[i] = kind;
+  c->prof_used = i + 1;
+}
+
 template <class Epi, int A_MN, int B_MN>
 void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const GemmShape& sh,
                  const typename Epi::Params& ep) {
-  const bool timed = c->prof_on && kind >= 0 && kind < kProfKinds && c->prof_used < kProfMax;
-  if (timed) {
-    for (int e = 0; e < 2; ++e)
-      if (!c->prof_ev[c->prof_used][e]) cudaEventCreate(&c->prof_ev[c->prof_used][e]);
-    cudaEventRecord(c->prof_ev[c->prof_used][0], c->stream);
-  }
+  const int prof = prof_begin(c, kind);
   if (c->cta_group == 2) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -157,10 +170,7 @@ void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b
                                                                                             c->dstatus);
   }
   c->launches++;
-  if (timed) {
-    cudaEventRecord(c->prof_ev[c->prof_used][1], c->stream);
-    c->prof_kind[c->prof_used++] = kind;
-  }
+  prof_end(c, prof, kind);
 }
 
 rl_status check_hw(const void* H, int64_t ldH, const void* W, int64_t ldW, int64_t T, int64_t d, int64_t V) {
@@ -189,10 +199,20 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   int* row_map = reinterpret_cast<int*>(ws + L.row_map);
   int* tokens_c = reinterpret_cast<int*>(ws + L.tokens_c);
   __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + L.Hc);
-  mask_scan_kernel<<<1, kScanThreads, 0, c->stream>>>(mask, (int)T, row_map, c->dstatus);
+  {
+    const int pr = prof_begin(c, 4);
+    int* block_counts = reinterpret_cast<int*>(ws + L.scan_counts);
+    const int n_blocks = (int)((T + kScanRowsPerBlock - 1) / kScanRowsPerBlock);
+    mask_count_kernel<<<n_blocks, kScanThreads, 0, c->stream>>>(mask, (int)T, block_counts);
+    mask_offsets_kernel<<<1, 1024, 0, c->stream>>>(block_counts, n_blocks, c->dstatus);
+    mask_write_kernel<<<n_blocks, kScanThreads, 0, c->stream>>>(mask, (int)T, block_counts, row_map);
+    prof_end(c, pr, 4);
+  }
+  const int pr_gather = prof_begin(c, 5);
   gather_rows_kernel<<<c->n_sm * 4, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16*>(H), ldH, (int)d, row_map,
                                                          tokens, (int)V, Hc, tokens_c, c->dstatus);
-  c->launches += 2;
+  prof_end(c, pr_gather, 5);
+  c->launches += 4;
   CUtensorMap tmA, tmB;
   if (!map_kmajor(c, &tmA, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM)) return RL_ERR_CUDA;
   if (!map_kmajor(c, &tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_rows(c))) return RL_ERR_CUDA;
@@ -405,6 +425,7 @@ rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, 
   if (n_seq == 0) return RL_OK;
   const int n_groups = (int)(n_seq / group_size);
   const int warps = 8;
+  const int pr_adv = prof_begin(c, 8);
   grpo_adv_kernel<<<(n_groups + warps - 1) / warps, warps * 32, 0, c->stream>>>(rewards, n_groups, group_size, ddof,
                                                                                 eps_std, adv_seq);
   c->launches++;
@@ -414,6 +435,7 @@ rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, 
     broadcast_adv_kernel<<<blocks, 256, 0, c->stream>>>(adv_seq, seq_offsets, (int)n_seq, adv_tok);
     c->launches++;
   }
+  prof_end(c, pr_adv, 8);
   return cuda_ok();
 }
 
@@ -525,8 +547,10 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   p.block_sums = reinterpret_cast<double*>(ws + L.block_sums);
   int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
   if (blocks > 1024) blocks = 1024;
+  const int pr_loss = prof_begin(c, 6);
   combine_loss_kernel<<<blocks, kLossThreads, 0, st>>>(p, c->dstatus);
   finalize_loss_kernel<<<1, 32, 0, st>>>(p.block_sums, blocks, loss, o.metrics_out, c->dstatus);
+  prof_end(c, pr_loss, 6);
   c->launches += 2;
 
   // ---- backward, one (row slab x vocabulary slab) at a time
@@ -604,8 +628,10 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, sh, ep);
       }
     }
+    const int pr_sc = prof_begin(c, 7);
     scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
                                                    static_cast<__nv_bfloat16*>(dH), c->dstatus);
+    prof_end(c, pr_sc, 7);
     c->launches++;
   }
   return cuda_ok();

@@ -9,49 +9,102 @@
 namespace rlh {
 
 // ------------------------------------------------------------------------------------------
-// Mask scan: row_map[i] = index of the i-th row with mask != 0 (ascending), n_valid = their
-// number.  One block; each thread scans a contiguous piece.
-constexpr int kScanThreads = 1024;
-__global__ void __launch_bounds__(kScanThreads) mask_scan_kernel(const uint8_t* __restrict__ mask, int T,
-                                                                 int* __restrict__ row_map, DevStatus* st) {
-  __shared__ int warp_sums[32];
-  __shared__ int total;
-  const int tid = threadIdx.x;
-  const int per = (T + kScanThreads - 1) / kScanThreads;
-  const int begin = min(tid * per, T), end = min(begin + per, T);
-  int cnt = 0;
-  if (mask) {
-    for (int i = begin; i < end; ++i) cnt += mask[i] != 0;
+// Mask scan in three launches: row_map[i] = index of the i-th row with mask != 0 (ascending),
+// n_valid = their number.  Each block owns 4096 consecutive rows, each thread 16 of them (one
+// 16-byte load when the mask is 16-byte aligned): (1) per-block counts, (2) one block turns the
+// counts into exclusive offsets, (3) every block scans its rows again and writes its indices.
+constexpr int kScanThreads = 256;
+constexpr int kScanRowsPerThread = 16;
+constexpr int kScanRowsPerBlock = kScanThreads * kScanRowsPerThread;
+
+// Bit i of the result = (mask[base + i] != 0), rows past T read as 0; mask == NULL means all valid.
+__device__ __forceinline__ unsigned scan_load_bits(const uint8_t* __restrict__ mask, long long base, int T) {
+  if (base >= T) return 0u;
+  const int n = (int)min((long long)kScanRowsPerThread, (long long)T - base);
+  if (!mask) return n == 16 ? 0xFFFFu : ((1u << n) - 1u);
+  unsigned bits = 0;
+  if (n == 16 && ((reinterpret_cast<uintptr_t>(mask + base) & 15) == 0)) {
+    const uint4 q = __ldg(reinterpret_cast<const uint4*>(mask + base));
+    const unsigned wds[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int w = 0; w < 4; ++w)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) bits |= ((wds[w] >> (8 * b)) & 0xFFu) ? (1u << (4 * w + b)) : 0u;
   } else {
-    cnt = end - begin;
+    for (int i = 0; i < n; ++i) bits |= __ldg(mask + base + i) ? (1u << i) : 0u;
   }
-  // block exclusive scan of cnt
-  int incl = cnt;
-  const int lane = tid & 31, warp = tid >> 5;
+  return bits;
+}
+
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    int v = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += v;
+    const int u = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += u;
   }
   if (lane == 31) warp_sums[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    int w = warp_sums[lane];
+    const int w = lane < (int)(blockDim.x >> 5) ? warp_sums[lane] : 0;
     int wi = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      int v = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += v;
+      const int u = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += u;
     }
     warp_sums[lane] = wi - w;
-    if (lane == 31) total = wi;
+    if (lane == 31 && total) *total = wi;
   }
   __syncthreads();
-  int pos = warp_sums[warp] + incl - cnt;
-  for (int i = begin; i < end; ++i) {
-    if (!mask || mask[i] != 0) row_map[pos++] = i;
+  return warp_sums[warp] + incl - v;
+}
+
+__global__ void __launch_bounds__(kScanThreads) mask_count_kernel(const uint8_t* __restrict__ mask, int T,
+                                                                  int* __restrict__ block_counts) {
+  __shared__ int warp_sums[32];
+  const long long base = ((long long)blockIdx.x * kScanThreads + threadIdx.x) * kScanRowsPerThread;
+  int c = __popc(scan_load_bits(mask, base, T));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = c;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int t = 0;
+    for (int w = 0; w < kScanThreads / 32; ++w) t += warp_sums[w];
+    block_counts[blockIdx.x] = t;
   }
-  if (tid == 0) st->n_valid = total;
+}
+
+// One block: block_counts[0..n) -> exclusive offsets in place, total -> st->n_valid.
+__global__ void __launch_bounds__(1024) mask_offsets_kernel(int* __restrict__ block_counts, int n, DevStatus* st) {
+  __shared__ int warp_sums[32];
+  __shared__ int chunk_total;
+  int carry = 0;
+  for (int base = 0; base < n; base += 1024) {
+    const int i = base + threadIdx.x;
+    const int v = i < n ? block_counts[i] : 0;
+    const int ex = block_exclusive_scan(v, warp_sums, &chunk_total);
+    if (i < n) block_counts[i] = carry + ex;
+    carry += chunk_total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) st->n_valid = carry;
+}
+
+__global__ void __launch_bounds__(kScanThreads) mask_write_kernel(const uint8_t* __restrict__ mask, int T,
+                                                                  const int* __restrict__ block_offsets,
+                                                                  int* __restrict__ row_map) {
+  __shared__ int warp_sums[32];
+  const long long base = ((long long)blockIdx.x * kScanThreads + threadIdx.x) * kScanRowsPerThread;
+  unsigned bits = scan_load_bits(mask, base, T);
+  int pos = block_offsets[blockIdx.x] + block_exclusive_scan(__popc(bits), warp_sums, nullptr);
+  while (bits) {
+    const int i = __ffs(bits) - 1;
+    bits &= bits - 1;
+    row_map[pos++] = (int)base + i;
+  }
 }
 
 // ------------------------------------------------------------------------------------------
