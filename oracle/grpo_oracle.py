@@ -67,6 +67,55 @@ def grpo_advantages(rewards, group_size, ddof=1, eps_std=1e-6):
     return adv
 
 
+# --------------------------------------------------------------------------- #
+# Other critic-free estimators the paper names in section 4.2 without printing a
+# formula ("RLOO's leave-one-out baselines", "OPO's length-weighted baselines",
+# REINFORCE++).  Readings, stated here because the paper is silent:
+#   RLOO          A_i = r_i - mean of the OTHER responses of the group
+#   OPO           A_i = r_i - sum_j(len_j r_j) / sum_j(len_j) over the group
+#   REINFORCE++   A_i = (c_i - mean(c)) / (std(c) + eps_std) over the whole batch,
+#                 c_i = r_i - mean of its group (population std)
+# Parity unpinned with respect to the authors' code; pinned to these readings.
+# --------------------------------------------------------------------------- #
+def rloo_advantages(rewards, group_size):
+    r = np.asarray(rewards, dtype=np.float64)
+    B = r.shape[0]
+    if group_size < 2 or B % group_size != 0:
+        raise ValueError("group_size must be >= 2 and divide the number of responses")
+    adv = np.zeros(B)
+    for g in range(B // group_size):
+        for i in range(group_size):
+            others = [r[g * group_size + j] for j in range(group_size) if j != i]
+            adv[g * group_size + i] = r[g * group_size + i] - sum(others) / (group_size - 1)
+    return adv
+
+
+def opo_advantages(rewards, lengths, group_size):
+    r = np.asarray(rewards, dtype=np.float64)
+    ln = np.asarray(lengths, dtype=np.float64)
+    B = r.shape[0]
+    if group_size < 1 or B % group_size != 0:
+        raise ValueError("group_size must divide the number of responses")
+    adv = np.zeros(B)
+    for g in range(B // group_size):
+        sl = slice(g * group_size, (g + 1) * group_size)
+        tot = ln[sl].sum()
+        base = (ln[sl] * r[sl]).sum() / tot if tot > 0 else 0.0
+        adv[sl] = r[sl] - base
+    return adv
+
+
+def reinforce_pp_advantages(rewards, group_size, eps_std=1e-6):
+    r = np.asarray(rewards, dtype=np.float64)
+    B = r.shape[0]
+    if group_size < 1 or B % group_size != 0:
+        raise ValueError("group_size must divide the number of responses")
+    c = r - np.repeat(r.reshape(-1, group_size).mean(axis=1), group_size)
+    mu = c.sum() / B
+    sigma = np.sqrt(((c - mu) ** 2).sum() / B)
+    return (c - mu) / (sigma + eps_std)
+
+
 def broadcast_to_tokens(adv_seq, seq_offsets, T):
     """Outcome supervision: every token of response i carries A_i
     (Algorithm 1: one advantage per time step from one reward per trajectory)."""

@@ -155,6 +155,33 @@ def test_advantages_zero_variance_affine_permutation():
         O.grpo_advantages(r, 5)
 
 
+def test_other_estimators_closed_forms():
+    rng = _rng(21)
+    G = 5
+    r = rng.normal(size=3 * G)
+    # RLOO: leaving one out of the mean equals scaling the centred reward by G/(G-1)
+    a = O.rloo_advantages(r, G)
+    mu = np.repeat(r.reshape(-1, G).mean(axis=1), G)
+    assert np.allclose(a, (r - mu) * G / (G - 1), atol=1e-13)
+    assert np.allclose(a.reshape(-1, G).sum(axis=1), 0.0, atol=1e-13)
+    assert np.allclose(O.rloo_advantages(np.array([1.0, 0.0]), 2), [1.0, -1.0])
+    # OPO: with equal lengths the length-weighted baseline is the plain mean; one long response pulls it
+    assert np.allclose(O.opo_advantages(r, np.full(3 * G, 7), G), r - mu, atol=1e-13)
+    o = O.opo_advantages(np.array([1.0, 0.0, 0.0, 0.0]), np.array([30, 10, 10, 10]), 4)
+    assert np.allclose(o, np.array([1.0, 0, 0, 0]) - 0.5, atol=1e-15)
+    # the length-weighted sum of OPO advantages vanishes in every group
+    ln = rng.integers(1, 50, size=3 * G)
+    o = O.opo_advantages(r, ln, G)
+    assert np.allclose((o * ln).reshape(-1, G).sum(axis=1), 0.0, atol=1e-12)
+    # REINFORCE++: zero mean, unit (population) std over the batch; invariant to per-group shifts
+    p = O.reinforce_pp_advantages(r, G, eps_std=0.0)
+    assert abs(p.mean()) < 1e-13 and abs(p.std() - 1.0) < 1e-13
+    shifted = r + np.repeat(np.array([3.0, -2.0, 10.0]), G)
+    assert np.allclose(O.reinforce_pp_advantages(shifted, G, eps_std=0.0), p, atol=1e-12)
+    with pytest.raises(ValueError):
+        O.rloo_advantages(r, 1)
+
+
 def test_broadcast_to_tokens():
     offs = np.array([0, 3, 3, 7])
     adv = O.broadcast_to_tokens(np.array([1.0, 2.0, -1.0]), offs, 9)
