@@ -97,6 +97,20 @@ rl_status rl_grpo_advantages_ex(rl_ctx* ctx, const float* rewards, int64_t n_seq
                                 int ddof, float eps_std, const int32_t* seq_offsets,
                                 int64_t T, float* adv_seq, float* adv_tok);
 
+/* The other critic-free advantage estimators that section 4.2 names ("RLOO's leave-one-out
+ * baselines", "OPO's length-weighted baselines", REINFORCE++) on the same grouped layout.  The
+ * paper prints no formula for them; the readings are
+ *   RL_ADV_GRPO          as rl_grpo_advantages (sample std, eps_std as given)
+ *   RL_ADV_RLOO          A_i = r_i - mean of the other responses of the group (group_size >= 2)
+ *   RL_ADV_OPO           A_i = r_i - sum_j(len_j r_j) / sum_j(len_j) over the group; lengths[n_seq]
+ *                        (int32, valid tokens per response) required
+ *   RL_ADV_REINFORCE_PP  c_i = r_i - group mean, then A_i = (c_i - mean(c)) / (std(c) + eps_std) over
+ *                        the whole batch (population std, fp64 fixed-order reduction)
+ * Errors as rl_grpo_advantages_ex. */
+typedef enum { RL_ADV_GRPO = 0, RL_ADV_RLOO = 1, RL_ADV_OPO = 2, RL_ADV_REINFORCE_PP = 3 } rl_adv_estimator;
+rl_status rl_advantages(rl_ctx* ctx, int estimator, const float* rewards, const int32_t* lengths,
+                        int64_t n_seq, int group_size, float eps_std, float* adv_seq);
+
 /* Per-token log-probability of the sampled token, entropy and log-sum-exp of the next-token
  * distribution softmax(W h_t) - section 2.2 (policy over the vocabulary; importance ratio
  * numerator) and section 2.2 "Regularization" (entropy).  Natural logarithms.

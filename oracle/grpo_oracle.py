@@ -183,6 +183,54 @@ def token_weights(mask):
     return m / n if n > 0 else np.zeros_like(m)
 
 
+def aggregation_weights(mask, seq_offsets, mode):
+    """Token weights w_t of the loss ("length normalization with token weights", section 2.2).
+
+    mode 0: token mean over the call, w_t = m_t / sum(m).
+    mode 1: mean over sequences of each sequence's token mean, w_t = m_t / (B * len_i).
+    mode 2: mean over sequences of the token sum divided by the longest row range,
+            w_t = m_t / (B * L_max).
+    B = number of sequences, len_i = valid tokens of sequence i, L_max = max_i(off[i+1] - off[i]).
+    """
+    m = np.asarray(mask).astype(np.float64)
+    if mode == 0:
+        return token_weights(m)
+    off = np.asarray(seq_offsets)
+    B = len(off) - 1
+    w = np.zeros_like(m)
+    L_max = max(int(off[i + 1] - off[i]) for i in range(B)) if B else 0
+    for i in range(B):
+        sl = slice(off[i], off[i + 1])
+        n = m[sl].sum()
+        if mode == 1:
+            if n > 0:
+                w[sl] = m[sl] / (B * n)
+        elif mode == 2:
+            if L_max > 0:
+                w[sl] = m[sl] / (B * L_max)
+        else:
+            raise ValueError("unknown aggregation mode")
+    return w
+
+
+def sequence_ratio(logp, old_logp, mask, seq_offsets):
+    """Sequence-level importance ratio ("GSPO's sequence-level aggregation", section 4.2; the
+    paper prints no formula - reading): rho_i = exp(mean over the valid tokens of sequence i of
+    (logp_t - old_logp_t)), i.e. the geometric mean of the token ratios; every token of the
+    sequence uses rho_i.  Returns (rho per row, len per row); rows outside any sequence get 1, 0."""
+    T = len(logp)
+    m = np.asarray(mask).astype(bool)
+    rho = np.ones(T)
+    ln = np.zeros(T)
+    off = np.asarray(seq_offsets)
+    for i in range(len(off) - 1):
+        idx = np.arange(off[i], off[i + 1])[m[off[i]:off[i + 1]]]
+        if idx.size:
+            rho[idx] = np.exp((logp[idx] - old_logp[idx]).sum() / idx.size)
+            ln[idx] = idx.size
+    return rho, ln
+
+
 def per_token_terms(logp, old_logp, ref_logp, adv, eps_low, eps_high, beta,
                     literal_clip=False):
     """Per-token surrogate s_t, k3_t, ratio rho_t and d(loss_t)/d(logp_t) (unweighted).
@@ -215,7 +263,8 @@ def per_token_terms(logp, old_logp, ref_logp, adv, eps_low, eps_high, beta,
 
 def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
                         eps_low, eps_high, beta, ent_coef=0.0,
-                        token_weight=None, literal_clip=False):
+                        token_weight=None, literal_clip=False,
+                        seq_offsets=None, agg_mode=0, sequence_level=False):
     """Loss of Eq. 6 (negated) and its gradients with respect to H and W.
 
     Returns a dict with loss, dH[T,d], dW[V,d], logp, entropy, lse, G (the
@@ -228,7 +277,10 @@ def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
     T, d = H.shape
     V = W.shape[0]
     m = np.asarray(mask).astype(bool)
-    w = token_weights(m) if token_weight is None else np.asarray(token_weight, dtype=np.float64) * m
+    if token_weight is not None:
+        w = np.asarray(token_weight, dtype=np.float64) * m
+    else:
+        w = aggregation_weights(m, seq_offsets, agg_mode)
     old_logp = np.asarray(old_logp, dtype=np.float64)
     adv = np.asarray(adv, dtype=np.float64)
     ref = np.zeros(T) if ref_logp is None else np.asarray(ref_logp, dtype=np.float64)
@@ -248,9 +300,36 @@ def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
     P = np.exp(LP)
     logp = LP[np.arange(rows.size), y]
 
-    s, k3, rho, active, dlogp = per_token_terms(
-        logp, old_logp[rows], ref[rows], adv[rows], eps_low, eps_high, beta, literal_clip)
     wr = w[rows]
+    if not sequence_level:
+        s, k3, rho, active, dlogp = per_token_terms(
+            logp, old_logp[rows], ref[rows], adv[rows], eps_low, eps_high, beta, literal_clip)
+        wdlogp = wr * dlogp                       # weighted d loss / d logp_t
+    else:
+        # sequence-level ratio: the surrogate of every token uses rho_i of its sequence
+        logp_full = np.zeros(T)
+        logp_full[rows] = logp
+        rho_full, len_full = sequence_ratio(logp_full, old_logp, m, seq_offsets)
+        rho = rho_full[rows]
+        a = adv[rows]
+        clipped = np.clip(rho, 1.0 - eps_low, 1.0 + eps_high)
+        s = np.minimum(rho * a, clipped * a)
+        active = (rho * a <= clipped * a)
+        # d rho_i / d logp_u = rho_i / len_i for every valid token u of sequence i, hence
+        # d loss / d logp_u = -(rho_i / len_i) * sum over the sequence of w_t A_t active_t
+        contrib = np.zeros(T)
+        contrib[rows] = wr * a * active
+        off = np.asarray(seq_offsets)
+        seq_sum = np.zeros(T)
+        for i in range(len(off) - 1):
+            seq_sum[off[i]:off[i + 1]] = contrib[off[i]:off[i + 1]].sum()
+        wdlogp = -(rho / np.maximum(len_full[rows], 1.0)) * seq_sum[rows]
+        if beta != 0.0:
+            delta = ref[rows] - logp
+            k3 = np.exp(delta) - delta - 1.0
+            wdlogp = wdlogp + wr * beta * (1.0 - np.exp(delta))
+        else:
+            k3 = np.zeros_like(logp)
     loss_t = -s + beta * k3 - ent_coef * ent
     loss = float((wr * loss_t).sum())
 
@@ -259,7 +338,7 @@ def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
     #   d Ent_t  / d z_tj = -p_tj * (log p_tj + Ent_t)
     onehot = np.zeros_like(P)
     onehot[np.arange(rows.size), y] = 1.0
-    G = (wr * dlogp)[:, None] * (onehot - P)
+    G = wdlogp[:, None] * (onehot - P)
     if ent_coef != 0.0:
         G += (wr * ent_coef)[:, None] * P * (LP + ent[:, None])
 

@@ -66,6 +66,8 @@ def load_library():
     lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
     lib.rl_grpo_advantages.argtypes = [P, P, c_int64, c_int, P]
     lib.rl_grpo_advantages_ex.argtypes = [P, P, c_int64, c_int, c_int, c_float, P, c_int64, P, P]
+    lib.rl_advantages.argtypes = [P, c_int, P, P, c_int64, c_int, c_float, P]
+    lib.rl_advantages.restype = c_int
     lib.rl_token_logprobs.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P]
     loss_args = [P, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int64, c_int64,
                  c_float, c_float, c_float, P, P, P]
@@ -170,6 +172,17 @@ class Context:
                                               _ptr(seq_offsets), T, _ptr(adv_seq), _ptr(adv_tok)),
                "rl_grpo_advantages_ex")
         return adv_seq, adv_tok
+
+    ESTIMATORS = {"grpo": 0, "rloo": 1, "opo": 2, "reinforce_pp": 3}
+
+    def rl_advantages(self, estimator, rewards, group_size, lengths=None, eps_std=1e-6):
+        self._bind_stream()
+        assert rewards.dtype == torch.float32 and rewards.is_cuda and rewards.is_contiguous()
+        assert lengths is None or lengths.dtype == torch.int32
+        adv_seq = torch.empty_like(rewards)
+        _check(self.lib.rl_advantages(self.handle, self.ESTIMATORS[estimator], _ptr(rewards), _ptr(lengths),
+                                      rewards.numel(), group_size, eps_std, _ptr(adv_seq)), "rl_advantages")
+        return adv_seq
 
     def rl_token_logprobs(self, H, W, tokens, mask=None):
         self._bind_stream()

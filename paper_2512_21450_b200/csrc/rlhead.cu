@@ -285,8 +285,9 @@ rl_status rl_create(rl_ctx** out, int device) {
     return RL_ERR_CUDA;
   }
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(&c->dstatus, sizeof(DevStatus)) != cudaSuccess) { delete c; return RL_ERR_CUDA; }
-  cudaMemset(c->dstatus, 0, sizeof(DevStatus));
+  // device block: status word, then two doubles for batch statistics
+  if (cudaMalloc(&c->dstatus, 256) != cudaSuccess) { delete c; return RL_ERR_CUDA; }
+  cudaMemset(c->dstatus, 0, 256);
   bool ok = set_smem_attr<EpiStats, 0, 0>() == cudaSuccess && set_smem_attr<EpiGrad, 0, 0>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 0, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 0, 1>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess;
@@ -436,6 +437,34 @@ rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, 
     c->launches++;
   }
   prof_end(c, pr_adv, 8);
+  return cuda_ok();
+}
+
+rl_status rl_advantages(rl_ctx* c, int estimator, const float* rewards, const int32_t* lengths, int64_t n_seq,
+                        int group_size, float eps_std, float* adv_seq) {
+  if (!c || n_seq < 0 || (n_seq > 0 && (!rewards || !adv_seq))) return RL_ERR_INVALID_ARG;
+  if (estimator < RL_ADV_GRPO || estimator > RL_ADV_REINFORCE_PP || !(eps_std >= 0.f)) return RL_ERR_INVALID_ARG;
+  if (estimator == RL_ADV_OPO && n_seq > 0 && !lengths) return RL_ERR_INVALID_ARG;
+  if (estimator == RL_ADV_GRPO)
+    return rl_grpo_advantages_ex(c, rewards, n_seq, group_size, 1, eps_std, nullptr, 0, adv_seq, nullptr);
+  const int min_group = estimator == RL_ADV_RLOO ? 2 : 1;
+  if (group_size < min_group || n_seq % group_size != 0 || n_seq >= (int64_t(1) << 31)) return RL_ERR_SHAPE;
+  if (n_seq == 0) return RL_OK;
+  const int n_groups = (int)(n_seq / group_size);
+  const int warps = 8;
+  const int pr = prof_begin(c, 8);
+  group_baseline_kernel<<<(n_groups + warps - 1) / warps, warps * 32, 0, c->stream>>>(rewards, lengths, n_groups,
+                                                                                      group_size, estimator, adv_seq);
+  c->launches++;
+  if (estimator == RL_ADV_REINFORCE_PP) {
+    double* stats = reinterpret_cast<double*>(reinterpret_cast<char*>(c->dstatus) + 64);
+    batch_stats_kernel<<<1, 1024, 0, c->stream>>>(adv_seq, (long long)n_seq, stats);
+    int blocks = (int)((n_seq + 255) / 256);
+    if (blocks > 4096) blocks = 4096;
+    batch_normalise_kernel<<<blocks, 256, 0, c->stream>>>(adv_seq, (long long)n_seq, stats, eps_std);
+    c->launches += 2;
+  }
+  prof_end(c, pr, 8);
   return cuda_ok();
 }
 

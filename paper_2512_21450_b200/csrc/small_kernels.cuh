@@ -174,6 +174,77 @@ __global__ void __launch_bounds__(256) grpo_adv_kernel(const float* __restrict__
   for (int i = lane; i < G; i += 32) adv_seq[(size_t)g * G + i] = (mx == mn) ? 0.f : (r[i] - mu) * inv;
 }
 
+// Other critic-free estimators named in section 4.2 (no formula printed there; readings):
+//   est 1 RLOO: A_i = r_i - mean of the other responses of the group
+//   est 2 OPO : A_i = r_i - sum_j(len_j r_j) / sum_j(len_j)          (length-weighted baseline)
+//   est 3     : c_i = r_i - group mean (first stage of REINFORCE++; batch normalisation follows)
+// One warp per group, shuffle reductions.
+__global__ void __launch_bounds__(256) group_baseline_kernel(const float* __restrict__ rewards,
+                                                             const int* __restrict__ lengths, int n_groups, int G,
+                                                             int est, float* __restrict__ adv_seq) {
+  const int lane = threadIdx.x & 31;
+  const int g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (g >= n_groups) return;
+  const float* r = rewards + (size_t)g * G;
+  float sr = 0.f, sl = 0.f, slr = 0.f;
+  for (int i = lane; i < G; i += 32) {
+    const float x = r[i];
+    const float l = (est == 2) ? (float)lengths[(size_t)g * G + i] : 1.f;
+    sr += x;
+    sl += l;
+    slr = fmaf(l, x, slr);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    sr += __shfl_xor_sync(0xffffffffu, sr, o);
+    sl += __shfl_xor_sync(0xffffffffu, sl, o);
+    slr += __shfl_xor_sync(0xffffffffu, slr, o);
+  }
+  for (int i = lane; i < G; i += 32) {
+    const float x = r[i];
+    float a;
+    if (est == 1) a = x - (sr - x) / (float)(G - 1);
+    else if (est == 2) a = x - (sl > 0.f ? slr / sl : 0.f);
+    else a = x - sr / (float)G;
+    adv_seq[(size_t)g * G + i] = a;
+  }
+}
+
+// Batch statistics of c[n] in double, fixed order (one block): stats[0] = mean, stats[1] = population std.
+__global__ void __launch_bounds__(1024) batch_stats_kernel(const float* __restrict__ c, long long n,
+                                                           double* __restrict__ stats) {
+  __shared__ double red[32];
+  __shared__ double mean_s;
+  double acc = 0.0;
+  for (long long i = threadIdx.x; i < n; i += blockDim.x) acc += (double)c[i];
+  for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double t = 0.0;
+      for (int w = 0; w < 32; ++w) t += red[w];
+      if (pass == 0) { mean_s = t / (double)n; stats[0] = mean_s; }
+      else stats[1] = sqrt(t / (double)n);
+    }
+    __syncthreads();
+    if (pass == 0) {
+      const double mu = mean_s;
+      acc = 0.0;
+      for (long long i = threadIdx.x; i < n; i += blockDim.x) { const double dlt = (double)c[i] - mu; acc += dlt * dlt; }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) batch_normalise_kernel(float* __restrict__ c, long long n,
+                                                              const double* __restrict__ stats, float eps_std) {
+  const double mu = stats[0];
+  const double inv = 1.0 / (stats[1] + (double)eps_std);
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    c[i] = (float)(((double)c[i] - mu) * inv);
+}
+
 // Broadcast of the per-response advantage to the rows of the response (outcome supervision).
 __global__ void __launch_bounds__(256) broadcast_adv_kernel(const float* __restrict__ adv_seq,
                                                             const int* __restrict__ seq_offsets, int n_seq,

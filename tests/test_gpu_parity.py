@@ -141,6 +141,21 @@ def test_advantages(ctx, n_groups, G):
                 assert not _np64(a).any()
 
 
+@pytest.mark.parametrize("n_groups,G", [(8, 8), (5, 3), (64, 16), (3, 40), (2048, 8)])
+def test_other_advantage_estimators(ctx, n_groups, G):
+    rng = np.random.default_rng(300 + G)
+    r = rng.uniform(size=n_groups * G).astype(np.float32)
+    ln = rng.integers(1, 513, size=n_groups * G).astype(np.int32)
+    rt, lt = torch.from_numpy(r).cuda(), torch.from_numpy(ln).cuda()
+    # rewards are O(1); fp32 arithmetic on them stays within the advantage tolerance
+    assert np.abs(_np64(ctx.rl_advantages("rloo", rt, G)) - O.rloo_advantages(r, G)).max() <= TOL_ADV
+    assert np.abs(_np64(ctx.rl_advantages("opo", rt, G, lengths=lt)) - O.opo_advantages(r, ln, G)).max() <= TOL_ADV
+    assert np.abs(_np64(ctx.rl_advantages("grpo", rt, G)) - O.grpo_advantages(r, G)).max() <= TOL_ADV
+    # batch-normalised values are O(3): allow a few fp32 ulps of that
+    pp = _np64(ctx.rl_advantages("reinforce_pp", rt, G))
+    assert np.abs(pp - O.reinforce_pp_advantages(r, G)).max() <= 4e-6
+
+
 def test_config0_full(ctx):
     from paper_2512_21450_b200.workloads import make_workload
     w = make_workload(0)

@@ -389,3 +389,90 @@ def test_custom_token_weight_and_sampled_helpers():
     dWs = O.dW_rows(H[rows], W[sel], sel, tokens[rows], out["lse"][rows], out["entropy"][rows],
                     w[rows] * dlogp, w[rows] * 0.02)
     assert np.allclose(dWs, out["dW"][sel], atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- aggregation / sequence level
+def test_aggregation_weights():
+    mask = np.array([1, 1, 0, 1, 0, 0, 1, 1, 1], dtype=np.uint8)
+    off = np.array([0, 3, 6, 9])
+    w0 = O.aggregation_weights(mask, off, 0)
+    assert np.allclose(w0, mask / 6.0)
+    w1 = O.aggregation_weights(mask, off, 1)
+    assert np.allclose(w1, [1 / 6, 1 / 6, 0, 1 / 3, 0, 0, 1 / 9, 1 / 9, 1 / 9])
+    assert abs(w1.sum() - 1.0) < 1e-15                      # every sequence has a valid token
+    w2 = O.aggregation_weights(mask, off, 2)
+    assert np.allclose(w2, mask / 9.0)
+    # equal, fully valid sequences: the three modes coincide
+    full = np.ones(12)
+    offs = np.array([0, 4, 8, 12])
+    for mode in (1, 2):
+        assert np.allclose(O.aggregation_weights(full, offs, mode), O.aggregation_weights(full, offs, 0))
+    # a sequence without valid tokens contributes nothing
+    assert np.allclose(O.aggregation_weights(np.array([1, 1, 0, 0]), np.array([0, 2, 4]), 1), [0.25, 0.25, 0, 0])
+
+
+def test_sequence_ratio_is_geometric_mean():
+    logp = np.log(np.array([0.5, 0.25, 0.1, 0.2]))
+    old = np.log(np.array([0.25, 0.25, 0.2, 0.2]))
+    rho, ln = O.sequence_ratio(logp, old, np.array([1, 1, 1, 0]), np.array([0, 2, 4]))
+    assert np.allclose(rho, [math.sqrt(2.0 * 1.0), math.sqrt(2.0), 0.5, 1.0]) and ln.tolist() == [2, 2, 1, 0]
+
+
+@pytest.mark.parametrize("agg_mode", [0, 1, 2])
+def test_sequence_level_gradient_finite_differences_and_autograd(agg_mode):
+    rng = _rng(31)
+    T, d, V = 9, 6, 12
+    off = np.array([0, 4, 5, 9])
+    H = rng.normal(size=(T, d))
+    W = rng.normal(size=(V, d)) * 0.5
+    tokens = rng.integers(0, V, size=T)
+    mask = np.array([1, 1, 0, 1, 1, 1, 1, 1, 0], dtype=np.uint8)
+    lp, _, _ = O.token_logprobs(H, W, tokens)
+    old = lp + rng.normal(size=T) * 0.4
+    ref = lp + rng.normal(size=T) * 0.2
+    adv = rng.normal(size=T)
+    kw = dict(eps_low=0.15, eps_high=0.2, beta=0.1, ent_coef=0.02, seq_offsets=off, agg_mode=agg_mode,
+              sequence_level=True)
+    out = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, **kw)
+    assert out["active"].any() and (~out["active"]).any()
+
+    def loss(Hx, Wx):
+        return O.policy_loss_fwd_bwd(Hx, Wx, tokens, old, ref, adv, mask, **kw)["loss"]
+
+    h = 1e-6
+    for (X, dX, which) in ((H, out["dH"], 0), (W, out["dW"], 1)):
+        num = np.zeros_like(X)
+        for idx in np.ndindex(*X.shape):
+            Xp = X.copy(); Xp[idx] += h
+            Xm = X.copy(); Xm[idx] -= h
+            num[idx] = ((loss(Xp, W) - loss(Xm, W)) if which == 0 else (loss(H, Xp) - loss(H, Xm))) / (2 * h)
+        assert np.abs(num - dX).max() / max(np.abs(num).max(), 1e-12) < 1e-6
+    # library second opinion: float64 autograd of the sequence-level objective
+    Ht = torch.tensor(H, requires_grad=True)
+    Wt = torch.tensor(W, requires_grad=True)
+    lsm = torch.log_softmax(Ht @ Wt.T, dim=1)
+    lpt = lsm.gather(1, torch.tensor(tokens)[:, None])[:, 0]
+    ent = -(lsm.exp() * lsm).sum(1)
+    mt = torch.tensor(mask.astype(np.float64))
+    wt = torch.tensor(O.aggregation_weights(mask, off, agg_mode))
+    total = 0.0
+    for i in range(3):
+        sl = slice(off[i], off[i + 1])
+        mi = mt[sl]
+        ratio = (((lpt[sl] - torch.tensor(old[sl])) * mi).sum() / mi.sum()).exp()
+        A = torch.tensor(adv[sl])
+        s = torch.minimum(ratio * A, ratio.clamp(1 - 0.15, 1 + 0.2) * A)
+        dl = torch.tensor(ref[sl]) - lpt[sl]
+        total = total + (wt[sl] * (-s + 0.1 * (dl.exp() - dl - 1) - 0.02 * ent[sl])).sum()
+    total.backward()
+    assert abs(total.item() - out["loss"]) < 1e-13
+    assert np.allclose(Ht.grad.numpy(), out["dH"], atol=1e-13) and np.allclose(Wt.grad.numpy(), out["dW"], atol=1e-13)
+
+
+def test_sequence_level_reduces_to_token_level_for_single_token_sequences():
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(33, T=6, d=8, V=16, masked=())
+    off = np.arange(7)
+    a = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, 0.2, 0.2, 0.04, seq_offsets=off, sequence_level=True)
+    b = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, 0.2, 0.2, 0.04)
+    assert abs(a["loss"] - b["loss"]) < 1e-15 and np.allclose(a["dH"], b["dH"], atol=1e-15)
+    assert np.allclose(a["dW"], b["dW"], atol=1e-15)
