@@ -148,6 +148,18 @@ typedef struct {
   float* entropy_out;         /* [T] or NULL                                                   */
   float* metrics_out;         /* [8] or NULL: pg_loss, kl_mean, entropy_mean, clip_frac,       */
                               /* ratio_mean, ratio_max, n_valid, reserved                      */
+  int agg_mode;               /* token weights when token_weight is NULL: 0 token mean over    */
+                              /* the call; 1 mean over responses of each response's token mean */
+                              /* (w = mask/(n_seq*len_i)); 2 mean over responses of the token  */
+                              /* sum over the longest row range (w = mask/(n_seq*L_max))       */
+  int sequence_level;         /* non-zero: sequence-level importance ratio ("GSPO's sequence-  */
+                              /* level aggregation", section 4.2; reading: rho_i = exp(mean    */
+                              /* token log-ratio over the valid tokens of response i), used    */
+                              /* and clipped for every token of the response                   */
+  int dH_dtype;               /* 0: dH is bf16 [T,d]; 1: dH is fp32 [T,d]                      */
+  const int32_t* seq_offsets; /* [n_seq+1] ascending row range of every response, needed by    */
+  int64_t n_seq;              /* agg_mode 1/2 and sequence_level; seq_offsets[n_seq] <= T;     */
+                              /* valid rows outside every range then take no part in the loss  */
 } rl_loss_opts;
 
 rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* ctx, const void* H, int64_t ldH, const void* W,

@@ -37,6 +37,11 @@ class rl_loss_opts(ctypes.Structure):
         ("logp_out", c_void_p),
         ("entropy_out", c_void_p),
         ("metrics_out", c_void_p),
+        ("agg_mode", c_int),
+        ("sequence_level", c_int),
+        ("dH_dtype", c_int),
+        ("seq_offsets", c_void_p),
+        ("n_seq", c_int64),
     ]
 
 
@@ -201,7 +206,8 @@ class Context:
 
     def rl_policy_loss_fwd_bwd(self, H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta,
                                ent_coef=0.0, token_weight=None, accumulate_dW=False, dW=None, want_aux=True,
-                               dH=None, loss=None):
+                               dH=None, loss=None, agg_mode=0, sequence_level=False, seq_offsets=None,
+                               dH_fp32=False):
         self._bind_stream()
         T, d = H.shape
         V = W.shape[0]
@@ -210,11 +216,13 @@ class Context:
         self.ensure_workspace(T, d, V)
         dev = W.device
         loss = torch.empty(1, dtype=torch.float32, device=dev) if loss is None else loss
-        dH = torch.empty(T, d, dtype=torch.bfloat16, device=dev) if dH is None else dH
+        if dH is None:
+            dH = torch.empty(T, d, dtype=torch.float32 if dH_fp32 else torch.bfloat16, device=dev)
         if dW is None:
             dW = torch.empty(V, d, dtype=torch.float32, device=dev)
         out = dict(loss=loss, dH=dH, dW=dW)
-        plain = (ent_coef == 0.0 and token_weight is None and not accumulate_dW and not want_aux)
+        plain = (ent_coef == 0.0 and token_weight is None and not accumulate_dW and not want_aux and agg_mode == 0
+                 and not sequence_level and not dH_fp32)
         args = [self.handle, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0), _ptr(tokens), _ptr(old_logp),
                 _ptr(ref_logp), _ptr(adv), _ptr(mask), T, d, V, eps_low, eps_high, beta, _ptr(loss), _ptr(dH),
                 _ptr(dW)]
@@ -226,6 +234,13 @@ class Context:
         opts.ent_coef = ent_coef
         opts.token_weight = token_weight.data_ptr() if token_weight is not None else None
         opts.accumulate_dW = int(accumulate_dW)
+        opts.agg_mode = agg_mode
+        opts.sequence_level = int(sequence_level)
+        opts.dH_dtype = int(dH_fp32)
+        if seq_offsets is not None:
+            assert seq_offsets.dtype == torch.int32 and seq_offsets.is_cuda
+            opts.seq_offsets = seq_offsets.data_ptr()
+            opts.n_seq = seq_offsets.numel() - 1
         if want_aux:
             out["logp"] = torch.empty(T, dtype=torch.float32, device=dev)
             out["entropy"] = torch.empty(T, dtype=torch.float32, device=dev)

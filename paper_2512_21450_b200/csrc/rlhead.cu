@@ -51,7 +51,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
   int Tpad, Ts, Vs;
-  size_t scan_counts, row_map, tokens_c, lse_c, ent_c, cp_c, ce_c, partials, block_sums, Hc, G, dH_acc, staging, total;
+  size_t scan_counts, row_map, tokens_c, logp_c, lse_c, ent_c, cp_c, ce_c, partials, block_sums, Hc, G, dH_acc, staging, total;
 };
 
 // staging_T > 0 adds room for host-call inputs (H, tokens, old, ref, adv, mask).
@@ -66,6 +66,7 @@ WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_s
   L.scan_counts = take(((size_t)L.Tpad / 4096 + 2) * 4);
   L.row_map = take((size_t)L.Tpad * 4);
   L.tokens_c = take((size_t)L.Tpad * 4);
+  L.logp_c = take((size_t)L.Tpad * 4);
   L.lse_c = take((size_t)L.Tpad * 4);
   L.ent_c = take((size_t)L.Tpad * 4);
   L.cp_c = take((size_t)L.Tpad * 4);
@@ -529,6 +530,10 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
     memcpy(&o, opts, opts->struct_size);
   }
   if (!(o.ent_coef >= 0.f)) return RL_ERR_INVALID_ARG;
+  if (o.agg_mode < 0 || o.agg_mode > 2 || (o.dH_dtype != 0 && o.dH_dtype != 1)) return RL_ERR_INVALID_ARG;
+  if ((o.sequence_level || (o.agg_mode != 0 && !o.token_weight)) && T > 0 &&
+      (!o.seq_offsets || o.n_seq <= 0 || o.n_seq > T))
+    return RL_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(dH) & 15) || (reinterpret_cast<uintptr_t>(dW) & 15)) return RL_ERR_ALIGNMENT;
   const WsLayout L = ws_layout(c, T, d, V, false);
   if ((s = check_ws(c, L)) != RL_OK) return s;
@@ -541,7 +546,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
     if (o.metrics_out) cudaMemsetAsync(o.metrics_out, 0, 32, st);
     return cuda_ok();
   }
-  cudaMemsetAsync(dH, 0, (size_t)T * d * 2, st);
+  cudaMemsetAsync(dH, 0, (size_t)T * d * (o.dH_dtype ? 4 : 2), st);
   if (o.logp_out) cudaMemsetAsync(o.logp_out, 0, (size_t)T * 4, st);
   if (o.entropy_out) cudaMemsetAsync(o.entropy_out, 0, (size_t)T * 4, st);
 
@@ -577,10 +582,45 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
   if (blocks > 1024) blocks = 1024;
   const int pr_loss = prof_begin(c, 6);
-  combine_loss_kernel<<<blocks, kLossThreads, 0, st>>>(p, c->dstatus);
+  const bool seq_path = o.sequence_level || (o.agg_mode != 0 && !o.token_weight);
+  if (!seq_path) {
+    combine_loss_kernel<<<blocks, kLossThreads, 0, st>>>(p, c->dstatus);
+    c->launches++;
+  } else {
+    // merge the statistics first, then one warp per response forms weights, ratios and the loss
+    p.with_loss = 0;
+    p.logp_c = reinterpret_cast<float*>(ws + L.logp_c);
+    combine_loss_kernel<<<blocks, kLossThreads, 0, st>>>(p, c->dstatus);
+    SeqParams q;
+    memset(&q, 0, sizeof(q));
+    q.seq_offsets = o.seq_offsets;
+    q.n_seq = (int)o.n_seq;
+    q.agg_mode = o.token_weight ? 0 : o.agg_mode;
+    q.sequence_level = o.sequence_level ? 1 : 0;
+    q.row_map = p.row_map;
+    q.logp_c = p.logp_c;
+    q.ent_c = p.ent_c;
+    q.old_logp = old_logp;
+    q.ref_logp = ref_logp;
+    q.adv = adv;
+    q.token_weight = o.token_weight;
+    q.eps_low = eps_low; q.eps_high = eps_high; q.beta = beta; q.ent_coef = o.ent_coef;
+    q.l_max = reinterpret_cast<int*>(reinterpret_cast<char*>(c->dstatus) + 96);
+    q.cp_c = p.cp_c;
+    q.ce_c = p.ce_c;
+    q.block_sums = p.block_sums;
+    // valid rows that lie outside every response range take no part: their coefficients stay 0
+    cudaMemsetAsync(q.cp_c, 0, (size_t)L.Tpad * 4, st);
+    cudaMemsetAsync(q.ce_c, 0, (size_t)L.Tpad * 4, st);
+    seq_lmax_kernel<<<1, 1024, 0, st>>>(o.seq_offsets, (int)o.n_seq, q.l_max);
+    blocks = (int)((o.n_seq + kLossThreads / 32 - 1) / (kLossThreads / 32));
+    if (blocks > 1024) blocks = 1024;
+    seq_loss_kernel<<<blocks, kLossThreads, 0, st>>>(q, c->dstatus);
+    c->launches += 3;
+  }
   finalize_loss_kernel<<<1, 32, 0, st>>>(p.block_sums, blocks, loss, o.metrics_out, c->dstatus);
   prof_end(c, pr_loss, 6);
-  c->launches += 2;
+  c->launches++;
 
   // ---- backward, one (row slab x vocabulary slab) at a time
   __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + L.Hc);
@@ -658,8 +698,12 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
       }
     }
     const int pr_sc = prof_begin(c, 7);
-    scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
-                                                   static_cast<__nv_bfloat16*>(dH), c->dstatus);
+    if (o.dH_dtype)
+      scatter_dH_f32_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
+                                                         static_cast<float*>(dH), c->dstatus);
+    else
+      scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
+                                                     static_cast<__nv_bfloat16*>(dH), c->dstatus);
     prof_end(c, pr_sc, 7);
     c->launches++;
   }

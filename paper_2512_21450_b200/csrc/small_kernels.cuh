@@ -276,6 +276,7 @@ struct LossParams {
   // compact outputs
   float* lse_c;
   float* ent_c;
+  float* logp_c;   // compact log-probabilities, or NULL
   float* cp_c;
   float* ce_c;
   // scattered outputs (original rows), any may be NULL
@@ -312,6 +313,7 @@ __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossPa
     const int row = p.row_map[i];
     p.lse_c[i] = lse;
     p.ent_c[i] = ent;
+    if (p.logp_c) p.logp_c[i] = logp;
     if (p.logp_out) p.logp_out[row] = logp;
     if (p.ent_out) p.ent_out[row] = ent;
     if (p.lse_out) p.lse_out[row] = lse;
@@ -364,6 +366,141 @@ __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossPa
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Sequence-aware loss path: aggregation weights that depend on each response's valid length
+// (section 2.2 "length normalization with token weights") and the sequence-level importance
+// ratio (section 4.2 "GSPO's sequence-level aggregation"; reading: rho_i = exp of the mean
+// token log-ratio over the valid tokens of response i, used by every token of the response).
+// One warp per response; its valid tokens are the compact rows [lo, hi) found by binary search
+// in the ascending row map.
+struct SeqParams {
+  const int* seq_offsets;   // [n_seq + 1] row range of each response
+  int n_seq;
+  int agg_mode;             // 0 token mean, 1 mean of per-response token means, 2 token sum / (B * L_max)
+  int sequence_level;       // 1: sequence-level ratio
+  const int* row_map;
+  const float* logp_c;
+  const float* ent_c;
+  const float* old_logp;
+  const float* ref_logp;
+  const float* adv;
+  const float* token_weight;  // overrides agg_mode when not NULL
+  float eps_low, eps_high, beta, ent_coef;
+  int* l_max;               // device scalar: longest row range
+  float* cp_c;
+  float* ce_c;
+  double* block_sums;       // [gridDim.x][kLossSums]
+};
+
+__global__ void __launch_bounds__(1024) seq_lmax_kernel(const int* __restrict__ seq_offsets, int n_seq, int* l_max) {
+  __shared__ int red[32];
+  int m = 0;
+  for (int i = threadIdx.x; i < n_seq; i += blockDim.x) m = max(m, seq_offsets[i + 1] - seq_offsets[i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 32; ++w) m = max(m, red[w]);
+    *l_max = m;
+  }
+}
+
+__device__ __forceinline__ int lower_bound_rows(const int* __restrict__ row_map, int n, int key) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (row_map[mid] < key) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void __launch_bounds__(kLossThreads) seq_loss_kernel(const SeqParams p, DevStatus* st) {
+  const int n = st->n_valid;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warps_per_block = kLossThreads / 32;
+  double acc[kLossSums];
+#pragma unroll
+  for (int k = 0; k < kLossSums; ++k) acc[k] = 0.0;
+  for (int sq = blockIdx.x * warps_per_block + warp; sq < p.n_seq; sq += gridDim.x * warps_per_block) {
+    const int lo = lower_bound_rows(p.row_map, n, p.seq_offsets[sq]);
+    const int hi = lower_bound_rows(p.row_map, n, p.seq_offsets[sq + 1]);
+    const int len = hi - lo;
+    if (len <= 0) continue;
+    float w_seq = 0.f;
+    if (p.agg_mode == 0) w_seq = 1.f / (float)n;
+    else if (p.agg_mode == 1) w_seq = 1.f / ((float)p.n_seq * (float)len);
+    else w_seq = 1.f / ((float)p.n_seq * (float)max(*p.l_max, 1));
+    float rho_seq = 1.f, seq_sum = 0.f;
+    if (p.sequence_level) {
+      float lr = 0.f;
+      for (int k = lo + lane; k < hi; k += 32) lr += p.logp_c[k] - p.old_logp[p.row_map[k]];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) lr += __shfl_xor_sync(0xffffffffu, lr, o);
+      rho_seq = expf(lr / (float)len);
+      const float clipped = fminf(fmaxf(rho_seq, 1.f - p.eps_low), 1.f + p.eps_high);
+      for (int k = lo + lane; k < hi; k += 32) {
+        const int row = p.row_map[k];
+        const float w = p.token_weight ? p.token_weight[row] : w_seq;
+        const float A_t = p.adv[row];
+        const bool active = rho_seq * A_t <= clipped * A_t;
+        seq_sum += active ? w * A_t : 0.f;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) seq_sum += __shfl_xor_sync(0xffffffffu, seq_sum, o);
+    }
+    for (int k = lo + lane; k < hi; k += 32) {
+      const int row = p.row_map[k];
+      const float w = p.token_weight ? p.token_weight[row] : w_seq;
+      const float A_t = p.adv[row];
+      const float logp = p.logp_c[k];
+      const float ent = p.ent_c[k];
+      const float rho = p.sequence_level ? rho_seq : expf(logp - p.old_logp[row]);
+      const float clipped = fminf(fmaxf(rho, 1.f - p.eps_low), 1.f + p.eps_high);
+      const float su = rho * A_t, sc = clipped * A_t;
+      const bool active = su <= sc;
+      const float s = active ? su : sc;
+      float k3 = 0.f, dk3 = 0.f;
+      if (p.beta != 0.f) {
+        const float delta = p.ref_logp[row] - logp;
+        const float ed = expf(delta);
+        k3 = ed - delta - 1.f;
+        dk3 = 1.f - ed;
+      }
+      // weighted d loss / d logp_t
+      const float wdlogp = (p.sequence_level ? -(rho_seq / (float)len) * seq_sum : -(active ? w * A_t * rho : 0.f)) +
+                           w * p.beta * dk3;
+      p.cp_c[k] = -wdlogp;
+      p.ce_c[k] = w * p.ent_coef;
+      acc[0] += (double)w * (double)(-s + p.beta * k3 - p.ent_coef * ent);
+      acc[1] += (double)w * (double)(-s);
+      acc[2] += (double)w * (double)k3;
+      acc[3] += (double)w * (double)ent;
+      acc[4] += active ? 0.0 : (double)w;
+      acc[5] += (double)w * (double)rho;
+      acc[6] = fmax(acc[6], (double)rho);
+    }
+  }
+  __shared__ double red[kLossThreads / 32][kLossSums];
+#pragma unroll
+  for (int k = 0; k < kLossSums; ++k) {
+    double v = acc[k];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double u = __shfl_xor_sync(0xffffffffu, v, o);
+      v = (k == 6) ? fmax(v, u) : v + u;
+    }
+    if (lane == 0) red[warp][k] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < kLossSums) {
+    const int k = threadIdx.x;
+    double v = red[0][k];
+    for (int w = 1; w < kLossThreads / 32; ++w) v = (k == 6) ? fmax(v, red[w][k]) : v + red[w][k];
+    p.block_sums[(size_t)blockIdx.x * kLossSums + k] = v;
+  }
+}
+
 // Second stage: fixed-order sum of the block partials -> loss[1] and metrics[8].
 __global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restrict__ block_sums, int n_blocks,
                                                            float* __restrict__ loss, float* __restrict__ metrics,
@@ -385,6 +522,21 @@ __global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restr
 // ------------------------------------------------------------------------------------------
 // dH of one row slab: fp32 accumulator rows -> bf16 rows of the caller's dH at their original
 // positions.  One warp per row.
+// Same with an fp32 destination.
+__global__ void __launch_bounds__(256) scatter_dH_f32_kernel(const float* __restrict__ acc, int d, int slab_base,
+                                                             int slab_rows, const int* __restrict__ row_map,
+                                                             float* __restrict__ dH, const DevStatus* st) {
+  const int n = st->n_valid;
+  const int rows = min(max(n - slab_base, 0), slab_rows);
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
+    const float4* src = reinterpret_cast<const float4*>(acc + (size_t)i * d);
+    float4* dst = reinterpret_cast<float4*>(dH + (size_t)row_map[slab_base + i] * d);
+    for (int v = lane; v < d / 4; v += 32) dst[v] = src[v];
+  }
+}
+
 __global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict__ acc, int d, int slab_base,
                                                          int slab_rows, const int* __restrict__ row_map,
                                                          __nv_bfloat16* __restrict__ dH, const DevStatus* st) {

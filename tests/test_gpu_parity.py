@@ -46,7 +46,8 @@ def _oracle_case(w, adv_tok_np, **kw):
         w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef, **kw)
 
 
-def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5):
+def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5, agg_mode=0, sequence_level=False,
+                          dH_fp32=False):
     from paper_2512_21450_b200.workloads import Workload  # noqa: F401
     adv_seq, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
     o_adv = O.grpo_advantages(w.rewards.cpu().numpy(), w.G)
@@ -56,10 +57,14 @@ def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5):
 
     out = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask,
                                      w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef,
-                                     token_weight=token_weight)
+                                     token_weight=token_weight, agg_mode=agg_mode, sequence_level=sequence_level,
+                                     seq_offsets=w.seq_offsets if (agg_mode or sequence_level) else None,
+                                     dH_fp32=dH_fp32)
     _assert_status_ok(ctx)
+    assert out["dH"].dtype == (torch.float32 if dH_fp32 else torch.bfloat16)
     # the oracle works from its own advantages; nothing it sees comes from the CUDA path
-    oo = _oracle_case(w, o_adv_tok, token_weight=None if token_weight is None else _np64(token_weight))
+    oo = _oracle_case(w, o_adv_tok, token_weight=None if token_weight is None else _np64(token_weight),
+                      seq_offsets=w.seq_offsets.cpu().numpy(), agg_mode=agg_mode, sequence_level=sequence_level)
     m = w.mask.cpu().numpy().astype(bool)
     assert np.abs(_np64(out["logp"]) - oo["logp"]).max() <= TOL_LOGP
     assert np.abs(_np64(out["entropy"]) - oo["entropy"]).max() <= TOL_ENT
@@ -180,6 +185,27 @@ def test_reduced_configs(ctx, cfg_id, prompts, L_max):
         assert (r.max(axis=1) == r.min(axis=1)).any()     # a zero-variance group is present
         assert w.ref_logp is None and w.ent_coef > 0
     _check_against_oracle(ctx, w)
+
+
+@pytest.mark.parametrize("agg_mode,sequence_level", [(1, False), (2, False), (0, True), (1, True), (2, True)])
+def test_aggregation_modes_and_sequence_level_ratio(ctx, agg_mode, sequence_level):
+    from paper_2512_21450_b200.workloads import make_workload
+    # ragged right-padded responses (3B-class head), and responses with masked spans inside
+    def shift_behaviour_policy(w):
+        # the sequence-level ratio averages the token noise away; a per-response offset of the
+        # behaviour log-probs puts some responses outside the clip band and leaves others inside
+        bias = torch.tensor([0.45, 0.0, -0.45, 0.1], device=w.old_logp.device).repeat(w.n_seq // 4 + 1)[:w.n_seq]
+        w.old_logp = (w.old_logp + bias.repeat_interleave(w.L_max)) * w.mask
+
+    w = make_workload(1, prompts=1, L_max=96, seed=800 + agg_mode, sigma_old=0.3)
+    shift_behaviour_policy(w)
+    out, oo = _check_against_oracle(ctx, w, agg_mode=agg_mode, sequence_level=sequence_level,
+                                    dH_fp32=(agg_mode == 2))
+    if sequence_level:
+        assert 0.0 < oo["clip_frac"] < 1.0            # some responses clipped, some not
+    w = make_workload(3, prompts=2, L_max=64, seed=810 + agg_mode, d=256, V=5000, sigma_old=0.3)
+    shift_behaviour_policy(w)
+    _check_against_oracle(ctx, w, agg_mode=agg_mode, sequence_level=sequence_level)
 
 
 def test_clip_exercised_and_peaked_rows(ctx):
