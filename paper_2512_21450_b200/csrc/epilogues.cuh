@@ -34,7 +34,7 @@ struct EpiStats {
     int y;
   };
   __device__ static __forceinline__ void begin_unit(const Params& p, State& st, int m_tile, int, int row_in_tile,
-                                                    int m_rows) {
+                                                    int m_rows, int) {
     st.m = -CUDART_INF_F;
     st.s = 0.f;
     st.a = 0.f;
@@ -116,7 +116,6 @@ struct EpiGrad {
     int ldG;
     int V;
     int vocab_base;  // global column of the slab's column 0
-    int row_base;    // compact row of the slab's row 0
   };
   struct State {
     float lse, ent, cp, ce;
@@ -124,10 +123,10 @@ struct EpiGrad {
     bool valid;
   };
   __device__ static __forceinline__ void begin_unit(const Params& p, State& st, int m_tile, int, int row_in_tile,
-                                                    int m_rows) {
+                                                    int m_rows, int slab_off) {
     const int rl = m_tile * BM + row_in_tile;
     st.valid = rl < m_rows;
-    const int gr = p.row_base + rl;
+    const int gr = slab_off + rl;   // compact row of this slab row
     st.lse = st.valid ? p.lse[gr] : 0.f;
     st.ent = st.valid ? p.ent[gr] : 0.f;
     st.cp = st.valid ? p.cp[gr] : 0.f;
@@ -204,7 +203,7 @@ struct EpiAcc {
     int row_base;
   };
   struct State {};
-  __device__ static __forceinline__ void begin_unit(const Params&, State&, int, int, int, int) {}
+  __device__ static __forceinline__ void begin_unit(const Params&, State&, int, int, int, int, int) {}
   __device__ static __forceinline__ void chunk(const Params& p, State&, int m_tile, int n_tile, int c,
                                                int row_in_tile, int m_rows, const float (&v)[32]) {
     const int rl = m_tile * BM + row_in_tile;

@@ -77,6 +77,11 @@ struct GemmShape {
   int n_range;      // consecutive column tiles per work unit; 0 = choose so that units fill the SMs
   int skip_if_k0;   // nothing to do at all when K is empty (otherwise the epilogue sees zeros)
   int n_fastest;    // 1: consecutive units walk the column ranges of one row tile first
+  // Row slabs of the backward pass: when slab_cap > 0 the valid rows are cut into
+  // ceil(n_valid / slab_cap) slabs of equal size (a multiple of 256, at most slab_cap) and this
+  // launch works on slab slab_index: its row offset replaces m_dyn_off / k_dyn_off, and is added
+  // to the A row coordinate (a_mn_slab) or the B k coordinate (b_k_slab).
+  int slab_cap, slab_index, a_mn_slab, b_k_slab;
   // coordinate offsets into the operands' global tensors
   int a_mn_off, a_k_off, b_mn_off, b_k_off;
 };
@@ -97,16 +102,34 @@ __host__ __device__ inline int choose_split(int m_units, int n_tiles, int n_work
 }
 
 struct GemmExtents {
-  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units;
+  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units, slab_off;
 };
+
+// Offset and row count of slab `index` when n_valid rows are cut into equal slabs of at most cap rows.
+__host__ __device__ inline void slab_extent(int n_valid, int cap, int index, int& off, int& rows) {
+  int n_slabs = (n_valid + cap - 1) / cap;
+  if (n_slabs < 1) n_slabs = 1;
+  int per = ((n_valid + n_slabs - 1) / n_slabs + 255) / 256 * 256;
+  if (per > cap) per = cap;
+  off = index * per;
+  rows = n_valid - off;
+  rows = rows < 0 ? 0 : (rows > per ? per : rows);
+}
 
 // cg = CTAs per output row tile, n_workers = gridDim.x / cg.
 __host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_valid, int cg, int n_workers) {
   GemmExtents e;
-  int m = n_valid - sh.m_dyn_off;
+  e.slab_off = 0;
+  int m, k;
+  if (sh.slab_cap > 0) {
+    slab_extent(n_valid, sh.slab_cap, sh.slab_index, e.slab_off, m);
+    k = m;
+  } else {
+    m = n_valid - sh.m_dyn_off;
+    k = n_valid - sh.k_dyn_off;
+  }
   m = m < 0 ? 0 : (m > sh.m_rows_cap ? sh.m_rows_cap : m);
   e.m_rows = sh.m_dyn ? m : sh.m_rows_cap;
-  int k = n_valid - sh.k_dyn_off;
   k = k < 0 ? 0 : (k > sh.k_cap ? sh.k_cap : k);
   const int k_len = sh.k_dyn ? k : sh.k_cap;
   e.m_units = (e.m_rows + BM * cg - 1) / (BM * cg);
@@ -127,7 +150,7 @@ __device__ __forceinline__ void unit_coords(const GemmShape& sh, const GemmExten
 
 // Epilogue functor contract (all methods run in the 128 epilogue threads, one tile row each):
 //   struct Epi { struct Params; struct State;
-//     static void begin_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows);
+//     static void begin_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows, int slab_off);
 //     static void chunk(const Params&, State&, int m_tile, int n_tile, int chunk, int row_in_tile, int m_rows, const float (&v)[32]);
 //     static void end_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows); };
 // m_tile counts 128-row tiles.
@@ -196,22 +219,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t full_local = smem_u32(&bar_full[stage]);
             const uint32_t a_dst = tiles_base + stage * Cfg::kStageBytes;
             const uint32_t b_dst = a_dst + kAStageBytes;
-            const int a_row = sh.a_mn_off + m * BM;
+            const int a_row = sh.a_mn_off + (sh.a_mn_slab ? ex.slab_off : 0) + m * BM;
             const int b_row = sh.b_mn_off + n * BN + (int)rank * Cfg::kBRows;
+            const int b_k = sh.b_k_off + (sh.b_k_slab ? ex.slab_off : 0) + kb * BK;
             if (CG == 1) {
               mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
               if (A_MN) tma_load_3d(a_dst, &tmA, full_local, 0, sh.a_k_off + kb * BK, a_row / 64);
               else      tma_load_2d(a_dst, &tmA, full_local, sh.a_k_off + kb * BK, a_row);
-              if (B_MN) tma_load_3d(b_dst, &tmB, full_local, 0, sh.b_k_off + kb * BK, b_row / 64);
-              else      tma_load_2d(b_dst, &tmB, full_local, sh.b_k_off + kb * BK, b_row);
+              if (B_MN) tma_load_3d(b_dst, &tmB, full_local, 0, b_k, b_row / 64);
+              else      tma_load_2d(b_dst, &tmB, full_local, b_k, b_row);
             } else {
               // the even CTA's barrier counts the bytes of both CTAs' copies
               if (rank == 0) mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
               const uint32_t full = mapa_cluster(full_local, 0);
               if (A_MN) tma_load_3d_pair(a_dst, &tmA, full, 0, sh.a_k_off + kb * BK, a_row / 64);
               else      tma_load_2d_pair(a_dst, &tmA, full, sh.a_k_off + kb * BK, a_row);
-              if (B_MN) tma_load_3d_pair(b_dst, &tmB, full, 0, sh.b_k_off + kb * BK, b_row / 64);
-              else      tma_load_2d_pair(b_dst, &tmB, full, sh.b_k_off + kb * BK, b_row);
+              if (B_MN) tma_load_3d_pair(b_dst, &tmB, full, 0, b_k, b_row / 64);
+              else      tma_load_2d_pair(b_dst, &tmB, full, b_k, b_row);
             }
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
@@ -298,7 +322,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       unit_coords(sh, ex, u, mu, nr);
       const int m = mu * CG + (int)rank;
       const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
-      Epi::begin_unit(ep, st, m, nr, row_in_tile, ex.m_rows);
+      Epi::begin_unit(ep, st, m, nr, row_in_tile, ex.m_rows, ex.slab_off);
       for (int n = n0; n < n1 && ok; ++n, ++t) {
         const uint32_t a = t & 1u, round = t >> 1;
         if (ex.k_blocks > 0) {

@@ -642,8 +642,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   const int n_col_slabs = (int)((V + L.Vs - 1) / L.Vs);
   const int d_tiles = (int)((d + BN - 1) / BN);
   for (int r = 0; r < n_row_slabs; ++r) {
-    const int row_base = r * L.Ts;
-    const int rows_cap = (L.Tpad - row_base) < L.Ts ? (L.Tpad - row_base) : L.Ts;
+    const int rows_cap = L.Ts;   // the valid rows are cut into equal slabs of at most Ts rows on the device
     for (int cs = 0; cs < n_col_slabs; ++cs) {
       const int vocab_base = cs * L.Vs;
       const int cols = (int)((V - vocab_base) < L.Vs ? (V - vocab_base) : L.Vs);
@@ -652,16 +651,16 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         GemmShape sh;
         memset(&sh, 0, sizeof(sh));
         sh.n_valid = n_valid;
-        sh.m_rows_cap = rows_cap; sh.m_dyn = 1; sh.m_dyn_off = row_base;
+        sh.m_rows_cap = rows_cap; sh.m_dyn = 1; sh.slab_cap = L.Ts; sh.slab_index = r;
         sh.k_cap = (int)d;
         sh.n_tiles = (cols + BN - 1) / BN;
         sh.n_range = 1;
-        sh.a_mn_off = row_base;
+        sh.a_mn_slab = 1;
         sh.b_mn_off = vocab_base;
         EpiGrad::Params ep;
         ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
         ep.lse = p.lse_c; ep.ent = p.ent_c; ep.cp = p.cp_c; ep.ce = p.ce_c;
-        ep.G = G; ep.ldG = L.Vs; ep.V = (int)V; ep.vocab_base = vocab_base; ep.row_base = row_base;
+        ep.G = G; ep.ldG = L.Vs; ep.V = (int)V; ep.vocab_base = vocab_base;
         launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, sh, ep);
       }
       // (2) dH_slab (+)= G * W_slab        [rows x d], K = vocabulary columns of the slab
@@ -669,7 +668,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         GemmShape sh;
         memset(&sh, 0, sizeof(sh));
         sh.n_valid = n_valid;
-        sh.m_rows_cap = rows_cap; sh.m_dyn = 1; sh.m_dyn_off = row_base;
+        sh.m_rows_cap = rows_cap; sh.m_dyn = 1; sh.slab_cap = L.Ts; sh.slab_index = r;
         sh.k_cap = cols;
         sh.n_tiles = d_tiles;
         sh.n_range = 1;
@@ -685,11 +684,11 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         memset(&sh, 0, sizeof(sh));
         sh.n_valid = n_valid;
         sh.m_rows_cap = cols;
-        sh.k_cap = rows_cap; sh.k_dyn = 1; sh.k_dyn_off = row_base;
+        sh.k_cap = rows_cap; sh.k_dyn = 1; sh.slab_cap = L.Ts; sh.slab_index = r;
         sh.n_tiles = d_tiles;
         sh.n_range = 1;
         sh.skip_if_k0 = (r > 0 || o.accumulate_dW) ? 1 : 0;
-        sh.b_k_off = row_base;
+        sh.b_k_slab = 1;
         sh.n_fastest = 1;
         EpiAcc::Params ep;
         ep.C = dW; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
@@ -699,10 +698,10 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
     }
     const int pr_sc = prof_begin(c, 7);
     if (o.dH_dtype)
-      scatter_dH_f32_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
+      scatter_dH_f32_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, r, L.Ts, row_map,
                                                          static_cast<float*>(dH), c->dstatus);
     else
-      scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, row_base, rows_cap, row_map,
+      scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, r, L.Ts, row_map,
                                                      static_cast<__nv_bfloat16*>(dH), c->dstatus);
     prof_end(c, pr_sc, 7);
     c->launches++;

@@ -523,11 +523,11 @@ __global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restr
 // dH of one row slab: fp32 accumulator rows -> bf16 rows of the caller's dH at their original
 // positions.  One warp per row.
 // Same with an fp32 destination.
-__global__ void __launch_bounds__(256) scatter_dH_f32_kernel(const float* __restrict__ acc, int d, int slab_base,
-                                                             int slab_rows, const int* __restrict__ row_map,
+__global__ void __launch_bounds__(256) scatter_dH_f32_kernel(const float* __restrict__ acc, int d, int slab_index,
+                                                             int slab_cap, const int* __restrict__ row_map,
                                                              float* __restrict__ dH, const DevStatus* st) {
-  const int n = st->n_valid;
-  const int rows = min(max(n - slab_base, 0), slab_rows);
+  int slab_base, rows;
+  slab_extent(st->n_valid, slab_cap, slab_index, slab_base, rows);
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
@@ -537,11 +537,11 @@ __global__ void __launch_bounds__(256) scatter_dH_f32_kernel(const float* __rest
   }
 }
 
-__global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict__ acc, int d, int slab_base,
-                                                         int slab_rows, const int* __restrict__ row_map,
+__global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict__ acc, int d, int slab_index,
+                                                         int slab_cap, const int* __restrict__ row_map,
                                                          __nv_bfloat16* __restrict__ dH, const DevStatus* st) {
-  const int n = st->n_valid;
-  const int rows = min(max(n - slab_base, 0), slab_rows);
+  int slab_base, rows;
+  slab_extent(st->n_valid, slab_cap, slab_index, slab_base, rows);
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
