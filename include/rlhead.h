@@ -236,6 +236,12 @@ rl_status rl_selftest_gemm(rl_ctx* ctx, const void* A, const void* B, float* C,
                            int64_t M, int64_t N, int64_t K, int a_mn_major, int b_mn_major,
                            int accumulate);
 
+/* Self-test of the bounded waits every kernel of this library uses: launches one warp that waits,
+ * for at most limit_ms (1..1000) milliseconds, on a barrier nothing ever signals.  The kernel
+ * returns by itself with RL_ERR_TIMEOUT latched (detail 0x70000000); rl_last_device_status()
+ * reports and clears it and the context stays usable.  The paper has no counterpart. */
+rl_status rl_selftest_wait_timeout(rl_ctx* ctx, int limit_ms);
+
 #ifdef __cplusplus
 }
 #endif

@@ -71,6 +71,8 @@ def load_library():
     lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
     lib.rl_grpo_advantages.argtypes = [P, P, c_int64, c_int, P]
     lib.rl_grpo_advantages_ex.argtypes = [P, P, c_int64, c_int, c_int, c_float, P, c_int64, P, P]
+    lib.rl_selftest_wait_timeout.argtypes = [P, c_int]
+    lib.rl_selftest_wait_timeout.restype = c_int
     lib.rl_advantages.argtypes = [P, c_int, P, P, c_int64, c_int, c_float, P]
     lib.rl_advantages.restype = c_int
     lib.rl_token_logprobs.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P]
@@ -250,6 +252,10 @@ class Context:
             opts.metrics_out = out["metrics"].data_ptr()
         _check(self.lib.rl_policy_loss_fwd_bwd_ex(*args, byref(opts)), "rl_policy_loss_fwd_bwd_ex")
         return out
+
+    def selftest_wait_timeout(self, limit_ms=20):
+        self._bind_stream()
+        _check(self.lib.rl_selftest_wait_timeout(self.handle, limit_ms), "rl_selftest_wait_timeout")
 
     def launch_count(self):
         n = c_int64()

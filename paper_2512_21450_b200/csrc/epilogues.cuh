@@ -186,7 +186,7 @@ struct EpiGrad {
       o.y = *reinterpret_cast<uint32_t*>(&b1);
       o.z = *reinterpret_cast<uint32_t*>(&b2);
       o.w = *reinterpret_cast<uint32_t*>(&b3);
-      dst[j] = o;
+      __stcs(dst + j, o);   // written once, far larger than L2: do not displace the operands
     }
   }
   __device__ static __forceinline__ void end_unit(const Params&, State&, int, int, int, int) {}
@@ -215,10 +215,10 @@ struct EpiAcc {
       if (col0 + 4 * j < p.n_cols) {
         float4 x = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
         if (p.accumulate) {
-          const float4 o = dst[j];
+          const float4 o = __ldcs(dst + j);
           x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w;
         }
-        dst[j] = x;
+        __stcs(dst + j, x);   // each element is touched once per launch
       }
     }
   }

@@ -41,7 +41,8 @@ constexpr int kGemmThreads = 192;
 constexpr int kRingBytes = 224 * 1024;             // shared-memory ring of operand stages
 constexpr int kGemmSmemBytes = kRingBytes + 1024;  // + slack for 1024-byte alignment
 constexpr int kTmemCols = 512;
-constexpr int kMaxSplit = 16;
+constexpr int kMaxSplit = 16;   // most column ranges per row tile when the split is chosen to fill the machine
+constexpr int kFwdRange = 8;    // column tiles per work unit when there is plenty of work
 
 template <int CG>
 struct StageCfg {
@@ -134,8 +135,16 @@ __host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_v
   const int k_len = sh.k_dyn ? k : sh.k_cap;
   e.m_units = (e.m_rows + BM * cg - 1) / (BM * cg);
   e.k_blocks = (k_len + BK - 1) / BK;
-  const int split = sh.n_range > 0 ? 1 : choose_split(e.m_units, sh.n_tiles, n_workers);
-  e.n_range = sh.n_range > 0 ? sh.n_range : (sh.n_tiles + split - 1) / split;
+  if (sh.n_range > 0) {
+    e.n_range = sh.n_range;
+  } else if ((long)e.m_units * ((sh.n_tiles + kFwdRange - 1) / kFwdRange) >= 4L * n_workers) {
+    // plenty of work: short fixed ranges, walked rows-first, keep every worker within a few
+    // column tiles of the others, so the B operand is fetched from DRAM about once
+    e.n_range = kFwdRange;
+  } else {
+    const int split = choose_split(e.m_units, sh.n_tiles, n_workers);
+    e.n_range = (sh.n_tiles + split - 1) / split;
+  }
   if (e.n_range < 1) e.n_range = 1;
   e.n_ranges = (sh.n_tiles + e.n_range - 1) / e.n_range;
   e.n_units = e.m_units * e.n_ranges;

@@ -71,7 +71,12 @@ WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_s
   L.ent_c = take((size_t)L.Tpad * 4);
   L.cp_c = take((size_t)L.Tpad * 4);
   L.ce_c = take((size_t)L.Tpad * 4);
-  L.partials = take((size_t)kMaxSplit * L.Tpad * sizeof(float4));
+  {
+    // one float4 per (column range, row): at most kMaxSplit ranges, or one per kFwdRange column tiles
+    const size_t by_range = (size_t)(((V + BN - 1) / BN + kFwdRange - 1) / kFwdRange);
+    const size_t n_ranges = by_range > (size_t)kMaxSplit ? by_range : (size_t)kMaxSplit;
+    L.partials = take(n_ranges * L.Tpad * sizeof(float4));
+  }
   L.block_sums = take((size_t)1024 * kLossSums * sizeof(double));
   L.Hc = take((size_t)L.Tpad * d * 2);
   L.G = take((size_t)L.Ts * L.Vs * 2);
@@ -776,6 +781,13 @@ rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* c, const void* H_host, int64_t ldH
   loss_host[0] = h_out[0];
   if (metrics_host) memcpy(metrics_host, h_out + 8, 32);
   return RL_OK;
+}
+
+rl_status rl_selftest_wait_timeout(rl_ctx* c, int limit_ms) {
+  if (!c || limit_ms < 1 || limit_ms > 1000) return RL_ERR_INVALID_ARG;
+  wait_timeout_probe_kernel<<<1, 32, 0, c->stream>>>((unsigned long long)limit_ms * 1000000ull, c->dstatus);
+  c->launches++;
+  return cuda_ok();
 }
 
 rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,

@@ -558,4 +558,23 @@ __global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Exercises the bounded wait: one warp waits on an mbarrier that nothing ever arrives on, with a
+// short limit, and must come back with the timeout latched instead of spinning forever.
+__global__ void __launch_bounds__(32) wait_timeout_probe_kernel(unsigned long long limit_ns, DevStatus* st) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncwarp();
+  volatile int* abort_p = &abort_flag;
+  if (threadIdx.x == 0) {
+    if (!mbar_wait_bounded(smem_u32(&bar), 0, abort_p, limit_ns)) latch_status(st, kStatusTimeout, 0x70000000);
+  }
+  __syncwarp();
+}
+
 }  // namespace rlh

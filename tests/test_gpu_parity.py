@@ -345,6 +345,22 @@ def test_error_reporting(ctx):
     assert torch.isfinite(lp).all()
 
 
+def test_bounded_wait_times_out_cleanly(ctx):
+    # a wait that nothing satisfies ends by itself, reports RL_ERR_TIMEOUT and leaves the context usable
+    import time
+    from paper_2512_21450_b200.workloads import make_workload
+    t0 = time.time()
+    ctx.selftest_wait_timeout(limit_ms=20)
+    s, detail = ctx.last_device_status()
+    assert s == 8 and (detail & 0xffffffff) == 0x70000000
+    assert time.time() - t0 < 5.0
+    assert ctx.last_device_status()[0] == 0           # cleared
+    w = make_workload(0, seed=71)
+    lp, _, _ = ctx.rl_token_logprobs(w.H, w.W, w.tokens, w.mask)
+    _assert_status_ok(ctx)
+    assert torch.isfinite(lp).all()
+
+
 def test_run_to_run_determinism(ctx):
     from paper_2512_21450_b200.workloads import make_workload
     w = make_workload(1, prompts=1, L_max=40, seed=61)
