@@ -27,7 +27,8 @@ KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant
 # kernel from an ncu capture, valid only for the kernel sources whose hash is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": None, "kind": None, "bytes_per_launch": None}
+NCU_TRAFFIC = {"sources_sha256": "b4ebd80b3b3fbe1c951e9b149a8919fced29ca07d862cbfb833ef67b0ac21d3d", "kind": 2, "config": 1,
+               "bytes_per_launch": 1416770000 + 136509440}   # profiles/gemm_kernels_config1_ncu_full.md
 
 
 def sources_hash():
@@ -123,6 +124,11 @@ def oracle_sample_time(w, n_rows, repeat=1):
     return rows.numel(), best
 
 
+def workload_label(cfg_id, w):
+    return (f"config {cfg_id}: {w.name} d={w.d} V={w.V} rows={w.T} valid_tokens={w.n_valid} "
+            f"G={w.G} eps=({w.eps_low},{w.eps_high}) beta={w.beta} ent_coef={w.ent_coef}")
+
+
 def run_reference(args):
     import torch
     from paper_2512_21450_b200.workloads import CONFIGS, make_workload
@@ -149,7 +155,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / max(args.steps, 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"config {args.config}: {w.name} d={w.d} V={w.V}", "sample": sample},
+        "config": {"workload": workload_label(args.config, w), "sample": sample},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -253,21 +259,29 @@ def main():
     e2e_steps = max(3, min(args.steps, 10))
 
     def e2e_step():
-        return ctx.rl_policy_loss_fwd_bwd_host(hH, w.W, htok, hold, href, None, hmask, w.eps_low, w.eps_high, w.beta,
-                                               w.ent_coef, dH, dW, rewards_host=hrew, group_size=w.G,
-                                               seq_offsets_host=hoff)
-    e2e_val = None
+        out = ctx.rl_policy_loss_fwd_bwd_host(hH, w.W, htok, hold, href, None, hmask, w.eps_low, w.eps_high, w.beta,
+                                              w.ent_coef, dH, dW, rewards_host=hrew, group_size=w.G,
+                                              seq_offsets_host=hoff)
+        if world > 1:
+            # the host entry normalises by the local token count; the gradient exchange is the same
+            par.allreduce_gradients(dW, loss)
+        return out
+
+    for _ in range(2):
+        e2e_step()
+    fence()
+    e0.record()
+    for _ in range(e2e_steps):
+        host_loss, _ = e2e_step()
+    e1.record()
+    fence()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        tm = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tm.item())
+    e2e_val = n_tok * e2e_steps / (e2e_ms / 1e3)
     if world == 1:
-        for _ in range(2):
-            e2e_step()
-        fence()
-        e0.record()
-        for _ in range(e2e_steps):
-            host_loss, _ = e2e_step()
-        e1.record()
-        fence()
-        e2e_ms = e0.elapsed_time(e1)
-        e2e_val = n_tok * e2e_steps / (e2e_ms / 1e3)
         assert abs(host_loss - loss.item()) <= 1e-5 * abs(loss.item()) + 1e-7
 
     if rank != 0:
@@ -285,7 +299,8 @@ def main():
     dom = max(range(4), key=lambda k: kind_ms[k])
     achieved = flops_pass / (kind_ms[dom] / 1e3) / 1e12
     traffic = None
-    if NCU_TRAFFIC["sources_sha256"] == sources_hash() and NCU_TRAFFIC["kind"] == dom:
+    if (NCU_TRAFFIC["sources_sha256"] == sources_hash() and NCU_TRAFFIC["kind"] == dom
+            and NCU_TRAFFIC["config"] == args.config):
         traffic = NCU_TRAFFIC["bytes_per_launch"]
     roofline = {
         "bound": "tensor", "kernel": KIND_NAMES[dom], "achieved": achieved, "peak": peaks["sustained"],
@@ -317,8 +332,7 @@ def main():
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"config {args.config}: {w.name} d={w.d} V={w.V} rows={w.T} valid_tokens={w.n_valid} "
-                               f"G={w.G} eps=({w.eps_low},{w.eps_high}) beta={w.beta} ent_coef={w.ent_coef}",
+        "config": {"workload": workload_label(args.config, w),
                    "l2": "inputs larger than L2 (W alone is %.0f MB; L2 126 MB)" % (w.V * w.d * 2 / 1e6),
                    "parallelism": f"dp{world}" if world > 1 else "single GPU",
                    "masked_rows": "skipped (row compaction)"},
