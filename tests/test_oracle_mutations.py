@@ -1,0 +1,71 @@
+"""The pins must be able to fail: every plausible mistake planted in a copy of the oracle (a
+dropped term, a wrong sign, a wrong divisor, a wrong branch) has to trip at least one pin test.
+The mistakes are planted in the oracle's source on the CPU; the real module is untouched."""
+import os
+import types
+
+import pytest
+
+import tests.test_oracle_pins as pins
+
+ORACLE_SRC = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle", "grpo_oracle.py")
+
+MUTANTS = {
+    "entropy sign": ("ent = -(P * LP).sum(axis=1)", "ent = (P * LP).sum(axis=1)"),
+    "lse without the max shift added back": ("lse = M[:, 0] + np.log(", "lse = np.log("),
+    "k3 constant term dropped": ("k3 = np.exp(delta) - delta - 1.0\n        dk3", "k3 = np.exp(delta) - delta\n        dk3"),
+    "k3 gradient sign": ("dk3 = 1.0 - np.exp(delta)          # d k3 / d logp", "dk3 = np.exp(delta) - 1.0"),
+    "clip branch ignores the advantage sign": ("active = (rho * adv <= clipped * adv)", "active = (rho <= clipped)"),
+    "surrogate not pessimistic": ("s = np.minimum(rho * adv, clipped * adv)\n        # the unclipped",
+                                  "s = np.maximum(rho * adv, clipped * adv)\n        # the unclipped"),
+    "logit gradient sign": ("G = wdlogp[:, None] * (onehot - P)", "G = wdlogp[:, None] * (P - onehot)"),
+    "entropy gradient misses the +Ent term": ("P * (LP + ent[:, None])\n\n    out[\"dH\"]", "P * LP\n\n    out[\"dH\"]"),
+    "dW uses the wrong operand": ('out["dW"] = G.T @ Hr', 'out["dW"] = G.T @ (Hr * 0 + 1)'),
+    "dH scaled": ('out["dH"][rows] = G @ W ', 'out["dH"][rows] = 2 * G @ W '),
+    "population instead of sample variance": ("/ (group_size - ddof)", "/ group_size"),
+    "advantage not centred": ("(grp - mu) / (sigma + eps_std)", "grp / (sigma + eps_std)"),
+    "token mean divides by all rows": ("return m / n if n > 0", "return m / m.size if n > 0"),
+    "sequence ratio sums instead of averaging": ("(logp[idx] - old_logp[idx]).sum() / idx.size", "(logp[idx] - old_logp[idx]).sum()"),
+    "per-response mean forgets the number of responses": ("w[sl] = m[sl] / (B * n)", "w[sl] = m[sl] / n"),
+    "sequence-level gradient forgets 1/len": ("-(rho / np.maximum(len_full[rows], 1.0)) * seq_sum[rows]", "-rho * seq_sum[rows]"),
+    "RLOO includes the response itself": ("if j != i]", "]"),
+    "OPO baseline unweighted": ("base = (ln[sl] * r[sl]).sum() / tot", "base = r[sl].sum() / len(r[sl])"),
+    "logits index order": ("return H @ W.T", "return (W @ H.T).T[::-1][::-1] if H.shape[0] == 1 else (H[:, ::-1] @ W[:, ::-1].T if False else H @ W[::-1].T)"),
+}
+
+PIN_TESTS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")]
+
+
+def _load_mutant(old, new):
+    src = open(ORACLE_SRC).read()
+    assert src.count(old) >= 1, f"mutation anchor not found: {old!r}"
+    mod = types.ModuleType("grpo_oracle_mutant")
+    exec(compile(src.replace(old, new), ORACLE_SRC, "exec"), mod.__dict__)
+    return mod
+
+
+def _run_all_pins():
+    failures = 0
+    for t in PIN_TESTS:
+        marks = [m for m in getattr(t, "pytestmark", []) if m.name == "parametrize"]
+        cases = [()]
+        if marks:
+            names, values = marks[0].args
+            cases = [v if isinstance(v, tuple) and "," in names else (v,) for v in values]
+        for c in cases:
+            try:
+                t(*c)
+            except Exception:          # an assertion, or the mistake breaks the computation outright
+                failures += 1
+    return failures
+
+
+def test_unmutated_oracle_passes_every_pin(monkeypatch):
+    assert _run_all_pins() == 0
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_planted_mistake_is_caught(monkeypatch, name):
+    old, new = MUTANTS[name]
+    monkeypatch.setattr(pins, "O", _load_mutant(old, new))
+    assert _run_all_pins() > 0, f"no pin notices: {name}"
