@@ -319,6 +319,13 @@ def test_error_reporting(ctx):
     assert status_of(lambda: ctx.rl_grpo_advantages(w.rewards, 1)) == 2
     assert status_of(lambda: ctx.rl_grpo_advantages(w.rewards, 5)) == 2
     assert status_of(lambda: ctx.rl_grpo_advantages(w.rewards, 4, ddof=2, eps_std=1e-6)) == 1
+    assert status_of(lambda: ctx.rl_advantages("opo", w.rewards, 4)) == 1                         # lengths missing
+    assert status_of(lambda: ctx.rl_advantages("rloo", w.rewards, 1)) == 2
+    assert status_of(lambda: ctx.set_cta_group(3)) == 1
+    assert status_of(lambda: ctx.set_slab_limits(100, 256)) == 2
+    assert status_of(lambda: ctx.rl_policy_loss_fwd_bwd(w.H, w.W, *args, 0.2, 0.2, 0.04, agg_mode=1)) == 1  # no offsets
+    assert ctx.workspace_bytes(1024, 256, 4096) <= ctx.workspace_bytes(4096, 256, 4096) <= \
+        ctx.workspace_bytes(4096, 512, 8192, host=True)
     # no workspace bound
     c2 = Context(0)
     try:
@@ -343,6 +350,34 @@ def test_error_reporting(ctx):
     lp, _, _ = ctx.rl_token_logprobs(w.H, w.W, w.tokens, w.mask)
     _assert_status_ok(ctx)
     assert torch.isfinite(lp).all()
+
+
+def test_host_buffer_step_matches_device_call(ctx):
+    # the host-buffer entry point (pinned inputs, advantages from rewards on the device) must give
+    # exactly what the device-pointer calls give
+    from paper_2512_21450_b200.workloads import make_workload
+    for cfg_id, kw in ((0, dict(seed=91)), (4, dict(prompts=2, L_max=16, seed=92, d=256, V=5000))):
+        w = make_workload(cfg_id, **kw)
+        _, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+        ref = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask,
+                                         w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef)
+        ref = {k: v.clone() for k, v in ref.items()}
+        pin = lambda x: None if x is None else x.cpu().pin_memory()  # noqa: E731
+        dH = torch.empty_like(ref["dH"])
+        dW = torch.empty_like(ref["dW"])
+        loss, metrics = ctx.rl_policy_loss_fwd_bwd_host(
+            pin(w.H), w.W, pin(w.tokens), pin(w.old_logp), pin(w.ref_logp), None, pin(w.mask), w.eps_low,
+            w.eps_high, w.beta, w.ent_coef, dH, dW, rewards_host=pin(w.rewards), group_size=w.G,
+            seq_offsets_host=pin(w.seq_offsets))
+        _assert_status_ok(ctx)
+        assert loss == ref["loss"].item()
+        assert torch.equal(dH, ref["dH"]) and torch.equal(dW, ref["dW"])
+        assert np.allclose(metrics, ref["metrics"].cpu().numpy(), rtol=0, atol=0)
+        # per-row advantages from the host instead of rewards
+        loss2, _ = ctx.rl_policy_loss_fwd_bwd_host(
+            pin(w.H), w.W, pin(w.tokens), pin(w.old_logp), pin(w.ref_logp), pin(adv_tok), pin(w.mask), w.eps_low,
+            w.eps_high, w.beta, w.ent_coef, dH, dW)
+        assert loss2 == ref["loss"].item() and torch.equal(dW, ref["dW"])
 
 
 def test_bounded_wait_times_out_cleanly(ctx):
