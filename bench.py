@@ -27,7 +27,7 @@ KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant
 # kernel from an ncu capture, valid only for the kernel sources whose hash is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "b4ebd80b3b3fbe1c951e9b149a8919fced29ca07d862cbfb833ef67b0ac21d3d", "kind": 2, "config": 1,
+NCU_TRAFFIC = {"sources_sha256": "fe905b9a38d1e2ce7bbff1c85fd84266a1846a8d52b4dedcc50587029ab768d5", "kind": 2, "config": 1,
                "bytes_per_launch": 1416770000 + 136509440}   # profiles/gemm_kernels_config1_ncu_full.md
 
 

@@ -15,9 +15,9 @@
 //         CTA issues tcgen05.mma.cta_group::2 (M = 256) which reads both halves of B and writes
 //         128 accumulator rows into each CTA's tensor memory; both CTAs run their own epilogue.
 //         All TMA completions of a stage are counted on the even CTA's barrier; stage-free and
-//         accumulator-ready signals are multicast to both CTAs by tcgen05.commit; the odd CTA's
+//         accumulator-ready signals reach both CTAs through one tcgen05.commit; the odd CTA's
 //         epilogue reports "accumulator drained" to the even CTA with a remote mbarrier arrive.
-//         No TMA load is multicast.
+//         Every TMA load is addressed to the shared memory of the CTA that issues it.
 //
 // Either operand may be K-major (its global tensor is [rows, K], K contiguous) or MN-major
 // (its global tensor is [K, rows], rows contiguous).  A K-major tile is one 2-D TMA box
