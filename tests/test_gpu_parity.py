@@ -226,6 +226,17 @@ def test_ragged_shapes(ctx, V, L_max):
     _check_against_oracle(ctx, w)
 
 
+@pytest.mark.parametrize("d,V,L_max", [(64, 300, 16), (64, 1, 5), (128, 2, 16), (192, 777, 1), (64, 70000, 3)])
+def test_extreme_shapes(ctx, d, V, L_max):
+    # smallest hidden size the TMA layout allows, one- and two-word vocabularies (entropy 0 /
+    # gradient exactly zero for V = 1), a single row per response, a vocabulary with many slabs
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, L_max=L_max, d=d, V=V, seed=600 + V)
+    out, oo = _check_against_oracle(ctx, w)
+    if V == 1:
+        assert not out["dH"].any() and not out["dW"].any() and not out["logp"].any()
+
+
 def test_multiple_slabs(ctx):
     # force several row slabs and several vocabulary slabs on a small case
     from paper_2512_21450_b200 import Context
