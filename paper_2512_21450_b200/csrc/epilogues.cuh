@@ -23,6 +23,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // range of the work unit, keeps the running maximum M, S = sum exp(z-M), A = sum exp(z-M) z and
 // the logit of the sampled token.  Logits never leave the chip; one float4 per (range, row) does.
 struct EpiStats {
+  static constexpr int kStagingBytes = 0;
   struct Params {
     const int* tokens_c;   // [rows] compact sampled-token ids
     float4* partials;      // [n_ranges][part_stride]
@@ -34,7 +35,7 @@ struct EpiStats {
     int y;
   };
   __device__ static __forceinline__ void begin_unit(const Params& p, State& st, int m_tile, int, int row_in_tile,
-                                                    int m_rows, int) {
+                                                    int m_rows, int, int) {
     st.m = -CUDART_INF_F;
     st.s = 0.f;
     st.a = 0.f;
@@ -42,8 +43,10 @@ struct EpiStats {
     const int row = m_tile * BM + row_in_tile;
     st.y = row < m_rows ? p.tokens_c[row] : -1;
   }
+  __device__ static __forceinline__ void init(State&) {}
+  __device__ static __forceinline__ void finish(State&) {}
   __device__ static __forceinline__ void chunk(const Params& p, State& st, int, int n_tile, int c, int, int,
-                                               const float (&v)[32]) {
+                                               const float (&v)[32], const CUtensorMap*, uint32_t) {
     const int col0 = n_tile * BN + c * 32;
     const int nvalid = p.V - col0;
     if (nvalid <= 0) return;
@@ -106,6 +109,7 @@ struct EpiStats {
 // cp_t = -w_t dloss_t/dlogp_t and ce_t = w_t ent_coef come from the per-token loss kernel.
 // Rows past the valid rows of the slab and columns past V are written as zero.
 struct EpiGrad {
+  static constexpr int kStagingBytes = 0;
   struct Params {
     const int* tokens_c;
     const float* lse;
@@ -123,7 +127,7 @@ struct EpiGrad {
     bool valid;
   };
   __device__ static __forceinline__ void begin_unit(const Params& p, State& st, int m_tile, int, int row_in_tile,
-                                                    int m_rows, int slab_off) {
+                                                    int m_rows, int slab_off, int) {
     const int rl = m_tile * BM + row_in_tile;
     st.valid = rl < m_rows;
     const int gr = slab_off + rl;   // compact row of this slab row
@@ -133,8 +137,11 @@ struct EpiGrad {
     st.ce = st.valid ? p.ce[gr] : 0.f;
     st.y = st.valid ? p.tokens_c[gr] : -1;
   }
+  __device__ static __forceinline__ void init(State&) {}
+  __device__ static __forceinline__ void finish(State&) {}
   __device__ static __forceinline__ void chunk(const Params& p, State& st, int m_tile, int n_tile, int c,
-                                               int row_in_tile, int m_rows, const float (&v)[32]) {
+                                               int row_in_tile, int m_rows, const float (&v)[32], const CUtensorMap*,
+                                               uint32_t) {
     // a CTA pair may own a 128-row tile that lies wholly past the slab's rows: nothing to write
     if (m_tile * BM >= ((m_rows + BM - 1) / BM) * BM) return;
     const int col_l = n_tile * BN + c * 32;
@@ -193,34 +200,58 @@ struct EpiGrad {
 };
 
 // ---------------------------------------------------------------------------------------------
-// Plain fp32 output tile: C[row_base + row, col] = acc (+ previous value when accumulating).
+// Plain fp32 output tile: C[slice][row_base + row, col] = acc (+ previous value when accumulating).
+// Each epilogue warp stages its 32x32 chunk in shared memory (128-byte swizzled, two buffers) and
+// one lane hands it to the TMA unit: a bulk tensor store, or a bulk tensor reduce-add when
+// accumulating.  The output is seen through a 3-D fp32 tensor map {columns, rows, K slices}, which
+// also clips rows past the tensor.  Every element is written by exactly one tile per launch, so
+// the result does not depend on timing.
 struct EpiAcc {
+  static constexpr int kStagingBytes = 4 * kStagingPerWarp;
   struct Params {
-    float* C;
-    long long ldc;
     int n_cols;
     int accumulate;
     int row_base;
   };
-  struct State {};
-  __device__ static __forceinline__ void begin_unit(const Params&, State&, int, int, int, int, int) {}
-  __device__ static __forceinline__ void chunk(const Params& p, State&, int m_tile, int n_tile, int c,
-                                               int row_in_tile, int m_rows, const float (&v)[32]) {
-    const int rl = m_tile * BM + row_in_tile;
+  struct State {
+    int k_slice;
+    uint32_t n_issued;   // chunks handed to the TMA unit so far (selects the staging buffer)
+  };
+  __device__ static __forceinline__ void init(State& st) { st.n_issued = 0; }
+  __device__ static __forceinline__ void finish(State& st) {
+    if ((threadIdx.x & 31) == 0 && st.n_issued) bulk_wait_group_all();
+    __syncwarp();
+  }
+  __device__ static __forceinline__ void begin_unit(const Params&, State& st, int, int, int, int, int, int k_slice) {
+    st.k_slice = k_slice;
+  }
+  __device__ static __forceinline__ void chunk(const Params& p, State& st, int m_tile, int n_tile, int c,
+                                               int row_in_tile, int m_rows, const float (&v)[32],
+                                               const CUtensorMap* tmC, uint32_t staging) {
+    const int lane = threadIdx.x & 31;
+    const int row0 = m_tile * BM + (row_in_tile - lane);   // first row of this warp's 32
     const int col0 = n_tile * BN + c * 32;
-    if (rl >= m_rows || col0 >= p.n_cols) return;
-    float4* dst = reinterpret_cast<float4*>(p.C + (size_t)(p.row_base + rl) * p.ldc + col0);
+    if (row0 >= m_rows || col0 >= p.n_cols) return;        // warp-uniform
+    const uint32_t buf = staging + (st.n_issued & 1u) * 4096u;
+    // the store issued from this buffer two chunks ago must have finished reading it
+    if (lane == 0) bulk_wait_group_read<1>();
+    __syncwarp();
+    // row `lane` of the box: 8 chunks of 16 bytes, chunk j stored at position j ^ (row & 7)
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      if (col0 + 4 * j < p.n_cols) {
-        float4 x = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-        if (p.accumulate) {
-          const float4 o = __ldcs(dst + j);
-          x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w;
-        }
-        __stcs(dst + j, x);   // each element is touched once per launch
-      }
+      const uint32_t addr = buf + lane * 128u + (uint32_t((j ^ (lane & 7)) << 4));
+      asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v[4 * j]), "f"(v[4 * j + 1]),
+                   "f"(v[4 * j + 2]), "f"(v[4 * j + 3])
+                   : "memory");
     }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      if (p.accumulate) tma_reduce_add_3d(tmC, buf, col0, p.row_base + row0, st.k_slice);
+      else              tma_store_3d(tmC, buf, col0, p.row_base + row0, st.k_slice);
+      bulk_commit_group();
+    }
+    st.n_issued++;
   }
   __device__ static __forceinline__ void end_unit(const Params&, State&, int, int, int, int) {}
 };

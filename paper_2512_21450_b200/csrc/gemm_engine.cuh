@@ -38,18 +38,21 @@ constexpr int BN = 256;   // accumulator columns
 constexpr int BK = 64;
 constexpr int kAStageBytes = BM * BK * 2;
 constexpr int kGemmThreads = 192;
-constexpr int kRingBytes = 224 * 1024;             // shared-memory ring of operand stages
-constexpr int kGemmSmemBytes = kRingBytes + 1024;  // + slack for 1024-byte alignment
+constexpr int kTileSmemBytes = 224 * 1024;             // operand ring + epilogue staging
+constexpr int kGemmSmemBytes = kTileSmemBytes + 1024;  // + slack for 1024-byte alignment
+constexpr int kStagingPerWarp = 8192;                  // two 32x32 fp32 boxes per epilogue warp
 constexpr int kTmemCols = 512;
 constexpr int kMaxSplit = 16;   // most column ranges per row tile when the split is chosen to fill the machine
 constexpr int kFwdRange = 8;    // column tiles per work unit when there is plenty of work
 
-template <int CG>
+// kStaging: bytes of shared memory the epilogue keeps for itself behind the ring.
+template <int CG, int kStaging>
 struct StageCfg {
   static constexpr int kBRows = BN / CG;                    // B rows (output columns) staged per CTA
   static constexpr int kBBytes = kBRows * BK * 2;
   static constexpr int kStageBytes = kAStageBytes + kBBytes;
-  static constexpr int kStages = kRingBytes / kStageBytes;  // 4 (CG = 1) or 7 (CG = 2)
+  static constexpr int kRingBytes = (kTileSmemBytes - kStaging) / kStageBytes * kStageBytes;
+  static constexpr int kStages = kRingBytes / kStageBytes;  // 4 (CG = 1); 7 or 6 (CG = 2)
   static constexpr uint32_t kTxBytes = uint32_t(kStageBytes) * CG;  // bytes counted on the issuing CTA's barrier
 };
 constexpr int kMaxStages = 7;
@@ -83,6 +86,10 @@ struct GemmShape {
   // launch works on slab slab_index: its row offset replaces m_dyn_off / k_dyn_off, and is added
   // to the A row coordinate (a_mn_slab) or the B k coordinate (b_k_slab).
   int slab_cap, slab_index, a_mn_slab, b_k_slab;
+  // K split: when k_split_max > 1 every output tile may be cut into up to k_split_max slices of
+  // the K range, each a work unit of its own that adds into its own output buffer (the epilogue
+  // gets the slice index); the slice count is chosen on the device to even out the last wave.
+  int k_split_max;
   // coordinate offsets into the operands' global tensors
   int a_mn_off, a_k_off, b_mn_off, b_k_off;
 };
@@ -103,8 +110,21 @@ __host__ __device__ inline int choose_split(int m_units, int n_tiles, int n_work
 }
 
 struct GemmExtents {
-  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units, slab_off;
+  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units, slab_off, k_split, kb_per;
 };
+
+// Number of K slices per tile (1..smax) that minimises the number of waves the tiles take on
+// n_workers workers, charging about 1 % per extra slice for the extra output traffic.
+__host__ __device__ inline int choose_k_split(long tiles, int n_workers, int smax) {
+  int best = 1;
+  long best_cost = -1;
+  for (int sp = 1; sp <= smax && sp <= 4; ++sp) {
+    const long waves = (tiles * sp + n_workers - 1) / n_workers;
+    const long cost = waves * (12 / sp) * (100 + sp - 1);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = sp; }
+  }
+  return best;
+}
 
 // Offset and row count of slab `index` when n_valid rows are cut into equal slabs of at most cap rows.
 __host__ __device__ inline void slab_extent(int n_valid, int cap, int index, int& off, int& rows) {
@@ -148,26 +168,39 @@ __host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_v
   if (e.n_range < 1) e.n_range = 1;
   e.n_ranges = (sh.n_tiles + e.n_range - 1) / e.n_range;
   e.n_units = e.m_units * e.n_ranges;
+  e.k_split = sh.k_split_max > 1 ? choose_k_split((long)e.n_units, n_workers, sh.k_split_max) : 1;
+  e.kb_per = (e.k_blocks + e.k_split - 1) / e.k_split;
+  e.n_units *= e.k_split;
   if (sh.skip_if_k0 && e.k_blocks == 0) e.n_units = 0;
   return e;
 }
 
-__device__ __forceinline__ void unit_coords(const GemmShape& sh, const GemmExtents& ex, int u, int& mu, int& nr) {
+// Unit u -> row tile mu, column range nr and the K-block range [kb0, kb1) of its K slice ks.
+__device__ __forceinline__ void unit_coords(const GemmShape& sh, const GemmExtents& ex, int u, int& mu, int& nr,
+                                            int& ks, int& kb0, int& kb1) {
+  ks = u % ex.k_split;
+  u /= ex.k_split;
+  kb0 = ks * ex.kb_per;
+  kb1 = min(kb0 + ex.kb_per, ex.k_blocks);
   if (sh.n_fastest) { nr = u % ex.n_ranges; mu = u / ex.n_ranges; }
   else              { mu = u % ex.m_units;  nr = u / ex.m_units; }
 }
 
 // Epilogue functor contract (all methods run in the 128 epilogue threads, one tile row each):
 //   struct Epi { struct Params; struct State;
-//     static void begin_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows, int slab_off);
+//     static void begin_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows, int slab_off, int k_slice);
 //     static void chunk(const Params&, State&, int m_tile, int n_tile, int chunk, int row_in_tile, int m_rows, const float (&v)[32]);
-//     static void end_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows); };
+//     static void end_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows);
+//     static void init(State&); static void finish(State&);     // once per kernel, per thread
+//     static constexpr int kStagingBytes;                      // shared memory behind the ring (0 or 32 KB) };
+//   chunk additionally receives the output tensor map and the warp's staging address.
 // m_tile counts 128-row tiles.
 template <class Epi, int A_MN, int B_MN, int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const GemmShape sh, const typename Epi::Params ep, DevStatus* status) {
-  using Cfg = StageCfg<CG>;
+            const __grid_constant__ CUtensorMap tmC, const GemmShape sh, const typename Epi::Params ep,
+            DevStatus* status) {
+  using Cfg = StageCfg<CG, Epi::kStagingBytes>;
   constexpr int kStages = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kMaxStages];
@@ -214,12 +247,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t phase = 0;
       bool ok = true;
       for (int u = worker; u < ex.n_units && ok; u += n_workers) {
-        int mu, nr;
-        unit_coords(sh, ex, u, mu, nr);
+        int mu, nr, ks, kb0, kb1;
+        unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
         const int m = mu * CG + (int)rank;
         const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
         for (int n = n0; n < n1 && ok; ++n) {
-          for (int kb = 0; kb < ex.k_blocks; ++kb) {
+          for (int kb = kb0; kb < kb1; ++kb) {
             if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p)) {
               latch_status(status, kStatusTimeout, (1 << 28) | (blockIdx.x << 8) | stage);
               ok = false;
@@ -274,8 +307,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       bool ok = true;
       if (ex.k_blocks > 0) {
         for (int u = worker; u < ex.n_units && ok; u += n_workers) {
-          int mu, nr;
-          unit_coords(sh, ex, u, mu, nr);
+          int mu, nr, ks, kb0, kb1;
+          unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
+          if (kb1 <= kb0) continue;   // empty K slice: the epilogue handles it without an accumulator
           const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
           for (int n = n0; n < n1 && ok; ++n, ++t) {
             const uint32_t a = t & 1u, round = t >> 1;
@@ -286,7 +320,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + a * BN;
-            for (int kb = 0; kb < ex.k_blocks; ++kb) {
+            for (int kb = kb0; kb < kb1; ++kb) {
               if (!mbar_wait_bounded_cluster(smem_u32(&bar_full[stage]), phase, abort_p)) {
                 latch_status(status, kStatusTimeout, (3 << 28) | (blockIdx.x << 8) | stage);
                 ok = false;
@@ -298,8 +332,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
               for (int k = 0; k < BK / 16; ++k) {
                 const uint64_t da = smem_desc(a_hi, a_src + k * a_kstep), db = smem_desc(b_hi, b_src + k * b_kstep);
-                if (CG == 2) umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
-                else         umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                if (CG == 2) umma_bf16_pair(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                else         umma_bf16(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
               }
               if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_empty[stage]), 3);
               else         umma_commit(smem_u32(&bar_empty[stage]));
@@ -323,18 +357,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------- epilogue warps (both CTAs)
     const int q = warp & 3;
     const int row_in_tile = q * 32 + lane;
+    const uint32_t staging = tiles_base + Cfg::kRingBytes + q * kStagingPerWarp;   // this warp's epilogue staging
     typename Epi::State st;
+    Epi::init(st);
     uint32_t t = 0;
     bool ok = true;
     for (int u = worker; u < ex.n_units && ok; u += n_workers) {
-      int mu, nr;
-      unit_coords(sh, ex, u, mu, nr);
+      int mu, nr, ks, kb0, kb1;
+      unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
+      const bool has_k = kb1 > kb0;   // an empty K slice contributes zeros
       const int m = mu * CG + (int)rank;
       const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
-      Epi::begin_unit(ep, st, m, nr, row_in_tile, ex.m_rows, ex.slab_off);
-      for (int n = n0; n < n1 && ok; ++n, ++t) {
+      Epi::begin_unit(ep, st, m, nr, row_in_tile, ex.m_rows, ex.slab_off, ks);
+      for (int n = n0; n < n1 && ok; ++n, t += has_k ? 1u : 0u) {
         const uint32_t a = t & 1u, round = t >> 1;
-        if (ex.k_blocks > 0) {
+        if (has_k) {
           if (!mbar_wait_bounded_cluster(smem_u32(&bar_acc_full[a]), round & 1u, abort_p)) {
             latch_status(status, kStatusTimeout, (5 << 28) | (blockIdx.x << 8) | a);
             ok = false;
@@ -347,7 +384,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           float v[32];
-          if (ex.k_blocks > 0) {
+          if (has_k) {
             uint32_t r[32];
             tmem_ld_32x32(taddr + c * 32, r);
             tmem_ld_wait();
@@ -357,9 +394,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0.f;
           }
-          Epi::chunk(ep, st, m, n, c, row_in_tile, ex.m_rows, v);
+          Epi::chunk(ep, st, m, n, c, row_in_tile, ex.m_rows, v, &tmC, staging);
         }
-        if (ex.k_blocks > 0) {
+        if (has_k) {
           tc_fence_before();
           __syncwarp();
           if (lane == 0) {
@@ -370,6 +407,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       if (ok) Epi::end_unit(ep, st, m, nr, row_in_tile, ex.m_rows);
     }
+    Epi::finish(st);   // e.g. wait for bulk stores that still read this warp's staging memory
   }
 
   tc_fence_before();

@@ -122,6 +122,19 @@ bool map_mnmajor(rl_ctx* c, CUtensorMap* m, const void* base, uint64_t k_rows, u
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 output seen by the accumulate epilogue: {cols, rows, slices} with 32x32 boxes, 128-byte
+// swizzled in shared memory.  slices > 1: identical [rows, ld] buffers slice_rows rows apart.
+bool map_out_f32(rl_ctx* c, CUtensorMap* m, const float* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                 uint64_t slices, uint64_t slice_rows) {
+  cuuint64_t dims[3] = {cols, rows, slices};
+  cuuint64_t strides[2] = {ld * 4, slice_rows * ld * 4};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return c->encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <class Epi, int A_MN, int B_MN>
 cudaError_t set_smem_attr() {
   cudaError_t e = cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -153,8 +166,8 @@ void prof_end(rl_ctx* c, int i, int kind) {
 }
 
 template <class Epi, int A_MN, int B_MN>
-void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const GemmShape& sh,
-                 const typename Epi::Params& ep) {
+void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& out,
+                 const GemmShape& sh, const typename Epi::Params& ep) {
   const int prof = prof_begin(c, kind);
   if (c->cta_group == 2) {
     cudaLaunchConfig_t cfg;
@@ -170,9 +183,9 @@ void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, gemm_kernel<Epi, A_MN, B_MN, 2>, a, b, sh, ep, c->dstatus);
+    cudaLaunchKernelEx(&cfg, gemm_kernel<Epi, A_MN, B_MN, 2>, a, b, out, sh, ep, c->dstatus);
   } else {
-    gemm_kernel<Epi, A_MN, B_MN, 1><<<c->grid[1], kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, sh, ep,
+    gemm_kernel<Epi, A_MN, B_MN, 1><<<c->grid[1], kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, out, sh, ep,
                                                                                             c->dstatus);
   }
   c->launches++;
@@ -235,7 +248,7 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   ep.partials = reinterpret_cast<float4*>(ws + L.partials);
   ep.part_stride = L.Tpad;
   ep.V = (int)V;
-  launch_gemm<EpiStats, 0, 0>(c, 0, tmA, tmB, sh, ep);
+  launch_gemm<EpiStats, 0, 0>(c, 0, tmA, tmB, tmA, sh, ep);   // no output map
   *shape_out = sh;
   return cuda_ok();
 }
@@ -634,13 +647,15 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   const int* row_map = reinterpret_cast<const int*>(ws + L.row_map);
   const int* n_valid = &c->dstatus->n_valid;
 
-  CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn;
+  CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn, tm_dH, tm_dW;
   bool ok = map_kmajor(c, &tmHc_k, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM) &&
             map_kmajor(c, &tmW_k, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_rows(c)) &&
             map_kmajor(c, &tmG_k, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM) &&
             map_mnmajor(c, &tmW_mn, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_panels(c)) &&
             map_mnmajor(c, &tmG_mn, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM / 64) &&
-            map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, b_box_panels(c));
+            map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, b_box_panels(c)) &&
+            map_out_f32(c, &tm_dH, dH_acc, (uint64_t)L.Ts, (uint64_t)d, (uint64_t)d, 1, (uint64_t)L.Ts) &&
+            map_out_f32(c, &tm_dW, dW, (uint64_t)V, (uint64_t)d, (uint64_t)d, 1, (uint64_t)V);
   if (!ok) return RL_ERR_CUDA;
 
   const int n_row_slabs = (L.Tpad + L.Ts - 1) / L.Ts;
@@ -666,7 +681,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
         ep.lse = p.lse_c; ep.ent = p.ent_c; ep.cp = p.cp_c; ep.ce = p.ce_c;
         ep.G = G; ep.ldG = L.Vs; ep.V = (int)V; ep.vocab_base = vocab_base;
-        launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, sh, ep);
+        launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, tmHc_k, sh, ep);   // no output map
       }
       // (2) dH_slab (+)= G * W_slab        [rows x d], K = vocabulary columns of the slab
       {
@@ -680,8 +695,8 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         sh.b_k_off = vocab_base;
         sh.n_fastest = 1;   // the CTAs that share a panel of G rows run together
         EpiAcc::Params ep;
-        ep.C = dH_acc; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0;
-        launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, sh, ep);
+        ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0;
+        launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, tm_dH, sh, ep);
       }
       // (3) dW_slab (+)= G^T * H_slab      [vocabulary rows x d], K = valid rows of the slab
       {
@@ -696,9 +711,9 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         sh.b_k_slab = 1;
         sh.n_fastest = 1;
         EpiAcc::Params ep;
-        ep.C = dW; ep.ldc = d; ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
+        ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
         ep.row_base = vocab_base;
-        launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, sh, ep);
+        launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, tm_dW, sh, ep);
       }
     }
     const int pr_sc = prof_begin(c, 7);
@@ -806,12 +821,14 @@ rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, in
   sh.k_cap = (int)K;
   sh.n_tiles = (int)(N / BN);
   sh.n_range = 1;
+  CUtensorMap tc;
+  if (!map_out_f32(c, &tc, C, (uint64_t)M, (uint64_t)N, (uint64_t)N, 1, (uint64_t)M)) return RL_ERR_CUDA;
   EpiAcc::Params ep;
-  ep.C = C; ep.ldc = N; ep.n_cols = (int)N; ep.accumulate = accumulate; ep.row_base = 0;
-  if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, -1, ta, tb, sh, ep);
-  else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, -1, ta, tb, sh, ep);
-  else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, -1, ta, tb, sh, ep);
-  else launch_gemm<EpiAcc, 1, 1>(c, -1, ta, tb, sh, ep);
+  ep.n_cols = (int)N; ep.accumulate = accumulate; ep.row_base = 0;
+  if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, -1, ta, tb, tc, sh, ep);
+  else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, -1, ta, tb, tc, sh, ep);
+  else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, -1, ta, tb, tc, sh, ep);
+  else launch_gemm<EpiAcc, 1, 1>(c, -1, ta, tb, tc, sh, ep);
   return cuda_ok();
 }
 
