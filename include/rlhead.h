@@ -73,6 +73,13 @@ rl_status rl_set_slab_limits(rl_ctx* ctx, int max_rows, int max_cols);
  * and L2 traffic of the B operand.  2 is the default when the device can co-schedule CTA pairs;
  * asking for 2 when it cannot returns RL_ERR_UNSUPPORTED_ARCH.  Results are identical up to fp32 summation order inside the tensor core. */
 rl_status rl_set_cta_group(rl_ctx* ctx, int cta_group);
+/* Upper bound (1..4, default 1) on the number of slices the K range of a dH tile may be cut
+ * into.  With more than one slice the dH pass picks, on the device, the slice count that evens
+ * out its last wave of tiles; every slice accumulates into its own fp32 buffer and the buffers
+ * are summed in slice order when dH is written, so results stay reproducible.  Costs
+ * (max_slices - 1) extra [slab rows x d] fp32 buffers of workspace: call before
+ * rl_workspace_bytes().  On the measured workloads the gain was within 1 %. */
+rl_status rl_set_dh_k_slices(rl_ctx* ctx, int max_slices);
 /* Caller-owned device scratch, 256-byte aligned; must outlive the calls that use it. */
 rl_status rl_set_workspace(rl_ctx* ctx, void* dev_ptr, size_t bytes);
 

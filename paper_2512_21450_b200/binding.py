@@ -66,6 +66,8 @@ def load_library():
     lib.rl_workspace_bytes_host.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
     lib.rl_set_workspace.argtypes = [P, P, c_size_t]
     lib.rl_set_slab_limits.argtypes = [P, c_int, c_int]
+    lib.rl_set_dh_k_slices.argtypes = [P, c_int]
+    lib.rl_set_dh_k_slices.restype = c_int
     lib.rl_set_cta_group.argtypes = [P, c_int]
     lib.rl_set_cta_group.restype = c_int
     lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
@@ -151,6 +153,9 @@ class Context:
 
     def set_slab_limits(self, max_rows=0, max_cols=0):
         _check(self.lib.rl_set_slab_limits(self.handle, max_rows, max_cols), "rl_set_slab_limits")
+
+    def set_dh_k_slices(self, max_slices):
+        _check(self.lib.rl_set_dh_k_slices(self.handle, max_slices), "rl_set_dh_k_slices")
 
     def set_cta_group(self, cta_group):
         _check(self.lib.rl_set_cta_group(self.handle, cta_group), "rl_set_cta_group")

@@ -33,6 +33,7 @@ struct rl_ctx {
   int slab_rows;  // rows of one gradient slab (multiple of 128)
   int slab_cols;  // vocabulary columns of one gradient slab (multiple of 256)
   int cta_group;  // 1: one CTA per 128x256 tile; 2: CTA pairs on 256x256 tiles
+  int dh_k_slices;  // upper bound on the K slices of the dH pass (1 = tiles are not cut)
   int grid[3];    // persistent grid for cta_group 1 and 2 (index = cta_group)
   long long launches;  // kernels launched by this context so far
   // optional per-kernel timing: event pairs around every tensor-core launch, by kernel kind
@@ -45,6 +46,7 @@ struct rl_ctx {
 namespace {
 
 constexpr int kSlabRowsMax = 32768;        // rows of one gradient slab
+constexpr int kDhSplitMax = 4;             // most K slices (separate fp32 accumulators) of the dH pass
 constexpr int kSlabColsMax = 148 * 128;    // vocabulary columns of one gradient slab (74 tiles of 256)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -80,7 +82,7 @@ WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_s
   L.block_sums = take((size_t)1024 * kLossSums * sizeof(double));
   L.Hc = take((size_t)L.Tpad * d * 2);
   L.G = take((size_t)L.Ts * L.Vs * 2);
-  L.dH_acc = take((size_t)L.Ts * d * 4);
+  L.dH_acc = take((size_t)c->dh_k_slices * L.Ts * d * 4);
   L.staging = o;
   if (host_staging) {
     take((size_t)T * d * 2);  // H
@@ -289,6 +291,7 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->slab_rows = kSlabRowsMax;
   c->slab_cols = kSlabColsMax;
   c->cta_group = 1;
+  c->dh_k_slices = 1;
   c->grid[0] = 0;
   c->grid[1] = c->n_sm;
   c->grid[2] = c->n_sm / 2 * 2;
@@ -373,6 +376,13 @@ rl_status rl_set_cta_group(rl_ctx* c, int cta_group) {
   if (cta_group != 1 && cta_group != 2) return RL_ERR_INVALID_ARG;
   if (cta_group == 2 && c->grid[2] < 2) return RL_ERR_UNSUPPORTED_ARCH;
   c->cta_group = cta_group;
+  return RL_OK;
+}
+
+rl_status rl_set_dh_k_slices(rl_ctx* c, int max_slices) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  if (max_slices < 1 || max_slices > kDhSplitMax) return RL_ERR_INVALID_ARG;
+  c->dh_k_slices = max_slices;
   return RL_OK;
 }
 
@@ -654,7 +664,7 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
             map_mnmajor(c, &tmW_mn, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_panels(c)) &&
             map_mnmajor(c, &tmG_mn, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM / 64) &&
             map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, b_box_panels(c)) &&
-            map_out_f32(c, &tm_dH, dH_acc, (uint64_t)L.Ts, (uint64_t)d, (uint64_t)d, 1, (uint64_t)L.Ts) &&
+            map_out_f32(c, &tm_dH, dH_acc, (uint64_t)L.Ts, (uint64_t)d, (uint64_t)d, (uint64_t)c->dh_k_slices, (uint64_t)L.Ts) &&
             map_out_f32(c, &tm_dW, dW, (uint64_t)V, (uint64_t)d, (uint64_t)d, 1, (uint64_t)V);
   if (!ok) return RL_ERR_CUDA;
 
@@ -662,6 +672,8 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   const int n_col_slabs = (int)((V + L.Vs - 1) / L.Vs);
   const int d_tiles = (int)((d + BN - 1) / BN);
   for (int r = 0; r < n_row_slabs; ++r) {
+    GemmShape dh_shape;
+    memset(&dh_shape, 0, sizeof(dh_shape));
     const int rows_cap = L.Ts;   // the valid rows are cut into equal slabs of at most Ts rows on the device
     for (int cs = 0; cs < n_col_slabs; ++cs) {
       const int vocab_base = cs * L.Vs;
@@ -694,6 +706,8 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         sh.n_range = 1;
         sh.b_k_off = vocab_base;
         sh.n_fastest = 1;   // the CTAs that share a panel of G rows run together
+        sh.k_split_max = c->dh_k_slices;
+        dh_shape = sh;      // the slice count depends only on rows, d tiles and grid: same for every slab
         EpiAcc::Params ep;
         ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0;
         launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, tm_dH, sh, ep);
@@ -718,10 +732,12 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
     }
     const int pr_sc = prof_begin(c, 7);
     if (o.dH_dtype)
-      scatter_dH_f32_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, r, L.Ts, row_map,
+      scatter_dH_f32_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, dh_shape, c->cta_group,
+                                                         c->grid[c->cta_group] / c->cta_group, (long long)L.Ts * d, row_map,
                                                          static_cast<float*>(dH), c->dstatus);
     else
-      scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, r, L.Ts, row_map,
+      scatter_dH_kernel<<<c->n_sm * 4, 256, 0, st>>>(dH_acc, (int)d, dh_shape, c->cta_group,
+                                                     c->grid[c->cta_group] / c->cta_group, (long long)L.Ts * d, row_map,
                                                      static_cast<__nv_bfloat16*>(dH), c->dstatus);
     prof_end(c, pr_sc, 7);
     c->launches++;
@@ -886,6 +902,7 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
     c.slab_rows = kSlabRowsMax;
     c.slab_cols = kSlabColsMax;
     c.cta_group = 1;
+    c.dh_k_slices = 1;
     c.grid[1] = c.n_sm;
     slot.ready = true;
   }

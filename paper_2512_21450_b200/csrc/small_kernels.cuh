@@ -522,33 +522,48 @@ __global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restr
 // ------------------------------------------------------------------------------------------
 // dH of one row slab: fp32 accumulator rows -> bf16 rows of the caller's dH at their original
 // positions.  One warp per row.
+// The dH pass may have cut K into slices that accumulate in separate buffers, split_stride
+// elements apart (same slice count as gemm_extents chose for the pass): summed here in slice order.
+__device__ __forceinline__ float4 sum_k_slices(const float4* p, int n_slices, long long split_stride) {
+  float4 x = __ldcs(p);
+  for (int s = 1; s < n_slices; ++s) {
+    const float4 y = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + s * split_stride));
+    x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+  }
+  return x;
+}
+
 // Same with an fp32 destination.
-__global__ void __launch_bounds__(256) scatter_dH_f32_kernel(const float* __restrict__ acc, int d, int slab_index,
-                                                             int slab_cap, const int* __restrict__ row_map,
+__global__ void __launch_bounds__(256) scatter_dH_f32_kernel(const float* __restrict__ acc, int d, const GemmShape dh_shape,
+                                                             int dh_cg, int dh_workers, long long split_stride,
+                                                             const int* __restrict__ row_map,
                                                              float* __restrict__ dH, const DevStatus* st) {
   int slab_base, rows;
-  slab_extent(st->n_valid, slab_cap, slab_index, slab_base, rows);
+  slab_extent(st->n_valid, dh_shape.slab_cap, dh_shape.slab_index, slab_base, rows);
+  const int n_slices = gemm_extents(dh_shape, st->n_valid, dh_cg, dh_workers).k_split;
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
     const float4* src = reinterpret_cast<const float4*>(acc + (size_t)i * d);
     float4* dst = reinterpret_cast<float4*>(dH + (size_t)row_map[slab_base + i] * d);
-    for (int v = lane; v < d / 4; v += 32) dst[v] = src[v];
+    for (int v = lane; v < d / 4; v += 32) dst[v] = sum_k_slices(src + v, n_slices, split_stride);
   }
 }
 
-__global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict__ acc, int d, int slab_index,
-                                                         int slab_cap, const int* __restrict__ row_map,
+__global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict__ acc, int d, const GemmShape dh_shape,
+                                                         int dh_cg, int dh_workers, long long split_stride,
+                                                         const int* __restrict__ row_map,
                                                          __nv_bfloat16* __restrict__ dH, const DevStatus* st) {
   int slab_base, rows;
-  slab_extent(st->n_valid, slab_cap, slab_index, slab_base, rows);
+  slab_extent(st->n_valid, dh_shape.slab_cap, dh_shape.slab_index, slab_base, rows);
+  const int n_slices = gemm_extents(dh_shape, st->n_valid, dh_cg, dh_workers).k_split;
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
     const float4* src = reinterpret_cast<const float4*>(acc + (size_t)i * d);
     uint2* dst = reinterpret_cast<uint2*>(dH + (size_t)row_map[slab_base + i] * d);
     for (int v = lane; v < d / 4; v += 32) {
-      const float4 x = src[v];
+      const float4 x = sum_k_slices(src + v, n_slices, split_stride);
       __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
       uint2 o;
       o.x = *reinterpret_cast<uint32_t*>(&lo);

@@ -251,6 +251,25 @@ def test_multiple_slabs(ctx):
         c2.close()
 
 
+@pytest.mark.parametrize("slices", [2, 3, 4])
+def test_dh_k_slices(slices):
+    # dH tiles cut along K into separately accumulated slices: same result, several slabs and CTA shapes
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    c2 = Context(0)
+    try:
+        c2.set_dh_k_slices(slices)
+        c2.set_slab_limits(256, 512)
+        _check_against_oracle(c2, make_workload(1, prompts=1, L_max=64, d=256, V=1500, seed=19 + slices))
+        c2.set_slab_limits(0, 0)
+        _check_against_oracle(c2, make_workload(0, L_max=13, V=4100, seed=29 + slices))     # a 1-block K range
+        if slices == 3:
+            c2.set_cta_group(1)
+            _check_against_oracle(c2, make_workload(1, prompts=1, L_max=40, seed=39))
+    finally:
+        c2.close()
+
+
 def test_token_weight_accumulate_and_strides(ctx):
     from paper_2512_21450_b200.workloads import make_workload
     w = make_workload(0, seed=31)
