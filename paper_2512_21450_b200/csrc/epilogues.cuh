@@ -104,20 +104,20 @@ struct EpiStats {
 
 // ---------------------------------------------------------------------------------------------
 // Gradient with respect to the logits for one slab of rows x vocabulary columns, rounded to
-// bf16 and written to the slab scratch (row-major, ldG):
+// bf16 and written to the slab scratch (row-major) by bulk tensor stores: each epilogue warp packs
+// two consecutive 32-column chunks of its 32 rows into a 128-byte-swizzled 32x64 bf16 box in
+// shared memory (two boxes per warp) and one lane hands the box to the TMA unit:
 //   g_tj = cp_t (p_tj - 1[j = y_t]) + ce_t p_tj (log p_tj + Ent_t),  p_tj = exp(z_tj - lse_t)
 // cp_t = -w_t dloss_t/dlogp_t and ce_t = w_t ent_coef come from the per-token loss kernel.
 // Rows past the valid rows of the slab and columns past V are written as zero.
 struct EpiGrad {
-  static constexpr int kStagingBytes = 0;
+  static constexpr int kStagingBytes = 4 * kStagingPerWarp;
   struct Params {
     const int* tokens_c;
     const float* lse;
     const float* ent;
     const float* cp;
     const float* ce;
-    __nv_bfloat16* G;
-    int ldG;
     int V;
     int vocab_base;  // global column of the slab's column 0
   };
@@ -125,6 +125,7 @@ struct EpiGrad {
     float lse, ent, cp, ce;
     int y;
     bool valid;
+    uint32_t n_issued;   // boxes handed to the TMA unit so far (selects the staging buffer)
   };
   __device__ static __forceinline__ void begin_unit(const Params& p, State& st, int m_tile, int, int row_in_tile,
                                                     int m_rows, int slab_off, int) {
@@ -137,11 +138,14 @@ struct EpiGrad {
     st.ce = st.valid ? p.ce[gr] : 0.f;
     st.y = st.valid ? p.tokens_c[gr] : -1;
   }
-  __device__ static __forceinline__ void init(State&) {}
-  __device__ static __forceinline__ void finish(State&) {}
+  __device__ static __forceinline__ void init(State& st) { st.n_issued = 0; }
+  __device__ static __forceinline__ void finish(State& st) {
+    if ((threadIdx.x & 31) == 0 && st.n_issued) bulk_wait_group_all();
+    __syncwarp();
+  }
   __device__ static __forceinline__ void chunk(const Params& p, State& st, int m_tile, int n_tile, int c,
-                                               int row_in_tile, int m_rows, const float (&v)[32], const CUtensorMap*,
-                                               uint32_t) {
+                                               int row_in_tile, int m_rows, const float (&v)[32],
+                                               const CUtensorMap* tmG, uint32_t staging) {
     // a CTA pair may own a 128-row tile that lies wholly past the slab's rows: nothing to write
     if (m_tile * BM >= ((m_rows + BM - 1) / BM) * BM) return;
     const int col_l = n_tile * BN + c * 32;
@@ -180,20 +184,35 @@ struct EpiGrad {
         for (int i = 0; i < 32; ++i) g[i] = i < nvalid ? g[i] : 0.f;
       }
     }
-    const int rl = m_tile * BM + row_in_tile;
-    uint4* dst = reinterpret_cast<uint4*>(p.G + (size_t)rl * p.ldG + col_l);
+    const int lane = threadIdx.x & 31;
+    const uint32_t buf = staging + (st.n_issued & 1u) * 4096u;
+    if ((c & 1) == 0) {
+      // first half of a new box: the store issued from this buffer two boxes ago must have read it
+      if (lane == 0) bulk_wait_group_read<1>();
+      __syncwarp();
+    }
+    // row `lane` of the box is 128 bytes = 8 chunks of 8 bf16; chunk j sits at position j ^ (row & 7)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      uint4 o;
       __nv_bfloat162 b0 = __floats2bfloat162_rn(g[8 * j + 0], g[8 * j + 1]);
       __nv_bfloat162 b1 = __floats2bfloat162_rn(g[8 * j + 2], g[8 * j + 3]);
       __nv_bfloat162 b2 = __floats2bfloat162_rn(g[8 * j + 4], g[8 * j + 5]);
       __nv_bfloat162 b3 = __floats2bfloat162_rn(g[8 * j + 6], g[8 * j + 7]);
-      o.x = *reinterpret_cast<uint32_t*>(&b0);
-      o.y = *reinterpret_cast<uint32_t*>(&b1);
-      o.z = *reinterpret_cast<uint32_t*>(&b2);
-      o.w = *reinterpret_cast<uint32_t*>(&b3);
-      __stcs(dst + j, o);   // written once, far larger than L2: do not displace the operands
+      const uint32_t jj = uint32_t(4 * (c & 1) + j);
+      const uint32_t addr = buf + lane * 128u + ((jj ^ uint32_t(lane & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t*>(&b0)),
+                   "r"(*reinterpret_cast<uint32_t*>(&b1)), "r"(*reinterpret_cast<uint32_t*>(&b2)),
+                   "r"(*reinterpret_cast<uint32_t*>(&b3))
+                   : "memory");
+    }
+    if (c & 1) {
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_2d(tmG, buf, col_l - 32, m_tile * BM + (row_in_tile - lane));
+        bulk_commit_group();
+      }
+      st.n_issued++;
     }
   }
   __device__ static __forceinline__ void end_unit(const Params&, State&, int, int, int, int) {}

@@ -137,6 +137,17 @@ bool map_out_f32(rl_ctx* c, CUtensorMap* m, const float* base, uint64_t rows, ui
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 [rows, cols] slab written by the dlogits epilogue in 32-row x 64-column boxes.
+bool map_out_bf16(rl_ctx* c, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {64, 32};
+  cuuint32_t es[2] = {1, 1};
+  return c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <class Epi, int A_MN, int B_MN>
 cudaError_t set_smem_attr() {
   cudaError_t e = cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -657,13 +668,14 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   const int* row_map = reinterpret_cast<const int*>(ws + L.row_map);
   const int* n_valid = &c->dstatus->n_valid;
 
-  CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn, tm_dH, tm_dW;
+  CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn, tm_dH, tm_dW, tm_G_out;
   bool ok = map_kmajor(c, &tmHc_k, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM) &&
             map_kmajor(c, &tmW_k, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_rows(c)) &&
             map_kmajor(c, &tmG_k, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM) &&
             map_mnmajor(c, &tmW_mn, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_panels(c)) &&
             map_mnmajor(c, &tmG_mn, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM / 64) &&
             map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, b_box_panels(c)) &&
+            map_out_bf16(c, &tm_G_out, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs) &&
             map_out_f32(c, &tm_dH, dH_acc, (uint64_t)L.Ts, (uint64_t)d, (uint64_t)d, (uint64_t)c->dh_k_slices, (uint64_t)L.Ts) &&
             map_out_f32(c, &tm_dW, dW, (uint64_t)V, (uint64_t)d, (uint64_t)d, 1, (uint64_t)V);
   if (!ok) return RL_ERR_CUDA;
@@ -692,8 +704,8 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         EpiGrad::Params ep;
         ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
         ep.lse = p.lse_c; ep.ent = p.ent_c; ep.cp = p.cp_c; ep.ce = p.ce_c;
-        ep.G = G; ep.ldG = L.Vs; ep.V = (int)V; ep.vocab_base = vocab_base;
-        launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, tmHc_k, sh, ep);   // no output map
+        ep.V = (int)V; ep.vocab_base = vocab_base;
+        launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, tm_G_out, sh, ep);
       }
       // (2) dH_slab (+)= G * W_slab        [rows x d], K = vocabulary columns of the slab
       {
