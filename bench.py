@@ -27,7 +27,7 @@ KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant
 # kernel from an ncu capture, valid only for the kernel sources whose hash is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "c0b16a0a8208b8d77b0394ec623be38b5348fffdb5bc96653861db97d3cb8d40", "kind": 2, "config": 1,
+NCU_TRAFFIC = {"sources_sha256": "d6abed72f57d7b2b3fe48569d0009bd64e21dbeba8e71af6061eed8eeae30b99", "kind": 2, "config": 1,
                "bytes_per_launch": 1334359000 + 137476608}   # profiles/gemm_kernels_config1_ncu_full.md
 
 

@@ -26,6 +26,9 @@
  *     valid.  Rows with mask 0 are skipped entirely (padding-free execution, section 4.4):
  *     their outputs are 0 and their token ids are ignored.
  *   - T = 0 or an all-zero mask is not an error: loss 0, gradients 0.
+ *   - A context is not thread-safe: use one context per host thread (contexts are cheap), or
+ *     serialise the calls on it.  Calls on different contexts may run concurrently as long as
+ *     their workspaces differ.
  */
 #ifndef RLHEAD_H_
 #define RLHEAD_H_

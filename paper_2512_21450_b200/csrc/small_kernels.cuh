@@ -526,6 +526,7 @@ __global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restr
 // elements apart (same slice count as gemm_extents chose for the pass): summed here in slice order.
 __device__ __forceinline__ float4 sum_k_slices(const float4* p, int n_slices, long long split_stride) {
   float4 x = __ldcs(p);
+  if (n_slices == 1) return x;
   for (int s = 1; s < n_slices; ++s) {
     const float4 y = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + s * split_stride));
     x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;

@@ -287,6 +287,12 @@ def test_token_weight_accumulate_and_strides(ctx):
                                      w.eps_low, w.eps_high, w.beta, accumulate_dW=True, dW=dW0.clone())
     _assert_status_ok(ctx)
     assert torch.allclose(acc["dW"], 2 * dW0, rtol=1e-5, atol=1e-12)
+    # a weight matrix that is a column slice of a wider one (ldW > d)
+    Wwide = torch.zeros(w.V, w.d + 128, dtype=torch.bfloat16, device="cuda")
+    Wwide[:, :w.d] = w.W
+    strided = ctx.rl_policy_loss_fwd_bwd(w.H, Wwide[:, :w.d], w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask,
+                                         w.eps_low, w.eps_high, w.beta)
+    assert torch.equal(strided["dW"], dW0) and torch.equal(strided["dH"], base["dH"])
     assert torch.equal(acc["dH"], base["dH"])
     assert acc["loss"].item() == base["loss"].item()     # deterministic reductions
 
