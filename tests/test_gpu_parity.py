@@ -416,6 +416,24 @@ def test_host_buffer_step_matches_device_call(ctx):
         assert loss2 == ref["loss"].item() and torch.equal(dW, ref["dW"])
 
 
+def test_autograd_front_end(ctx):
+    from paper_2512_21450_b200.autograd import fused_grpo_head_loss
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, seed=95)
+    o_adv = O.broadcast_to_tokens(O.grpo_advantages(w.rewards.cpu().numpy(), w.G), w.seq_offsets.cpu().numpy(), w.T)
+    adv = torch.from_numpy(o_adv).float().cuda()
+    H = w.H.clone().requires_grad_(True)
+    W = w.W.clone().requires_grad_(True)
+    loss, logp, ent, metrics = fused_grpo_head_loss(H, W, w.tokens, w.old_logp, w.ref_logp, adv, w.mask,
+                                                    w.eps_low, w.eps_high, w.beta)
+    (3.0 * loss).backward()
+    oo = _oracle_case(w, o_adv)
+    assert abs(loss.item() - oo["loss"]) <= TOL_LOSS_REL * abs(oo["loss"]) + 1e-7
+    assert _rel(_np64(H.grad), 3.0 * oo["dH"]) <= TOL_GRAD_REL
+    assert _rel(_np64(W.grad), 3.0 * oo["dW"]) <= TOL_GRAD_REL      # includes the rounding of dW to bf16
+    assert not logp.requires_grad and np.abs(_np64(logp) - oo["logp"]).max() <= TOL_LOGP
+
+
 def test_bounded_wait_times_out_cleanly(ctx):
     # a wait that nothing satisfies ends by itself, reports RL_ERR_TIMEOUT and leaves the context usable
     import time
