@@ -27,7 +27,7 @@ KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant
 # kernel from an ncu capture, valid only for the kernel sources whose hash is recorded with it.
-NCU_TRAFFIC = {"sources_sha256": "d6abed72f57d7b2b3fe48569d0009bd64e21dbeba8e71af6061eed8eeae30b99", "kind": 2, "config": 1,
+NCU_TRAFFIC = {"sources_sha256": "adf7f31006c1e4af98d5770e480822920a5e9bd4834808687d72ec7ce66fd89d", "kind": 2, "config": 1,
                "bytes_per_launch": 1334359000 + 137476608}   # profiles/gemm_kernels_config1_ncu_full.md
 
 
@@ -162,6 +162,61 @@ def run_reference(args):
     }))
 
 
+def run_library_comparison(args):
+    """Context for the roofline numbers: the library's tensor-core kernels and torch.matmul (cuBLAS)
+    on the same operand shapes, each looped for a few seconds so both sit at the board's power cap."""
+    import torch
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    ctx = Context(0)
+    w = make_workload(args.config)
+    rows = torch.nonzero(w.mask)[:, 0]
+    Hc = w.H[rows].contiguous()
+    N = Hc.shape[0] // 256 * 256
+    Hc = Hc[:N]
+    slab = 18944
+    G = torch.randn(N, slab, device="cuda").to(torch.bfloat16)
+    Ws = w.W[:slab].contiguous()
+    Vq = w.V // 4 // 256 * 256
+    Wq = w.W[:Vq].contiguous()
+
+    def sustained(fn, flops, secs=2.5):
+        for _ in range(10):
+            fn()
+        torch.cuda.synchronize()
+        smp = ClockSampler(0)
+        smp.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0, n = time.time(), 0
+        e0.record()
+        while time.time() - t0 < secs:
+            for _ in range(20):
+                fn()
+            n += 20
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        ck = smp.stop()
+        ms = e0.elapsed_time(e1) / n
+        return dict(ms=ms, tflops=flops / ms / 1e9, sm_mhz=ck["sm_mhz"])
+
+    out_q = torch.empty(N, Vq, dtype=torch.bfloat16, device="cuda")
+    C_h = torch.empty(N, w.d, dtype=torch.float32, device="cuda")
+    C_w = torch.empty(slab, w.d, dtype=torch.float32, device="cuda")
+    res = {
+        "forward_shape": {"shape": [N, w.d, Vq], "library_matmul": sustained(lambda: torch.matmul(Hc, Wq.T, out=out_q), 2.0 * N * w.d * Vq),
+                          "ours_fused_forward_full_vocab": sustained(lambda: ctx.rl_token_logprobs(w.H, w.W, w.tokens, w.mask),
+                                                                     2.0 * w.n_valid * w.d * w.V)},
+        "dH_shape": {"shape": [N, w.d, slab], "library_matmul": sustained(lambda: torch.matmul(G, Ws), 2.0 * N * w.d * slab),
+                     "ours_gemm_engine": sustained(lambda: ctx.rl_selftest_gemm(G, Ws, N, w.d, slab, 0, 1, C=C_h), 2.0 * N * w.d * slab)},
+        "dW_shape": {"shape": [slab, w.d, N], "library_matmul": sustained(lambda: torch.matmul(G.T, Hc), 2.0 * N * w.d * slab),
+                     "ours_gemm_engine": sustained(lambda: ctx.rl_selftest_gemm(G, Hc, slab, w.d, N, 1, 1, C=C_w), 2.0 * N * w.d * slab)},
+    }
+    status, _ = ctx.last_device_status()
+    assert status == 0
+    print(json.dumps({"library_comparison": res, "note": "sustained loops of 2.5 s each, one kernel at a time"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -172,11 +227,16 @@ def main():
     ap.add_argument("--reference-rows", type=int, default=256)
     ap.add_argument("--cpu-baseline-rows", type=int, default=512)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--compare-library", action="store_true",
+                    help="instead of the benchmark line, time the tensor-core kernels against torch.matmul")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.compare_library:
+        run_library_comparison(args)
         return
 
     import torch

@@ -849,6 +849,7 @@ rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, in
   sh.k_cap = (int)K;
   sh.n_tiles = (int)(N / BN);
   sh.n_range = 1;
+  sh.n_fastest = 1;   // walk the column tiles of one row panel first, as the gradient passes do
   CUtensorMap tc;
   if (!map_out_f32(c, &tc, C, (uint64_t)M, (uint64_t)N, (uint64_t)N, 1, (uint64_t)M)) return RL_ERR_CUDA;
   EpiAcc::Params ep;
