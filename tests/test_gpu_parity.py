@@ -434,6 +434,56 @@ def test_autograd_front_end(ctx):
     assert not logp.requires_grad and np.abs(_np64(logp) - oo["logp"]).max() <= TOL_LOGP
 
 
+def test_calls_can_be_captured_in_a_cuda_graph():
+    # the calls neither allocate nor synchronise, so a whole step can be captured once and replayed
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(0, seed=97)
+    c2 = Context(0)
+    try:
+        c2.ensure_workspace(w.T, w.d, w.V)
+        adv_seq = torch.empty_like(w.rewards)
+        adv_tok = torch.empty(w.T, device="cuda")
+        loss = torch.empty(1, device="cuda")
+        dH = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+        dW = torch.empty(w.V, w.d, device="cuda")
+        import ctypes
+        P = ctypes.c_void_p
+
+        def step():
+            s1 = c2.lib.rl_grpo_advantages_ex(c2.handle, P(w.rewards.data_ptr()), w.n_seq, w.G, 1, 1e-6,
+                                              P(w.seq_offsets.data_ptr()), w.T, P(adv_seq.data_ptr()),
+                                              P(adv_tok.data_ptr()))
+            s2 = c2.lib.rl_policy_loss_fwd_bwd(c2.handle, P(w.H.data_ptr()), w.d, P(w.W.data_ptr()), w.d,
+                                               P(w.tokens.data_ptr()), P(w.old_logp.data_ptr()),
+                                               P(w.ref_logp.data_ptr()), P(adv_tok.data_ptr()), P(w.mask.data_ptr()),
+                                               w.T, w.d, w.V, w.eps_low, w.eps_high, w.beta, P(loss.data_ptr()),
+                                               P(dH.data_ptr()), P(dW.data_ptr()))
+            assert s1 == 0 and s2 == 0
+
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            c2._bind_stream()
+            step()                                   # eager reference run on the side stream
+            torch.cuda.synchronize()
+            ref = (loss.clone(), dH.clone(), dW.clone())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                c2._bind_stream()
+                step()
+        for t in (loss, dH, dW):
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(loss, ref[0]) and torch.equal(dH, ref[1]) and torch.equal(dW, ref[2])
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(dW, ref[2])
+        assert c2.last_device_status()[0] == 0
+    finally:
+        c2.close()
+
+
 def test_bounded_wait_times_out_cleanly(ctx):
     # a wait that nothing satisfies ends by itself, reports RL_ERR_TIMEOUT and leaves the context usable
     import time
