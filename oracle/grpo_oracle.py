@@ -261,10 +261,17 @@ def per_token_terms(logp, old_logp, ref_logp, adv, eps_low, eps_high, beta,
     return s, k3, rho, active, dlogp
 
 
+def full_kl(LP, LQ):
+    """KL(pi_theta(.|s_t) || pi_ref(.|s_t)) per row from the two log-probability matrices: the
+    regulariser exactly as section 2.2 / 3.1 print it, sum_j p_j (log p_j - log q_j)."""
+    return (np.exp(LP) * (LP - LQ)).sum(axis=1)
+
+
 def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
                         eps_low, eps_high, beta, ent_coef=0.0,
                         token_weight=None, literal_clip=False,
-                        seq_offsets=None, agg_mode=0, sequence_level=False):
+                        seq_offsets=None, agg_mode=0, sequence_level=False,
+                        H_ref=None, W_ref=None):
     """Loss of Eq. 6 (negated) and its gradients with respect to H and W.
 
     Returns a dict with loss, dH[T,d], dW[V,d], logp, entropy, lse, G (the
@@ -330,6 +337,17 @@ def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
             wdlogp = wdlogp + wr * beta * (1.0 - np.exp(delta))
         else:
             k3 = np.zeros_like(logp)
+    kl_full = None
+    if H_ref is not None:
+        # full-distribution KL to the (frozen) reference policy softmax(W_ref h_ref) replaces the
+        # sampled-token k3 estimate: remove what k3 contributed, add beta * KL_t and its gradient
+        Zr = logits(np.asarray(H_ref, dtype=np.float64)[rows], W_ref)
+        _, LQ, _ = log_softmax_stats(Zr)
+        kl_full = full_kl(LP, LQ)
+        if beta != 0.0:
+            delta_k3 = ref[rows] - logp
+            wdlogp = wdlogp - wr * beta * (1.0 - np.exp(delta_k3))
+        k3 = kl_full
     loss_t = -s + beta * k3 - ent_coef * ent
     loss = float((wr * loss_t).sum())
 
@@ -341,6 +359,9 @@ def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
     G = wdlogp[:, None] * (onehot - P)
     if ent_coef != 0.0:
         G += (wr * ent_coef)[:, None] * P * (LP + ent[:, None])
+    if kl_full is not None and beta != 0.0:
+        # d KL_t / d z_tj = p_tj (log p_tj - log q_tj - KL_t)
+        G += (wr * beta)[:, None] * P * (LP - LQ - kl_full[:, None])
 
     out["dH"][rows] = G @ W                         # dH_tk = sum_j g_tj W_jk
     out["dW"] = G.T @ Hr                            # dW_jk = sum_t g_tj H_tk

@@ -19,7 +19,7 @@ MUTANTS = {
     "surrogate not pessimistic": ("s = np.minimum(rho * adv, clipped * adv)\n        # the unclipped",
                                   "s = np.maximum(rho * adv, clipped * adv)\n        # the unclipped"),
     "logit gradient sign": ("G = wdlogp[:, None] * (onehot - P)", "G = wdlogp[:, None] * (P - onehot)"),
-    "entropy gradient misses the +Ent term": ("P * (LP + ent[:, None])\n\n    out[\"dH\"]", "P * LP\n\n    out[\"dH\"]"),
+    "entropy gradient misses the +Ent term": ("G += (wr * ent_coef)[:, None] * P * (LP + ent[:, None])\n    if kl_full", "G += (wr * ent_coef)[:, None] * P * LP\n    if kl_full"),
     "dW uses the wrong operand": ('out["dW"] = G.T @ Hr', 'out["dW"] = G.T @ (Hr * 0 + 1)'),
     "dH scaled": ('out["dH"][rows] = G @ W ', 'out["dH"][rows] = 2 * G @ W '),
     "population instead of sample variance": ("/ (group_size - ddof)", "/ group_size"),
@@ -30,6 +30,8 @@ MUTANTS = {
     "sequence-level gradient forgets 1/len": ("-(rho / np.maximum(len_full[rows], 1.0)) * seq_sum[rows]", "-rho * seq_sum[rows]"),
     "RLOO includes the response itself": ("if j != i]", "]"),
     "OPO baseline unweighted": ("base = (ln[sl] * r[sl]).sum() / tot", "base = r[sl].sum() / len(r[sl])"),
+    "full KL gradient misses the -KL term": ("P * (LP - LQ - kl_full[:, None])", "P * (LP - LQ)"),
+    "full KL direction swapped": ("return (np.exp(LP) * (LP - LQ)).sum(axis=1)", "return (np.exp(LQ) * (LQ - LP)).sum(axis=1)"),
     "logits index order": ("return H @ W.T", "return (W @ H.T).T[::-1][::-1] if H.shape[0] == 1 else (H[:, ::-1] @ W[:, ::-1].T if False else H @ W[::-1].T)"),
 }
 

@@ -476,3 +476,71 @@ def test_sequence_level_reduces_to_token_level_for_single_token_sequences():
     b = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, 0.2, 0.2, 0.04)
     assert abs(a["loss"] - b["loss"]) < 1e-15 and np.allclose(a["dH"], b["dH"], atol=1e-15)
     assert np.allclose(a["dW"], b["dW"], atol=1e-15)
+
+
+# ----------------------------------------------------------------------------- full-distribution KL
+def test_full_kl_values():
+    rng = _rng(41)
+    Z = rng.normal(size=(5, 9))
+    Zr = rng.normal(size=(5, 9))
+    _, LP, ent = O.log_softmax_stats(Z)
+    _, LQ, _ = O.log_softmax_stats(Zr)
+    kl = O.full_kl(LP, LQ)
+    for t in range(5):
+        p = np.exp(Z[t]) / np.exp(Z[t]).sum()
+        q = np.exp(Zr[t]) / np.exp(Zr[t]).sum()
+        assert abs(kl[t] - sum(p[j] * math.log(p[j] / q[j]) for j in range(9))) < 1e-13
+    assert np.all(kl >= 0)
+    assert np.allclose(O.full_kl(LP, LP), 0.0, atol=1e-15)
+    _, LU, _ = O.log_softmax_stats(np.zeros((5, 9)))
+    assert np.allclose(O.full_kl(LP, LU), math.log(9) - ent, atol=1e-13)       # uniform reference
+    ref = torch.nn.functional.kl_div(torch.tensor(LQ), torch.tensor(LP), log_target=True, reduction="none").sum(1)
+    assert np.allclose(kl, ref.numpy(), atol=1e-13)                             # library second opinion
+
+
+def test_full_kl_loss_and_gradient():
+    rng = _rng(42)
+    T, d, dr, V = 7, 6, 5, 11
+    H = rng.normal(size=(T, d)); W = rng.normal(size=(V, d)) * 0.6
+    Hr = rng.normal(size=(T, dr)); Wr = rng.normal(size=(V, dr)) * 0.6
+    tokens = rng.integers(0, V, size=T)
+    mask = np.array([1, 1, 0, 1, 1, 1, 1], dtype=np.uint8)
+    lp, _, _ = O.token_logprobs(H, W, tokens)
+    old = lp + rng.normal(size=T) * 0.3
+    adv = rng.normal(size=T)
+    kw = dict(eps_low=0.2, eps_high=0.2, beta=0.3, ent_coef=0.02, H_ref=Hr, W_ref=Wr)
+    out = O.policy_loss_fwd_bwd(H, W, tokens, old, None, adv, mask, **kw)
+    base = O.policy_loss_fwd_bwd(H, W, tokens, old, None, adv, mask, 0.2, 0.2, 0.0, ent_coef=0.02)
+    w = O.token_weights(mask)
+    Z, Zr = H @ W.T, Hr @ Wr.T
+    _, LP, _ = O.log_softmax_stats(Z)
+    _, LQ, _ = O.log_softmax_stats(Zr)
+    assert abs(out["loss"] - base["loss"] - 0.3 * (w * O.full_kl(LP, LQ)).sum()) < 1e-14
+    # same policy and reference: the KL term and its gradient vanish
+    same = O.policy_loss_fwd_bwd(H, W, tokens, old, None, adv, mask, 0.2, 0.2, 0.3, ent_coef=0.02, H_ref=H, W_ref=W)
+    assert abs(same["loss"] - base["loss"]) < 1e-14 and np.allclose(same["dH"], base["dH"], atol=1e-15)
+
+    def loss(Hx, Wx):
+        return O.policy_loss_fwd_bwd(Hx, Wx, tokens, old, None, adv, mask, **kw)["loss"]
+
+    h = 1e-6
+    for (X, dX, which) in ((H, out["dH"], 0), (W, out["dW"], 1)):
+        num = np.zeros_like(X)
+        for idx in np.ndindex(*X.shape):
+            Xp = X.copy(); Xp[idx] += h
+            Xm = X.copy(); Xm[idx] -= h
+            num[idx] = ((loss(Xp, W) - loss(Xm, W)) if which == 0 else (loss(H, Xp) - loss(H, Xm))) / (2 * h)
+        assert np.abs(num - dX).max() / max(np.abs(num).max(), 1e-12) < 1e-6
+    Ht = torch.tensor(H, requires_grad=True); Wt = torch.tensor(W, requires_grad=True)
+    lsm = torch.log_softmax(Ht @ Wt.T, dim=1)
+    lq = torch.log_softmax(torch.tensor(Hr) @ torch.tensor(Wr).T, dim=1)
+    lpt = lsm.gather(1, torch.tensor(tokens)[:, None])[:, 0]
+    ratio = (lpt - torch.tensor(old)).exp()
+    A = torch.tensor(adv)
+    s = torch.minimum(ratio * A, ratio.clamp(0.8, 1.2) * A)
+    kl = (lsm.exp() * (lsm - lq)).sum(1)
+    ent = -(lsm.exp() * lsm).sum(1)
+    L = ((-s + 0.3 * kl - 0.02 * ent) * torch.tensor(w)).sum()
+    L.backward()
+    assert abs(L.item() - out["loss"]) < 1e-13
+    assert np.allclose(Ht.grad.numpy(), out["dH"], atol=1e-13) and np.allclose(Wt.grad.numpy(), out["dW"], atol=1e-13)
