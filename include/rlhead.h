@@ -65,6 +65,9 @@ const char* rl_status_string(rl_status s);
  * size does not grow with T*V: the gradient with respect to the logits only ever exists for a
  * bounded slab of rows x vocabulary columns. */
 rl_status rl_workspace_bytes(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_t* bytes);
+/* The same for calls that set rl_loss_opts.kl_full with a reference model of hidden size d_ref
+ * (adds the compacted reference rows and five per-row arrays). */
+rl_status rl_workspace_bytes_kl(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, int64_t d_ref, size_t* bytes);
 /* Size of the slab the backward pass works in: at most max_rows token rows x max_cols vocabulary
  * columns of the gradient with respect to the logits exist at a time (bf16, in the workspace).
  * max_rows a multiple of 128, max_cols a multiple of 256; 0 restores a default (32768 x 18944,
@@ -170,6 +173,21 @@ typedef struct {
   const int32_t* seq_offsets; /* [n_seq+1] ascending row range of every response, needed by    */
   int64_t n_seq;              /* agg_mode 1/2 and sequence_level; seq_offsets[n_seq] <= T;     */
                               /* valid rows outside every range then take no part in the loss  */
+  int kl_full;                /* non-zero: the regulariser is the full-distribution            */
+                              /* KL(pi_theta(.|s_t) || pi_ref(.|s_t)) = sum_j p_j (log p_j -   */
+                              /* log q_j) over the vocabulary, as sections 2.2 and 3.1 print   */
+                              /* it, instead of the sampled-token k3 estimate; q = softmax(    */
+                              /* W_ref h_ref_t) is recomputed tile by tile next to p, never    */
+                              /* stored.  ref_logp is then unused (may be NULL).  Not          */
+                              /* combined with sequence_level / agg_mode 1, 2 (INVALID_ARG).   */
+  const void* H_ref;          /* [T, d_ref] bf16 device, row stride ldH_ref: hidden states of  */
+  int64_t ldH_ref;            /* the frozen reference model for the same rows                  */
+  const void* W_ref;          /* [V, d_ref] bf16 device, row stride ldW_ref: its LM head       */
+  int64_t ldW_ref;
+  int64_t d_ref;              /* multiple of 64 (whole 128-byte k-slices), strides multiples   */
+                              /* of 8, bases 16-byte aligned; the reference model is a         */
+                              /* constant: no gradient flows to H_ref / W_ref                  */
+  float* kl_out;              /* [T] or NULL: per-token KL_t of the kl_full mode (masked rows 0) */
 } rl_loss_opts;
 
 rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* ctx, const void* H, int64_t ldH, const void* W,

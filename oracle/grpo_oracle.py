@@ -385,8 +385,11 @@ def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
 # the logits for every valid token plus per-token statistics.
 # --------------------------------------------------------------------------- #
 def dH_rows(H_rows, W, tokens_rows, old_rows, ref_rows, adv_rows, w_rows,
-            eps_low, eps_high, beta, ent_coef=0.0):
-    """dH for a subset of valid rows whose token weights w_rows are given."""
+            eps_low, eps_high, beta, ent_coef=0.0, H_ref_rows=None, W_ref=None):
+    """dH for a subset of valid rows whose token weights w_rows are given.
+
+    With H_ref_rows / W_ref the regulariser is the full-distribution KL to
+    softmax(W_ref h_ref) as in policy_loss_fwd_bwd (ref_rows is then unused)."""
     H_rows = np.asarray(H_rows, dtype=np.float64)
     W = np.asarray(W, dtype=np.float64)
     n = H_rows.shape[0]
@@ -402,10 +405,19 @@ def dH_rows(H_rows, W, tokens_rows, old_rows, ref_rows, adv_rows, w_rows,
     onehot = np.zeros_like(P)
     onehot[np.arange(n), y] = 1.0
     w_rows = np.asarray(w_rows, dtype=np.float64)
+    kl = None
+    if H_ref_rows is not None:
+        _, LQ, _ = log_softmax_stats(logits(np.asarray(H_ref_rows, dtype=np.float64), W_ref))
+        kl = full_kl(LP, LQ)
+        # the sampled-token estimate plays no part: take its derivative back out
+        dlogp = dlogp - beta * (1.0 - np.exp(ref - logp)) if beta != 0.0 else dlogp
+        k3 = kl
     G = (w_rows * dlogp)[:, None] * (onehot - P)
     if ent_coef != 0.0:
         G += (w_rows * ent_coef)[:, None] * P * (LP + ent[:, None])
-    return dict(dH=G @ W, logp=logp, entropy=ent, lse=lse,
+    if kl is not None and beta != 0.0:
+        G += (w_rows * beta)[:, None] * P * (LP - LQ - kl[:, None])
+    return dict(dH=G @ W, logp=logp, entropy=ent, lse=lse, kl=kl,
                 loss_t=-s + beta * k3 - ent_coef * ent)
 
 

@@ -42,6 +42,13 @@ class rl_loss_opts(ctypes.Structure):
         ("dH_dtype", c_int),
         ("seq_offsets", c_void_p),
         ("n_seq", c_int64),
+        ("kl_full", c_int),
+        ("H_ref", c_void_p),
+        ("ldH_ref", c_int64),
+        ("W_ref", c_void_p),
+        ("ldW_ref", c_int64),
+        ("d_ref", c_int64),
+        ("kl_out", c_void_p),
     ]
 
 
@@ -64,6 +71,7 @@ def load_library():
     lib.rl_set_stream.argtypes = [P, P]
     lib.rl_workspace_bytes.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
     lib.rl_workspace_bytes_host.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
+    lib.rl_workspace_bytes_kl.argtypes = [P, c_int64, c_int64, c_int64, c_int64, POINTER(c_size_t)]
     lib.rl_set_workspace.argtypes = [P, P, c_size_t]
     lib.rl_set_slab_limits.argtypes = [P, c_int, c_int]
     lib.rl_set_dh_k_slices.argtypes = [P, c_int]
@@ -92,6 +100,7 @@ def load_library():
     lib.rl_token_logprobs_static.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P, P]
     lib.rl_token_logprobs_static.restype = c_int
     for name in ("rl_create", "rl_destroy", "rl_set_stream", "rl_workspace_bytes", "rl_workspace_bytes_host",
+                 "rl_workspace_bytes_kl",
                  "rl_set_workspace", "rl_set_slab_limits", "rl_last_device_status", "rl_grpo_advantages", "rl_grpo_advantages_ex",
                  "rl_token_logprobs", "rl_policy_loss_fwd_bwd", "rl_policy_loss_fwd_bwd_ex",
                  "rl_policy_loss_fwd_bwd_host", "rl_selftest_gemm", "rl_launch_count", "rl_set_profiling",
@@ -138,14 +147,17 @@ class Context:
         _check(self.lib.rl_set_stream(self.handle, c_void_p(torch.cuda.current_stream(self.device).cuda_stream)),
                "rl_set_stream")
 
-    def workspace_bytes(self, T, d, V, host=False):
+    def workspace_bytes(self, T, d, V, host=False, d_ref=0):
         n = c_size_t()
+        if d_ref:
+            _check(self.lib.rl_workspace_bytes_kl(self.handle, T, d, V, d_ref, byref(n)), "rl_workspace_bytes_kl")
+            return n.value
         fn = self.lib.rl_workspace_bytes_host if host else self.lib.rl_workspace_bytes
         _check(fn(self.handle, T, d, V, byref(n)), "rl_workspace_bytes")
         return n.value
 
-    def ensure_workspace(self, T, d, V, host=False):
-        need = self.workspace_bytes(T, d, V, host)
+    def ensure_workspace(self, T, d, V, host=False, d_ref=0):
+        need = self.workspace_bytes(T, d, V, host, d_ref)
         if self._ws is None or self._ws.numel() < need:
             self._ws = None
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
@@ -214,13 +226,20 @@ class Context:
     def rl_policy_loss_fwd_bwd(self, H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta,
                                ent_coef=0.0, token_weight=None, accumulate_dW=False, dW=None, want_aux=True,
                                dH=None, loss=None, agg_mode=0, sequence_level=False, seq_offsets=None,
-                               dH_fp32=False):
+                               dH_fp32=False, H_ref=None, W_ref=None):
+        """H_ref [T, d_ref] and W_ref [V, d_ref] (bf16) switch the regulariser to the full-distribution
+        KL(pi_theta || pi_ref) against softmax(W_ref h_ref); ref_logp is then unused."""
         self._bind_stream()
         T, d = H.shape
         V = W.shape[0]
         assert H.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and tokens.dtype == torch.int32
         assert H.stride(1) == 1 and W.stride(1) == 1
-        self.ensure_workspace(T, d, V)
+        kl_full = W_ref is not None
+        if kl_full:
+            assert H_ref is not None and H_ref.dtype == torch.bfloat16 and W_ref.dtype == torch.bfloat16
+            assert H_ref.shape[0] == T and W_ref.shape[0] == V and H_ref.shape[1] == W_ref.shape[1]
+            assert H_ref.stride(1) == 1 and W_ref.stride(1) == 1
+        self.ensure_workspace(T, d, V, d_ref=W_ref.shape[1] if kl_full else 0)
         dev = W.device
         loss = torch.empty(1, dtype=torch.float32, device=dev) if loss is None else loss
         if dH is None:
@@ -229,7 +248,7 @@ class Context:
             dW = torch.empty(V, d, dtype=torch.float32, device=dev)
         out = dict(loss=loss, dH=dH, dW=dW)
         plain = (ent_coef == 0.0 and token_weight is None and not accumulate_dW and not want_aux and agg_mode == 0
-                 and not sequence_level and not dH_fp32)
+                 and not sequence_level and not dH_fp32 and not kl_full)
         args = [self.handle, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0), _ptr(tokens), _ptr(old_logp),
                 _ptr(ref_logp), _ptr(adv), _ptr(mask), T, d, V, eps_low, eps_high, beta, _ptr(loss), _ptr(dH),
                 _ptr(dW)]
@@ -244,6 +263,13 @@ class Context:
         opts.agg_mode = agg_mode
         opts.sequence_level = int(sequence_level)
         opts.dH_dtype = int(dH_fp32)
+        if kl_full:
+            opts.kl_full = 1
+            opts.H_ref = H_ref.data_ptr() if T else None
+            opts.ldH_ref = H_ref.stride(0) if T else W_ref.shape[1]
+            opts.W_ref = W_ref.data_ptr()
+            opts.ldW_ref = W_ref.stride(0)
+            opts.d_ref = W_ref.shape[1]
         if seq_offsets is not None:
             assert seq_offsets.dtype == torch.int32 and seq_offsets.is_cuda
             opts.seq_offsets = seq_offsets.data_ptr()
@@ -255,6 +281,9 @@ class Context:
             opts.logp_out = out["logp"].data_ptr()
             opts.entropy_out = out["entropy"].data_ptr()
             opts.metrics_out = out["metrics"].data_ptr()
+            if kl_full:
+                out["kl"] = torch.empty(T, dtype=torch.float32, device=dev)
+                opts.kl_out = out["kl"].data_ptr()
         _check(self.lib.rl_policy_loss_fwd_bwd_ex(*args, byref(opts)), "rl_policy_loss_fwd_bwd_ex")
         return out
 

@@ -54,16 +54,27 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct WsLayout {
   int Tpad, Ts, Vs;
   size_t scan_counts, row_map, tokens_c, logp_c, lse_c, ent_c, cp_c, ce_c, partials, block_sums, Hc, G, dH_acc, staging, total;
+  size_t Hc_ref, partials2, lse_ref_c, kl_c, cb_c;   // only with a reference model (full KL)
+};
+
+// Reference-model operands of the full-distribution KL (all NULL / 0 when it is not used).
+struct KlRef {
+  const void* H_ref;
+  int64_t ldH_ref;
+  const void* W_ref;
+  int64_t ldW_ref;
+  int64_t d_ref;
 };
 
 // staging_T > 0 adds room for host-call inputs (H, tokens, old, ref, adv, mask).
-WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_staging) {
+WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_staging, int64_t d_ref = 0) {
   WsLayout L;
   L.Tpad = (int)align_up((size_t)(T > 0 ? T : 1), 128);
   L.Ts = L.Tpad < c->slab_rows ? L.Tpad : c->slab_rows;
   const int Vpad = (int)align_up((size_t)V, 256);
   L.Vs = Vpad < c->slab_cols ? Vpad : c->slab_cols;
   size_t o = 0;
+  size_t n_part_ranges = kMaxSplit;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 1024); return at; };
   L.scan_counts = take(((size_t)L.Tpad / 4096 + 2) * 4);
   L.row_map = take((size_t)L.Tpad * 4);
@@ -76,13 +87,21 @@ WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_s
   {
     // one float4 per (column range, row): at most kMaxSplit ranges, or one per kFwdRange column tiles
     const size_t by_range = (size_t)(((V + BN - 1) / BN + kFwdRange - 1) / kFwdRange);
-    const size_t n_ranges = by_range > (size_t)kMaxSplit ? by_range : (size_t)kMaxSplit;
-    L.partials = take(n_ranges * L.Tpad * sizeof(float4));
+    n_part_ranges = by_range > (size_t)kMaxSplit ? by_range : (size_t)kMaxSplit;
+    L.partials = take(n_part_ranges * L.Tpad * sizeof(float4));
   }
   L.block_sums = take((size_t)1024 * kLossSums * sizeof(double));
   L.Hc = take((size_t)L.Tpad * d * 2);
   L.G = take((size_t)L.Ts * L.Vs * 2);
   L.dH_acc = take((size_t)c->dh_k_slices * L.Ts * d * 4);
+  L.Hc_ref = L.partials2 = L.lse_ref_c = L.kl_c = L.cb_c = 0;
+  if (d_ref > 0) {
+    L.Hc_ref = take((size_t)L.Tpad * d_ref * 2);
+    L.partials2 = take((size_t)n_part_ranges * L.Tpad * sizeof(float4));
+    L.lse_ref_c = take((size_t)L.Tpad * 4);
+    L.kl_c = take((size_t)L.Tpad * 4);
+    L.cb_c = take((size_t)L.Tpad * 4);
+  }
   L.staging = o;
   if (host_staging) {
     take((size_t)T * d * 2);  // H
@@ -157,6 +176,14 @@ cudaError_t set_smem_attr() {
                               kGemmSmemBytes);
 }
 
+template <class Epi>
+cudaError_t set_smem_attr_dual() {
+  cudaError_t e = cudaFuncSetAttribute(dual_gemm_kernel<Epi, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kGemmSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(dual_gemm_kernel<Epi, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+}
+
 // Rows of B that one CTA stages per k-slice (box height of a K-major B map) and the number of
 // 64-wide panels of an MN-major B map, for the context's CTA grouping.
 inline uint32_t b_box_rows(const rl_ctx* c) { return BN / c->cta_group; }
@@ -205,6 +232,34 @@ void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b
   prof_end(c, prof, kind);
 }
 
+template <class Epi>
+void launch_dual(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
+                 const CUtensorMap& b2, const CUtensorMap& out, const GemmShape& sh, int k2_len,
+                 const typename Epi::Params& ep) {
+  const int prof = prof_begin(c, kind);
+  if (c->cta_group == 2) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->grid[2]);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = kGemmSmemBytes;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, dual_gemm_kernel<Epi, 2>, a, b, a2, b2, out, sh, k2_len, ep, c->dstatus);
+  } else {
+    dual_gemm_kernel<Epi, 1><<<c->grid[1], kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, a2, b2, out, sh, k2_len,
+                                                                                     ep, c->dstatus);
+  }
+  c->launches++;
+  prof_end(c, prof, kind);
+}
+
 rl_status check_hw(const void* H, int64_t ldH, const void* W, int64_t ldW, int64_t T, int64_t d, int64_t V) {
   if (T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
   if (T > 0 && (!H || !W)) return RL_ERR_INVALID_ARG;
@@ -226,7 +281,7 @@ inline rl_status cuda_ok() { return cudaGetLastError() == cudaSuccess ? RL_OK : 
 // Mask scan + row compaction + forward statistics.  Leaves per-range partials in the workspace.
 rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, const void* W, int64_t ldW,
                       const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
-                      GemmShape* shape_out) {
+                      GemmShape* shape_out, const KlRef* kl = nullptr) {
   char* ws = static_cast<char*>(c->ws);
   int* row_map = reinterpret_cast<int*>(ws + L.row_map);
   int* tokens_c = reinterpret_cast<int*>(ws + L.tokens_c);
@@ -261,7 +316,27 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   ep.partials = reinterpret_cast<float4*>(ws + L.partials);
   ep.part_stride = L.Tpad;
   ep.V = (int)V;
-  launch_gemm<EpiStats, 0, 0>(c, 0, tmA, tmB, tmA, sh, ep);   // no output map
+  if (!kl) {
+    launch_gemm<EpiStats, 0, 0>(c, 0, tmA, tmB, tmA, sh, ep);   // no output map
+  } else {
+    // full KL: compact the reference hidden states with the same row map and form both logit
+    // tiles per output tile
+    __nv_bfloat16* Hc_ref = reinterpret_cast<__nv_bfloat16*>(ws + L.Hc_ref);
+    gather_plain_kernel<<<c->n_sm * 4, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16*>(kl->H_ref), kl->ldH_ref,
+                                                            (int)kl->d_ref, row_map, Hc_ref, c->dstatus);
+    c->launches++;
+    CUtensorMap tmA2, tmB2;
+    if (!map_kmajor(c, &tmA2, Hc_ref, (uint64_t)L.Tpad, (uint64_t)kl->d_ref, (uint64_t)kl->d_ref, BM)) return RL_ERR_CUDA;
+    if (!map_kmajor(c, &tmB2, kl->W_ref, (uint64_t)V, (uint64_t)kl->d_ref, (uint64_t)kl->ldW_ref, b_box_rows(c)))
+      return RL_ERR_CUDA;
+    EpiStatsKL::Params ek;
+    ek.tokens_c = tokens_c;
+    ek.partials = ep.partials;
+    ek.partials2 = reinterpret_cast<float4*>(ws + L.partials2);
+    ek.part_stride = L.Tpad;
+    ek.V = (int)V;
+    launch_dual<EpiStatsKL>(c, 0, tmA, tmB, tmA2, tmB2, tmA, sh, (int)kl->d_ref, ek);
+  }
   *shape_out = sh;
   return cuda_ok();
 }
@@ -323,7 +398,8 @@ rl_status rl_create(rl_ctx** out, int device) {
   cudaMemset(c->dstatus, 0, 256);
   bool ok = set_smem_attr<EpiStats, 0, 0>() == cudaSuccess && set_smem_attr<EpiGrad, 0, 0>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 0, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 0, 1>() == cudaSuccess &&
-            set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess;
+            set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess &&
+            set_smem_attr_dual<EpiStatsKL>() == cudaSuccess && set_smem_attr_dual<EpiGradKL>() == cudaSuccess;
   if (!ok) { cudaFree(c->dstatus); delete c; return RL_ERR_CUDA; }
   {
     // how many CTA pairs can be resident at once (pairs must share a TPC): the persistent grid
@@ -373,6 +449,12 @@ rl_status rl_set_stream(rl_ctx* c, void* s) {
 rl_status rl_workspace_bytes(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t* bytes) {
   if (!c || !bytes || T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
   *bytes = ws_layout(c, T, d, V, false).total;
+  return RL_OK;
+}
+
+rl_status rl_workspace_bytes_kl(rl_ctx* c, int64_t T, int64_t d, int64_t V, int64_t d_ref, size_t* bytes) {
+  if (!c || !bytes || T < 0 || d <= 0 || V <= 0 || d_ref <= 0) return RL_ERR_INVALID_ARG;
+  *bytes = ws_layout(c, T, d, V, false, d_ref).total;
   return RL_OK;
 }
 
@@ -560,7 +642,6 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   if (!(eps_low >= 0.f && eps_low < 1.f) || !(eps_high >= 0.f) || !(beta >= 0.f)) return RL_ERR_INVALID_ARG;
   if (!loss || !dW || !W) return RL_ERR_INVALID_ARG;
   if (T > 0 && (!tokens || !old_logp || !adv || !dH)) return RL_ERR_INVALID_ARG;
-  if (beta != 0.f && T > 0 && !ref_logp) return RL_ERR_INVALID_ARG;
   rl_loss_opts o;
   memset(&o, 0, sizeof(o));
   if (opts) {
@@ -569,12 +650,27 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
     memcpy(&o, opts, opts->struct_size);
   }
   if (!(o.ent_coef >= 0.f)) return RL_ERR_INVALID_ARG;
+  if (beta != 0.f && T > 0 && !ref_logp && !o.kl_full) return RL_ERR_INVALID_ARG;
   if (o.agg_mode < 0 || o.agg_mode > 2 || (o.dH_dtype != 0 && o.dH_dtype != 1)) return RL_ERR_INVALID_ARG;
   if ((o.sequence_level || (o.agg_mode != 0 && !o.token_weight)) && T > 0 &&
       (!o.seq_offsets || o.n_seq <= 0 || o.n_seq > T))
     return RL_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(dH) & 15) || (reinterpret_cast<uintptr_t>(dW) & 15)) return RL_ERR_ALIGNMENT;
-  const WsLayout L = ws_layout(c, T, d, V, false);
+  const bool seq_path = o.sequence_level || (o.agg_mode != 0 && !o.token_weight);
+  KlRef klref;
+  memset(&klref, 0, sizeof(klref));
+  if (o.kl_full) {
+    if (seq_path) return RL_ERR_INVALID_ARG;
+    if (!o.W_ref || (T > 0 && !o.H_ref) || o.d_ref <= 0) return RL_ERR_INVALID_ARG;
+    if (o.d_ref % 64 != 0 || o.ldH_ref < o.d_ref || o.ldW_ref < o.d_ref || o.ldH_ref % 8 != 0 || o.ldW_ref % 8 != 0)
+      return RL_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(o.H_ref) & 15) || (reinterpret_cast<uintptr_t>(o.W_ref) & 15))
+      return RL_ERR_ALIGNMENT;
+    klref.H_ref = o.H_ref; klref.ldH_ref = o.ldH_ref;
+    klref.W_ref = o.W_ref; klref.ldW_ref = o.ldW_ref;
+    klref.d_ref = o.d_ref;
+  }
+  const WsLayout L = ws_layout(c, T, d, V, false, o.kl_full ? o.d_ref : 0);
   if ((s = check_ws(c, L)) != RL_OK) return s;
   char* ws = static_cast<char*>(c->ws);
   cudaStream_t st = c->stream;
@@ -591,7 +687,9 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
 
   // ---- forward: statistics per (row, vocabulary range)
   GemmShape fwd_shape;
-  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &fwd_shape)) != RL_OK) return s;
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &fwd_shape, o.kl_full ? &klref : nullptr)) !=
+      RL_OK)
+    return s;
 
   // ---- merge + per-token loss, coefficients of the backward pass
   LossParams p;
@@ -618,10 +716,18 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   p.logp_out = o.logp_out;
   p.ent_out = o.entropy_out;
   p.block_sums = reinterpret_cast<double*>(ws + L.block_sums);
+  if (o.kl_full) {
+    p.kl_full = 1;
+    p.partials2 = reinterpret_cast<const float4*>(ws + L.partials2);
+    p.lse_ref_c = reinterpret_cast<float*>(ws + L.lse_ref_c);
+    p.kl_c = reinterpret_cast<float*>(ws + L.kl_c);
+    p.cb_c = reinterpret_cast<float*>(ws + L.cb_c);
+    p.kl_out = o.kl_out;
+    if (o.kl_out) cudaMemsetAsync(o.kl_out, 0, (size_t)T * 4, st);
+  }
   int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
   if (blocks > 1024) blocks = 1024;
   const int pr_loss = prof_begin(c, 6);
-  const bool seq_path = o.sequence_level || (o.agg_mode != 0 && !o.token_weight);
   if (!seq_path) {
     combine_loss_kernel<<<blocks, kLossThreads, 0, st>>>(p, c->dstatus);
     c->launches++;
@@ -668,7 +774,12 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   const int* row_map = reinterpret_cast<const int*>(ws + L.row_map);
   const int* n_valid = &c->dstatus->n_valid;
 
-  CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn, tm_dH, tm_dW, tm_G_out;
+  CUtensorMap tmHc_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmHc_mn, tm_dH, tm_dW, tm_G_out, tmHr_k, tmWr_k;
+  if (o.kl_full) {
+    if (!map_kmajor(c, &tmHr_k, ws + L.Hc_ref, (uint64_t)L.Tpad, (uint64_t)o.d_ref, (uint64_t)o.d_ref, BM) ||
+        !map_kmajor(c, &tmWr_k, o.W_ref, (uint64_t)V, (uint64_t)o.d_ref, (uint64_t)o.ldW_ref, b_box_rows(c)))
+      return RL_ERR_CUDA;
+  }
   bool ok = map_kmajor(c, &tmHc_k, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM) &&
             map_kmajor(c, &tmW_k, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_rows(c)) &&
             map_kmajor(c, &tmG_k, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM) &&
@@ -701,11 +812,20 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
         sh.n_range = 1;
         sh.a_mn_slab = 1;
         sh.b_mn_off = vocab_base;
-        EpiGrad::Params ep;
-        ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
-        ep.lse = p.lse_c; ep.ent = p.ent_c; ep.cp = p.cp_c; ep.ce = p.ce_c;
-        ep.V = (int)V; ep.vocab_base = vocab_base;
-        launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, tm_G_out, sh, ep);
+        if (!o.kl_full) {
+          EpiGrad::Params ep;
+          ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
+          ep.lse = p.lse_c; ep.ent = p.ent_c; ep.cp = p.cp_c; ep.ce = p.ce_c;
+          ep.V = (int)V; ep.vocab_base = vocab_base;
+          launch_gemm<EpiGrad, 0, 0>(c, 1, tmHc_k, tmW_k, tm_G_out, sh, ep);
+        } else {
+          EpiGradKL::Params ep;
+          ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
+          ep.lse = p.lse_c; ep.lse_ref = p.lse_ref_c; ep.ent = p.ent_c; ep.kl = p.kl_c;
+          ep.cp = p.cp_c; ep.cb = p.cb_c; ep.ce = p.ce_c;
+          ep.V = (int)V; ep.vocab_base = vocab_base;
+          launch_dual<EpiGradKL>(c, 1, tmHc_k, tmW_k, tmHr_k, tmWr_k, tm_G_out, sh, (int)o.d_ref, ep);
+        }
       }
       // (2) dH_slab (+)= G * W_slab        [rows x d], K = vocabulary columns of the slab
       {

@@ -4,7 +4,7 @@
 // conversion of dH.  All of them are bandwidth- or latency-bound; loads are coalesced and
 // vectorised where a row is wide enough to matter.
 #pragma once
-#include "epilogues.cuh"
+#include "kl_epilogues.cuh"
 
 namespace rlh {
 
@@ -135,6 +135,26 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
     } else {
       for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
       if (lane == 0) tokens_c[i] = -1;
+    }
+  }
+}
+
+// Row compaction of a second hidden-state matrix (the reference model's) with the same row map.
+__global__ void __launch_bounds__(256) gather_plain_kernel(const __nv_bfloat16* __restrict__ H, long long ldH, int d,
+                                                           const int* __restrict__ row_map,
+                                                           __nv_bfloat16* __restrict__ Hc, const DevStatus* st) {
+  const int n = st->n_valid;
+  const int n_pad = (n + 127) / 128 * 128;
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  const int vec_per_row = d / 8;
+  for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < n_pad; i += gridDim.x * warps_per_block) {
+    uint4* dst = reinterpret_cast<uint4*>(Hc + (size_t)i * d);
+    if (i < n) {
+      const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)row_map[i] * ldH);
+      for (int v = lane; v < vec_per_row; v += 32) dst[v] = __ldg(src + v);
+    } else {
+      for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
     }
   }
 }
@@ -273,6 +293,13 @@ struct LossParams {
   const float* token_weight;  // [T] or NULL
   float eps_low, eps_high, beta, ent_coef;
   int with_loss;
+  // full-distribution KL to the reference policy (two-product forward): second partial per
+  // (range, row) = {D, Mr, Sr, 0}; outputs lse_ref, KL_t and the coefficient cb_t = w_t beta
+  const float4* partials2;
+  int kl_full;
+  float* lse_ref_c;
+  float* kl_c;
+  float* cb_c;
   // compact outputs
   float* lse_c;
   float* ent_c;
@@ -283,6 +310,7 @@ struct LossParams {
   float* logp_out;
   float* ent_out;
   float* lse_out;
+  float* kl_out;
   // reduction scratch: [gridDim.x][kLossSums] doubles
   double* block_sums;
 };
@@ -310,7 +338,23 @@ __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossPa
     const float lse = M + logf(S);
     const float logp = zy - lse;
     const float ent = lse - A / S;
+    float kl = 0.f;
+    if (p.kl_full) {
+      float Mr = -CUDART_INF_F;
+      for (int r = 0; r < n_ranges; ++r) Mr = fmaxf(Mr, p.partials2[(size_t)r * p.part_stride + i].y);
+      float D = 0.f, Sr = 0.f;
+      for (int r = 0; r < n_ranges; ++r) {
+        const float4 q2 = p.partials2[(size_t)r * p.part_stride + i];
+        D = fmaf(q2.x, exp2f((p.partials[(size_t)r * p.part_stride + i].x - M) * kLog2e), D);
+        Sr = fmaf(q2.z, exp2f((q2.y - Mr) * kLog2e), Sr);
+      }
+      const float lse_ref = Mr + logf(Sr);
+      kl = (A - D) / S - lse + lse_ref;      // sum_j p_j (z_j - zr_j) - lse + lse_ref
+      p.lse_ref_c[i] = lse_ref;
+      p.kl_c[i] = kl;
+    }
     const int row = p.row_map[i];
+    if (p.kl_out) p.kl_out[row] = kl;
     p.lse_c[i] = lse;
     p.ent_c[i] = ent;
     if (p.logp_c) p.logp_c[i] = logp;
@@ -326,7 +370,10 @@ __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossPa
       const bool active = su <= sc;          // unclipped branch is the minimum (ties: unclipped)
       const float s = active ? su : sc;
       float k3 = 0.f, dk3 = 0.f;
-      if (p.beta != 0.f) {
+      if (p.kl_full) {
+        k3 = kl;                              // its gradient is applied per vocabulary entry (cb)
+        p.cb_c[i] = w * p.beta;
+      } else if (p.beta != 0.f) {
         const float delta = p.ref_logp[row] - logp;
         const float ed = expf(delta);
         k3 = ed - delta - 1.f;

@@ -165,3 +165,23 @@ def make_workload(cfg_id, device=None, prompts=None, L_max=None, seed=None, sigm
     w.n_valid = int(mask.sum().item())
     w.extra = dict(lens=lens, seed=seed)
     return w
+
+
+def make_reference_model(w, d_ref=None, drift=0.05, seed_offset=7919):
+    """Frozen reference model for the full-distribution KL: hidden states H_ref [T, d_ref] and LM head
+    W_ref [V, d_ref] (bf16).  With d_ref equal to the policy's d the reference is the policy before
+    training: the same tensors plus a relative Gaussian drift, the situation of an RL run that started
+    from the reference checkpoint.  With another d_ref it is an unrelated random model of that width
+    with the same logit scale."""
+    dev = w.H.device
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.extra["seed"] + seed_offset)
+    d_ref = w.d if d_ref is None else d_ref
+    if d_ref == w.d:
+        H_ref = (w.H.float() + drift * torch.randn(w.T, w.d, generator=gen, device=dev)).to(torch.bfloat16)
+        W_ref = (w.W.float() * (1.0 + drift * torch.randn(w.V, w.d, generator=gen, device=dev))).to(torch.bfloat16)
+    else:
+        w_std = float(w.W.float().std().item()) * (w.d / d_ref) ** 0.5
+        H_ref = torch.randn(w.T, d_ref, generator=gen, device=dev).to(torch.bfloat16)
+        W_ref = (torch.randn(w.V, d_ref, generator=gen, device=dev) * w_std).to(torch.bfloat16)
+    return H_ref, W_ref

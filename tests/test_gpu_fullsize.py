@@ -110,3 +110,64 @@ def test_full_size_sampled(cfg_id, n_rows, n_cols):
     finally:
         ctx.close()
         torch.cuda.empty_cache()
+
+
+def test_full_size_full_kl():
+    """Config 1 at full size with the full-distribution KL to a reference model (drifted copy of the
+    policy): per-token KL, log-prob, entropy and dH on sampled rows, the loss recomputed in float64
+    from the per-token outputs, and the two identities."""
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload, make_reference_model
+    ctx = Context(0)
+    try:
+        w = make_workload(1)
+        beta, ent_coef = 0.04, 0.001
+        H_ref, W_ref = make_reference_model(w, drift=0.1)
+        adv_seq, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+        out = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, None, adv_tok, w.mask, w.eps_low,
+                                         w.eps_high, beta, ent_coef=ent_coef, H_ref=H_ref, W_ref=W_ref)
+        status, detail = ctx.last_device_status()
+        assert status == 0, (status, hex(detail & 0xffffffff))
+        o_adv_tok = O.broadcast_to_tokens(O.grpo_advantages(w.rewards.cpu().numpy(), w.G),
+                                          w.seq_offsets.cpu().numpy(), w.T)
+        valid = torch.nonzero(w.mask, as_tuple=False)[:, 0].cpu().numpy()
+        N = valid.size
+        rng = np.random.default_rng(977)
+        special = [0, 127, 128, 255, 256, N - 129, N - 1, 32767, 32768]
+        idx = np.unique(np.concatenate([np.array([i for i in special if 0 <= i < N]),
+                                        rng.choice(N, size=160, replace=False)]))
+        rows = valid[idx]
+        W64, Wr64 = _np64(w.W), _np64(W_ref)
+        r = O.dH_rows(_np64(w.H[rows]), W64, w.tokens[rows].cpu().numpy(), _np64(w.old_logp[rows]), None,
+                      o_adv_tok[rows], np.full(rows.size, 1.0 / N), w.eps_low, w.eps_high, beta, ent_coef=ent_coef,
+                      H_ref_rows=_np64(H_ref[rows]), W_ref=Wr64)
+        del W64, Wr64
+        assert r["kl"].mean() > 1e-3
+        assert np.abs(_np64(out["logp"][rows]) - r["logp"]).max() <= TOL_LOGP
+        assert np.abs(_np64(out["entropy"][rows]) - r["entropy"]).max() <= TOL_ENT
+        # KL_t = (A - D)/S - lse + lse_ref in fp32: a few ulp of quantities of size lse (about 12)
+        assert np.abs(_np64(out["kl"][rows]) - r["kl"]).max() <= 2e-3 * np.abs(r["kl"]).max() + 2e-5
+        assert _rel(_np64(out["dH"][rows]), r["dH"]) <= TOL_GRAD_REL
+        masked = torch.nonzero(w.mask == 0, as_tuple=False)[:, 0]
+        if masked.numel():
+            assert not out["dH"][masked[:4096]].any() and not out["kl"][masked[:4096]].any()
+        # loss from the per-token outputs, in float64
+        logp = _np64(out["logp"])[valid]
+        ent = _np64(out["entropy"])[valid]
+        kl = _np64(out["kl"])[valid]
+        s, _, _, _, _ = O.per_token_terms(logp, _np64(w.old_logp)[valid], np.zeros(N), o_adv_tok[valid],
+                                          w.eps_low, w.eps_high, 0.0)
+        loss64 = float(((-s + beta * kl - ent_coef * ent) / N).sum())
+        assert abs(out["loss"].item() - loss64) <= TOL_LOSS_REL * abs(loss64) + 1e-7
+        assert abs(out["metrics"][1].item() - kl.mean()) <= 1e-3 * kl.mean()
+        dW = out["dW"]
+        col_sum = dW.double().sum(dim=0)
+        col_abs = dW.double().abs().sum(dim=0)
+        assert (col_sum.abs() <= 1e-3 * col_abs + 1e-12).all()
+        rowdot = torch.cat([(out["dH"][i:i + 65536].double() * w.H[i:i + 65536].double()).sum(dim=1)
+                            for i in range(0, w.T, 65536)])
+        rhs = (dW.double() * w.W.double()).sum().item()
+        assert abs(rowdot.sum().item() - rhs) <= 1e-2 * rowdot.abs().sum().item()
+    finally:
+        ctx.close()
+        torch.cuda.empty_cache()

@@ -208,6 +208,81 @@ def test_aggregation_modes_and_sequence_level_ratio(ctx, agg_mode, sequence_leve
     _check_against_oracle(ctx, w, agg_mode=agg_mode, sequence_level=sequence_level)
 
 
+@pytest.mark.parametrize("cta_group", [2, 1])
+@pytest.mark.parametrize("cfg_id,prompts,L_max,d_ref,V,ent", [
+    (0, None, None, None, None, 0.0),      # config 0 as it stands, reference = drifted policy
+    (1, 1, 40, 192, 4100, 0.01),           # reference model of another width, ragged vocabulary tail
+    (3, 2, 64, None, 600, 0.0),            # several row slabs and column slabs (limits set below)
+])
+def test_full_distribution_kl(cta_group, cfg_id, prompts, L_max, d_ref, V, ent):
+    """Regulariser = sum_j p_j (log p_j - log q_j) over the whole vocabulary (sections 2.2 / 3.1),
+    q from a second hidden-state / LM-head pair; loss, metrics, dH and dW against the oracle."""
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload, make_reference_model
+    c = Context(0)
+    try:
+        try:
+            c.set_cta_group(cta_group)
+        except RuntimeError:
+            pytest.skip("CTA pairs cannot be co-scheduled on this device")
+        kw = {} if cfg_id == 0 else dict(prompts=prompts, L_max=L_max, d=128, V=V)
+        w = make_workload(cfg_id, **kw)
+        if cfg_id == 3:
+            c.set_slab_limits(128, 256)
+        beta = w.beta if w.beta > 0 else 0.04
+        H_ref, W_ref = make_reference_model(w, d_ref=d_ref, drift=0.3)
+        adv_seq, adv_tok = c.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+        out = c.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, None, adv_tok, w.mask, w.eps_low,
+                                       w.eps_high, beta, ent_coef=ent, H_ref=H_ref, W_ref=W_ref)
+        status, detail = c.last_device_status()
+        assert status == 0, (status, hex(detail & 0xffffffff))
+        o_adv_tok = O.broadcast_to_tokens(O.grpo_advantages(w.rewards.cpu().numpy(), w.G),
+                                          w.seq_offsets.cpu().numpy(), w.T)
+        oo = O.policy_loss_fwd_bwd(_np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), _np64(w.old_logp), None,
+                                   o_adv_tok, w.mask.cpu().numpy(), w.eps_low, w.eps_high, beta, ent_coef=ent,
+                                   H_ref=_np64(H_ref), W_ref=_np64(W_ref))
+        assert oo["kl_mean"] > 1e-4          # the regulariser is really exercised
+        assert np.abs(_np64(out["logp"]) - oo["logp"]).max() <= TOL_LOGP
+        assert np.abs(_np64(out["entropy"]) - oo["entropy"]).max() <= TOL_ENT
+        met = _np64(out["metrics"])
+        # KL_t is a difference of fp32 quantities of the size of lse (about 10): a few ulp of that
+        assert abs(met[1] - oo["kl_mean"]) <= 2e-3 * abs(oo["kl_mean"]) + 5e-6
+        assert abs(out["loss"].item() - oo["loss"]) <= TOL_LOSS_REL * abs(oo["loss"]) + 1e-6
+        m = w.mask.cpu().numpy().astype(bool)
+        dH = _np64(out["dH"])
+        assert not dH[~m].any()
+        assert _rel(dH, oo["dH"]) <= TOL_GRAD_REL
+        assert _rel(_np64(out["dW"]), oo["dW"]) <= TOL_GRAD_REL
+        # the gradient of the regulariser alone (no advantage signal): compare at A = 0
+        zero_adv = torch.zeros_like(adv_tok)
+        out0 = c.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, None, zero_adv, w.mask, w.eps_low,
+                                        w.eps_high, beta, H_ref=H_ref, W_ref=W_ref)
+        oo0 = O.policy_loss_fwd_bwd(_np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), _np64(w.old_logp), None,
+                                    np.zeros(w.T), w.mask.cpu().numpy(), w.eps_low, w.eps_high, beta,
+                                    H_ref=_np64(H_ref), W_ref=_np64(W_ref))
+        assert _rel(_np64(out0["dH"]), oo0["dH"]) <= TOL_GRAD_REL
+        assert _rel(_np64(out0["dW"]), oo0["dW"]) <= TOL_GRAD_REL
+        assert abs(out0["loss"].item() - oo0["loss"]) <= TOL_LOSS_REL * abs(oo0["loss"]) + 1e-6
+    finally:
+        c.close()
+
+
+def test_full_kl_argument_checks(ctx):
+    from paper_2512_21450_b200.workloads import make_workload, make_reference_model
+    w = make_workload(0)
+    H_ref, W_ref = make_reference_model(w)
+    adv = torch.zeros(w.T, device=w.H.device)
+    # not combined with the sequence-level path
+    with pytest.raises(RuntimeError):
+        ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, None, adv, w.mask, 0.2, 0.2, 0.04,
+                                   H_ref=H_ref, W_ref=W_ref, sequence_level=True, seq_offsets=w.seq_offsets)
+    # the reference hidden size must be a whole number of 64-element k-slices
+    with pytest.raises(RuntimeError):
+        ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, None, adv, w.mask, 0.2, 0.2, 0.04,
+                                   H_ref=H_ref[:, :40].contiguous(), W_ref=W_ref[:, :40].contiguous())
+    _assert_status_ok(ctx)
+
+
 def test_clip_exercised_and_peaked_rows(ctx):
     from paper_2512_21450_b200.workloads import make_workload
     w = make_workload(0, sigma_old=0.3, peaked_frac=0.05, seed=77)

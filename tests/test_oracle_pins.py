@@ -544,3 +544,9 @@ def test_full_kl_loss_and_gradient():
     L.backward()
     assert abs(L.item() - out["loss"]) < 1e-13
     assert np.allclose(Ht.grad.numpy(), out["dH"], atol=1e-13) and np.allclose(Wt.grad.numpy(), out["dW"], atol=1e-13)
+    # the sampled-row helper agrees with autograd on a subset of rows, and returns KL_t itself
+    sub = np.array([1, 4, 6])
+    r = O.dH_rows(H[sub], W, tokens[sub], old[sub], None, adv[sub], w[sub], 0.2, 0.2, 0.3, ent_coef=0.02,
+                  H_ref_rows=Hr[sub], W_ref=Wr)
+    assert np.allclose(r["dH"], Ht.grad.numpy()[sub], atol=1e-13)
+    assert np.allclose(r["kl"], kl.detach().numpy()[sub], atol=1e-13)
