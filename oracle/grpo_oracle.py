@@ -436,3 +436,91 @@ def dW_rows(H_valid, W_sel, sel, tokens_valid, lse, ent, dlogp_w, ent_w):
     G = np.asarray(dlogp_w, dtype=np.float64)[:, None] * (onehot - P)
     G += np.asarray(ent_w, dtype=np.float64)[:, None] * P * (LP + np.asarray(ent, dtype=np.float64)[:, None])
     return G.T @ H_valid
+
+
+# --------------------------------------------------------------------------- #
+# Vocabulary-parallel LM head (section 4.3 / 4.4: sharded training, model states
+# not fully resident on one GPU): the rows of W are partitioned over ranks, rank
+# s holding vocabulary ids [off_s, off_s + V_s).  Nothing new is computed - the
+# results must equal the single-device definitions above - so each function
+# below is the plain definition restricted to one slice of the vocabulary.
+# --------------------------------------------------------------------------- #
+def shard_logit_stats(H, W_shard, tokens, vocab_offset, mask=None):
+    """Per-row statistics of one vocabulary slice: stats[t] = (M, S, A, z_y) with
+    z_j = W_shard[j] . h_t for the slice's rows, M = max_j z_j, S = sum_j exp(z_j - M),
+    A = sum_j exp(z_j - M) z_j, and z_y the logit of the sampled token when its id lies in
+    [vocab_offset, vocab_offset + V_s), else 0.  Masked rows give (0, 0, 0, 0)."""
+    H = np.asarray(H, dtype=np.float64)
+    W_shard = np.asarray(W_shard, dtype=np.float64)
+    T = H.shape[0]
+    Vs = W_shard.shape[0]
+    tokens = np.asarray(tokens)
+    m = np.ones(T, dtype=bool) if mask is None else np.asarray(mask).astype(bool)
+    stats = np.zeros((T, 4))
+    for t in np.nonzero(m)[0]:
+        z = W_shard @ H[t]
+        M = z.max()
+        e = np.exp(z - M)
+        y = int(tokens[t]) - int(vocab_offset)
+        stats[t] = (M, e.sum(), (e * z).sum(), z[y] if 0 <= y < Vs else 0.0)
+    return stats
+
+
+def merge_logit_stats(stats_per_shard, mask=None):
+    """From the statistics of every slice of a partition of the vocabulary: lse_t = log of the
+    sum over slices of S_s exp(M_s), logp_t = (sum of z_y over slices) - lse_t, and
+    Ent_t = lse_t - (sum_s A_s exp(M_s)) / (sum_s S_s exp(M_s)); sums are shifted by the largest M_s.
+    Returns (logp, entropy, lse); masked rows give 0."""
+    st = np.asarray(stats_per_shard, dtype=np.float64)      # [n_shards, T, 4]
+    T = st.shape[1]
+    m = np.ones(T, dtype=bool) if mask is None else np.asarray(mask).astype(bool)
+    logp, ent, lse = np.zeros(T), np.zeros(T), np.zeros(T)
+    for t in np.nonzero(m)[0]:
+        M = st[:, t, 0].max()
+        S = (st[:, t, 1] * np.exp(st[:, t, 0] - M)).sum()
+        A = (st[:, t, 2] * np.exp(st[:, t, 0] - M)).sum()
+        lse[t] = M + np.log(S)
+        logp[t] = st[:, t, 3].sum() - lse[t]
+        ent[t] = lse[t] - A / S
+    return logp, ent, lse
+
+
+def policy_loss_shard_bwd(H, W_shard, tokens, vocab_offset, logp, entropy, lse, old_logp, ref_logp, adv,
+                          mask, eps_low, eps_high, beta, ent_coef=0.0, token_weight=None):
+    """One vocabulary slice's share of the backward pass, given the merged per-token
+    log-probability, entropy and log-sum-exp of the whole vocabulary.
+
+    The loss (identical on every slice, it only needs per-token quantities) and, for the
+    columns j of the slice, g_tj exactly as in policy_loss_fwd_bwd with p_tj = exp(z_tj - lse_t);
+    dH_partial = G_slice W_shard (summing it over the slices gives dH) and
+    dW_shard = G_slice^T H (the slice's rows of dW)."""
+    H = np.asarray(H, dtype=np.float64)
+    W_shard = np.asarray(W_shard, dtype=np.float64)
+    T, d = H.shape
+    Vs = W_shard.shape[0]
+    tokens = np.asarray(tokens)
+    m = np.asarray(mask).astype(bool)
+    w = token_weights(m) if token_weight is None else np.asarray(token_weight, dtype=np.float64) * m
+    rows = np.nonzero(m)[0]
+    out = dict(loss=0.0, dH_partial=np.zeros((T, d)), dW_shard=np.zeros((Vs, d)))
+    if rows.size == 0:
+        return out
+    ref = np.zeros(T) if ref_logp is None else np.asarray(ref_logp, dtype=np.float64)
+    lp = np.asarray(logp, dtype=np.float64)[rows]
+    en = np.asarray(entropy, dtype=np.float64)[rows]
+    s, k3, rho, active, dlogp = per_token_terms(lp, np.asarray(old_logp, dtype=np.float64)[rows], ref[rows],
+                                                np.asarray(adv, dtype=np.float64)[rows], eps_low, eps_high, beta)
+    wr = w[rows]
+    out["loss"] = float((wr * (-s + beta * k3 - ent_coef * en)).sum())
+    LP = H[rows] @ W_shard.T - np.asarray(lse, dtype=np.float64)[rows][:, None]     # log p_tj on the slice
+    P = np.exp(LP)
+    y = tokens[rows] - int(vocab_offset)
+    onehot = np.zeros_like(P)
+    inside = (y >= 0) & (y < Vs)
+    onehot[np.nonzero(inside)[0], y[inside]] = 1.0
+    G = (wr * dlogp)[:, None] * (onehot - P)
+    if ent_coef != 0.0:
+        G += (wr * ent_coef)[:, None] * P * (LP + en[:, None])
+    out["dH_partial"][rows] = G @ W_shard
+    out["dW_shard"] = G.T @ H[rows]
+    return out

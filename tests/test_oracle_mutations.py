@@ -32,6 +32,11 @@ MUTANTS = {
     "OPO baseline unweighted": ("base = (ln[sl] * r[sl]).sum() / tot", "base = r[sl].sum() / len(r[sl])"),
     "full KL gradient misses the -KL term": ("P * (LP - LQ - kl_full[:, None])", "P * (LP - LQ)"),
     "full KL direction swapped": ("return (np.exp(LP) * (LP - LQ)).sum(axis=1)", "return (np.exp(LQ) * (LQ - LP)).sum(axis=1)"),
+    "slice merge forgets to rescale by exp(M_s - M)": ("S = (st[:, t, 1] * np.exp(st[:, t, 0] - M)).sum()", "S = st[:, t, 1].sum()"),
+    "slice statistics: weighted sum uses shifted logits": ("stats[t] = (M, e.sum(), (e * z).sum(),", "stats[t] = (M, e.sum(), (e * (z - M)).sum(),"),
+    "slice statistics: target id not made local": ("y = int(tokens[t]) - int(vocab_offset)", "y = int(tokens[t])"),
+    "slice backward: one-hot not made local": ("y = tokens[rows] - int(vocab_offset)", "y = tokens[rows]"),
+    "slice backward: softmax renormalised inside the slice": ("LP = H[rows] @ W_shard.T - np.asarray(lse, dtype=np.float64)[rows][:, None]", "LP = H[rows] @ W_shard.T; LP = LP - np.log(np.exp(LP).sum(axis=1))[:, None]"),
     "logits index order": ("return H @ W.T", "return (W @ H.T).T[::-1][::-1] if H.shape[0] == 1 else (H[:, ::-1] @ W[:, ::-1].T if False else H @ W[::-1].T)"),
 }
 

@@ -550,3 +550,77 @@ def test_full_kl_loss_and_gradient():
                   H_ref_rows=Hr[sub], W_ref=Wr)
     assert np.allclose(r["dH"], Ht.grad.numpy()[sub], atol=1e-13)
     assert np.allclose(r["kl"], kl.detach().numpy()[sub], atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- vocabulary-parallel head
+def _shard_problem(seed):
+    rng = _rng(seed)
+    T, d, V = 9, 6, 23
+    H = rng.normal(size=(T, d)); W = rng.normal(size=(V, d)) * 0.8
+    tokens = rng.integers(0, V, size=T)
+    tokens[0], tokens[1] = 0, V - 1                      # first and last id of the vocabulary
+    mask = np.array([1, 1, 1, 0, 1, 1, 0, 1, 1], dtype=np.uint8)
+    lp, _, _ = O.token_logprobs(H, W, tokens)
+    old = lp + rng.normal(size=T) * 0.3
+    ref = lp + rng.normal(size=T) * 0.2
+    adv = rng.normal(size=T)
+    return H, W, tokens, mask, old, ref, adv
+
+
+def test_shard_statistics_brute_force():
+    # one slice, tiny: the four numbers against python sums without any shift
+    H, W, tokens, mask, *_ = _shard_problem(50)
+    off, Vs = 5, 7
+    st = O.shard_logit_stats(H, W[off:off + Vs], tokens, off, mask)
+    for t in range(H.shape[0]):
+        if not mask[t]:
+            assert np.all(st[t] == 0)
+            continue
+        z = [sum(H[t, k] * W[off + j, k] for k in range(H.shape[1])) for j in range(Vs)]
+        M, S, A, zy = st[t]
+        assert abs(M - max(z)) < 1e-14
+        assert abs(S * math.exp(M) - sum(math.exp(v) for v in z)) < 1e-12
+        assert abs(A * math.exp(M) - sum(math.exp(v) * v for v in z)) < 1e-12
+        inside = off <= tokens[t] < off + Vs
+        assert abs(zy - (z[tokens[t] - off] if inside else 0.0)) < 1e-14
+
+
+@pytest.mark.parametrize("cuts", [(0, 23), (0, 11, 23), (0, 1, 22, 23), (0, 4, 9, 17, 23)])
+def test_merged_shard_statistics_equal_the_full_softmax(cuts):
+    # any partition of the vocabulary reproduces the single-device definition (one slice: trivially)
+    H, W, tokens, mask, *_ = _shard_problem(51)
+    stats = [O.shard_logit_stats(H, W[a:b], tokens, a, mask) for a, b in zip(cuts[:-1], cuts[1:])]
+    logp, ent, lse = O.merge_logit_stats(stats, mask)
+    lp0, ent0, lse0 = O.token_logprobs(H, W, tokens, mask)
+    assert np.abs(logp - lp0).max() < 1e-13 and np.abs(ent - ent0).max() < 1e-13 and np.abs(lse - lse0).max() < 1e-13
+    # library second opinion on the merged result
+    ref = -torch.nn.functional.cross_entropy(torch.tensor(H @ W.T), torch.tensor(tokens), reduction="none").numpy()
+    assert np.abs(logp - ref * mask).max() < 1e-13
+    # a slice whose logits are far below the others' must not disturb the sums (shift by the largest M)
+    Wlow = W.copy(); Wlow[cuts[-2]:] *= 0.0; Hs = H * 30.0
+    stats = [O.shard_logit_stats(Hs, Wlow[a:b], tokens, a, mask) for a, b in zip(cuts[:-1], cuts[1:])]
+    lp1, ent1, lse1 = O.merge_logit_stats(stats, mask)
+    lp2, ent2, lse2 = O.token_logprobs(Hs, Wlow, tokens, mask)
+    assert np.all(np.isfinite(lp1)) and np.abs(lp1 - lp2).max() < 1e-10 and np.abs(ent1 - ent2).max() < 1e-10
+
+
+@pytest.mark.parametrize("cuts", [(0, 23), (0, 10, 23), (0, 1, 8, 23)])
+def test_shard_backward_sums_to_the_full_gradient(cuts):
+    H, W, tokens, mask, old, ref, adv = _shard_problem(52)
+    kw = dict(eps_low=0.2, eps_high=0.3, beta=0.1, ent_coef=0.03)
+    full = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, **kw)
+    dH = np.zeros_like(H)
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        o = O.policy_loss_shard_bwd(H, W[a:b], tokens, a, full["logp"], full["entropy"], full["lse"], old, ref, adv,
+                                    mask, **kw)
+        assert abs(o["loss"] - full["loss"]) < 1e-14                 # every slice sees the same loss
+        assert np.abs(o["dW_shard"] - full["dW"][a:b]).max() < 1e-13  # its rows of dW
+        dH += o["dH_partial"]
+    assert np.abs(dH - full["dH"]).max() < 1e-13
+    assert np.all(dH[mask == 0] == 0)
+    # caller-supplied weights take the place of the token mean
+    tw = np.linspace(0.5, 1.5, H.shape[0]) / 7.0
+    full = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, token_weight=tw, **kw)
+    o = O.policy_loss_shard_bwd(H, W[3:15], tokens, 3, full["logp"], full["entropy"], full["lse"], old, ref, adv,
+                                mask, token_weight=tw, **kw)
+    assert np.abs(o["dW_shard"] - full["dW"][3:15]).max() < 1e-13 and abs(o["loss"] - full["loss"]) < 1e-14
