@@ -216,6 +216,58 @@ rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* ctx, const void* H_host, int64_t l
                                       float eps_low, float eps_high, float beta, float ent_coef,
                                       float* loss_host, float* metrics_host, void* dH, float* dW);
 
+/* Scoring with several models in one call - Algorithm 1 evaluates the same sampled tokens under
+ * the old policy pi_theta_old ("update the old policy model", importance-ratio denominator of
+ * section 2.2) and under the frozen reference pi_ref (section 3.2.1, Reference role) before the
+ * update.  Model i has hidden states H[i] ([T, d[i]] bf16, row stride ldH[i]) and LM head W[i]
+ * ([V, d[i]] bf16, row stride ldW[i]); tokens, mask, T and V are shared.  The arrays H, ldH, W,
+ * ldW, d, logp, entropy are HOST arrays of n_models (1..16) entries holding device pointers /
+ * sizes; logp[i][T] required, entropy (the array, or single entries) may be NULL.  The mask is
+ * scanned once and every model reuses the row map; each model then takes one sweep over its own
+ * W.  Workspace: rl_workspace_bytes() with the largest d[i].  Errors as rl_token_logprobs. */
+rl_status rl_token_logprobs_multi(rl_ctx* ctx, int n_models, const void* const* H, const int64_t* ldH,
+                                  const void* const* W, const int64_t* ldW, const int64_t* d,
+                                  const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t V,
+                                  float* const* logp, float* const* entropy);
+
+/* Vocabulary-parallel LM head - for training engines that shard the model states so that the
+ * head weight is never resident on one GPU in full (section 4.3 "finer-grained control over
+ * sharding behavior", section 4.4 "model states do not need to be fully resident on a single
+ * GPU").  The rows of W are partitioned over ranks; this rank holds W_shard[V_shard, d] =
+ * rows [vocab_offset, vocab_offset + V_shard) of the V_total-row head.  tokens are ids in
+ * [0, V_total) (checked against V_total; an id outside this rank's slice simply has no logit
+ * here).  The three calls compute exactly what rl_token_logprobs and rl_policy_loss_fwd_bwd_ex
+ * compute on one device; between them the caller moves 16 bytes per row (all-gather of the
+ * statistics) and the partial dH (all-reduce).
+ *
+ * rl_shard_logit_stats: stats[T][4] (fp32, 16-byte aligned) receives per row (M, S, A, z_y) over the
+ *   slice: M = max_j z_j, S = sum_j exp(z_j - M), A = sum_j exp(z_j - M) z_j, z_y = the logit of
+ *   the sampled token if its id lies in the slice, else 0.  Masked rows get four zeros.
+ * rl_merge_logit_stats: stats[n_shards][T][4] -> logp[T], entropy[T] (may be NULL), lse[T] (may be
+ *   NULL) over the whole vocabulary; masked rows 0.  Slices are combined in index order, so every
+ *   rank that merges the same gathered array gets the same bits.
+ * rl_policy_loss_shard_bwd: arguments as rl_policy_loss_fwd_bwd_ex plus the slice position and the
+ *   merged logp, entropy, lse ([T] each, as rl_merge_logit_stats wrote them).  loss[1] is the loss
+ *   of the whole vocabulary (every rank computes the same value: do not sum it over ranks);
+ *   dH_partial[T,d] is this slice's contribution to dH (sum over ranks = dH; ask for fp32 with
+ *   opts->dH_dtype = 1 when it is to be all-reduced); dW_shard[V_shard,d] is this rank's rows of dW.
+ *   opts->kl_full is not supported here (RL_ERR_INVALID_ARG).
+ * Errors: vocab_offset < 0 or vocab_offset + V_shard > V_total -> RL_ERR_SHAPE; the rest as the
+ * single-device calls.  Workspace: rl_workspace_bytes(T, d, V_shard). */
+rl_status rl_shard_logit_stats(rl_ctx* ctx, const void* H, int64_t ldH, const void* W_shard, int64_t ldW,
+                               const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d,
+                               int64_t V_shard, int64_t vocab_offset, int64_t V_total, float* stats);
+rl_status rl_merge_logit_stats(rl_ctx* ctx, const float* stats, int n_shards, const uint8_t* mask,
+                               int64_t T, float* logp, float* entropy, float* lse);
+rl_status rl_policy_loss_shard_bwd(rl_ctx* ctx, const void* H, int64_t ldH, const void* W_shard,
+                                   int64_t ldW, const int32_t* tokens, const float* old_logp,
+                                   const float* ref_logp, const float* adv, const uint8_t* mask,
+                                   int64_t T, int64_t d, int64_t V_shard, int64_t vocab_offset,
+                                   int64_t V_total, const float* logp, const float* entropy,
+                                   const float* lse, float eps_low, float eps_high, float beta,
+                                   float* loss, void* dH_partial, float* dW_shard,
+                                   const rl_loss_opts* opts);
+
 /* rl_token_logprobs without any device allocation and without a context (the paper has no
  * counterpart).  It is meant for callers that cannot allocate GPU memory when they need
  * log-probabilities: a scoring pass that shares the GPU with a rollout engine which has already

@@ -99,6 +99,18 @@ def load_library():
     lib.rl_selftest_gemm.argtypes = [P, P, P, P, c_int64, c_int64, c_int64, c_int, c_int, c_int]
     lib.rl_token_logprobs_static.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P, P]
     lib.rl_token_logprobs_static.restype = c_int
+    lib.rl_token_logprobs_multi.argtypes = [P, c_int, POINTER(c_void_p), POINTER(c_int64), POINTER(c_void_p),
+                                            POINTER(c_int64), POINTER(c_int64), P, P, c_int64, c_int64,
+                                            POINTER(c_void_p), POINTER(c_void_p)]
+    lib.rl_token_logprobs_multi.restype = c_int
+    lib.rl_shard_logit_stats.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, c_int64, c_int64, P]
+    lib.rl_shard_logit_stats.restype = c_int
+    lib.rl_merge_logit_stats.argtypes = [P, P, c_int, P, c_int64, P, P, P]
+    lib.rl_merge_logit_stats.restype = c_int
+    lib.rl_policy_loss_shard_bwd.argtypes = [P, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int64, c_int64,
+                                             c_int64, c_int64, P, P, P, c_float, c_float, c_float, P, P, P,
+                                             POINTER(rl_loss_opts)]
+    lib.rl_policy_loss_shard_bwd.restype = c_int
     for name in ("rl_create", "rl_destroy", "rl_set_stream", "rl_workspace_bytes", "rl_workspace_bytes_host",
                  "rl_workspace_bytes_kl",
                  "rl_set_workspace", "rl_set_slab_limits", "rl_last_device_status", "rl_grpo_advantages", "rl_grpo_advantages_ex",
@@ -286,6 +298,96 @@ class Context:
                 opts.kl_out = out["kl"].data_ptr()
         _check(self.lib.rl_policy_loss_fwd_bwd_ex(*args, byref(opts)), "rl_policy_loss_fwd_bwd_ex")
         return out
+
+    def rl_token_logprobs_multi(self, Hs, Ws, tokens, mask=None, want_entropy=True):
+        """Log-probabilities of the same tokens under several models (e.g. old policy and reference):
+        lists of H [T, d_i] and W [V, d_i]; returns (list of logp, list of entropy or None)."""
+        self._bind_stream()
+        n = len(Hs)
+        assert n == len(Ws) and n >= 1
+        T, V = Hs[0].shape[0], Ws[0].shape[0]
+        for H, W in zip(Hs, Ws):
+            assert H.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and H.shape[0] == T and W.shape[0] == V
+            assert H.stride(1) == 1 and W.stride(1) == 1 and H.shape[1] == W.shape[1]
+        assert tokens.dtype == torch.int32
+        self.ensure_workspace(T, max(W.shape[1] for W in Ws), V)
+        dev = Ws[0].device
+        logp = [torch.empty(T, dtype=torch.float32, device=dev) for _ in range(n)]
+        ent = [torch.empty(T, dtype=torch.float32, device=dev) for _ in range(n)] if want_entropy else None
+        arr_p = lambda ts: (c_void_p * n)(*[t.data_ptr() if t.numel() else None for t in ts])  # noqa: E731
+        arr_i = lambda xs: (c_int64 * n)(*xs)  # noqa: E731
+        _check(self.lib.rl_token_logprobs_multi(
+            self.handle, n, arr_p(Hs), arr_i([H.stride(0) if T else H.shape[1] for H in Hs]), arr_p(Ws),
+            arr_i([W.stride(0) for W in Ws]), arr_i([W.shape[1] for W in Ws]), _ptr(tokens), _ptr(mask), T, V,
+            arr_p(logp), arr_p(ent) if ent is not None else None), "rl_token_logprobs_multi")
+        return logp, ent
+
+    # ------------------------------------------------------------------ vocabulary-parallel head
+    def rl_shard_logit_stats(self, H, W_shard, tokens, mask, vocab_offset, V_total, stats=None):
+        """Per-row (M, S, A, z_y) over this rank's rows of the head; stats [T, 4] fp32."""
+        self._bind_stream()
+        T, d = H.shape
+        Vs = W_shard.shape[0]
+        assert H.dtype == torch.bfloat16 and W_shard.dtype == torch.bfloat16 and tokens.dtype == torch.int32
+        assert H.stride(1) == 1 and W_shard.stride(1) == 1
+        self.ensure_workspace(T, d, Vs)
+        if stats is None:
+            stats = torch.empty(T, 4, dtype=torch.float32, device=H.device)
+        assert stats.dtype == torch.float32 and stats.is_contiguous() and stats.numel() == 4 * T
+        _check(self.lib.rl_shard_logit_stats(self.handle, _ptr(H), H.stride(0) if T else d, _ptr(W_shard),
+                                             W_shard.stride(0), _ptr(tokens), _ptr(mask), T, d, Vs, vocab_offset,
+                                             V_total, _ptr(stats)), "rl_shard_logit_stats")
+        return stats
+
+    def rl_merge_logit_stats(self, stats, mask=None):
+        """stats [n_shards, T, 4] (all slices of the vocabulary) -> (logp, entropy, lse), each [T]."""
+        self._bind_stream()
+        assert stats.dtype == torch.float32 and stats.is_contiguous() and stats.dim() == 3 and stats.shape[2] == 4
+        n_shards, T = stats.shape[0], stats.shape[1]
+        logp = torch.empty(T, dtype=torch.float32, device=stats.device)
+        ent = torch.empty_like(logp)
+        lse = torch.empty_like(logp)
+        _check(self.lib.rl_merge_logit_stats(self.handle, _ptr(stats), n_shards, _ptr(mask), T, _ptr(logp), _ptr(ent),
+                                             _ptr(lse)), "rl_merge_logit_stats")
+        return logp, ent, lse
+
+    def rl_policy_loss_shard_bwd(self, H, W_shard, tokens, old_logp, ref_logp, adv, mask, vocab_offset, V_total,
+                                 logp, entropy, lse, eps_low, eps_high, beta, ent_coef=0.0, token_weight=None,
+                                 dH_fp32=True, accumulate_dW=False, dW=None, dH=None, agg_mode=0,
+                                 sequence_level=False, seq_offsets=None):
+        """This rank's share of the backward pass given the merged per-token statistics: returns
+        dict(loss (whole vocabulary, same on every rank), dH (partial: sum over ranks), dW (its rows))."""
+        self._bind_stream()
+        T, d = H.shape
+        Vs = W_shard.shape[0]
+        assert H.dtype == torch.bfloat16 and W_shard.dtype == torch.bfloat16 and tokens.dtype == torch.int32
+        assert H.stride(1) == 1 and W_shard.stride(1) == 1
+        for x in (logp, entropy, lse):
+            assert x.dtype == torch.float32 and x.is_contiguous() and x.numel() == T
+        self.ensure_workspace(T, d, Vs)
+        dev = W_shard.device
+        loss = torch.empty(1, dtype=torch.float32, device=dev)
+        if dH is None:
+            dH = torch.empty(T, d, dtype=torch.float32 if dH_fp32 else torch.bfloat16, device=dev)
+        if dW is None:
+            dW = torch.empty(Vs, d, dtype=torch.float32, device=dev)
+        opts = rl_loss_opts()
+        opts.struct_size = ctypes.sizeof(rl_loss_opts)
+        opts.ent_coef = ent_coef
+        opts.token_weight = token_weight.data_ptr() if token_weight is not None else None
+        opts.accumulate_dW = int(accumulate_dW)
+        opts.agg_mode = agg_mode
+        opts.sequence_level = int(sequence_level)
+        opts.dH_dtype = int(dH.dtype == torch.float32)
+        if seq_offsets is not None:
+            opts.seq_offsets = seq_offsets.data_ptr()
+            opts.n_seq = seq_offsets.numel() - 1
+        _check(self.lib.rl_policy_loss_shard_bwd(
+            self.handle, _ptr(H), H.stride(0) if T else d, _ptr(W_shard), W_shard.stride(0), _ptr(tokens),
+            _ptr(old_logp), _ptr(ref_logp), _ptr(adv), _ptr(mask), T, d, Vs, vocab_offset, V_total, _ptr(logp),
+            _ptr(entropy), _ptr(lse), eps_low, eps_high, beta, _ptr(loss), _ptr(dH), _ptr(dW), byref(opts)),
+            "rl_policy_loss_shard_bwd")
+        return dict(loss=loss, dH=dH, dW=dW)
 
     def selftest_wait_timeout(self, limit_ms=20):
         self._bind_stream()

@@ -276,17 +276,34 @@ rl_status check_ws(rl_ctx* c, const WsLayout& L) {
   return RL_OK;
 }
 
+// Vocabulary-parallel call: W holds the vocabulary ids [vocab_off, vocab_off + V) of V_total and the
+// per-token statistics of the whole vocabulary come from the caller.
+struct ShardArgs {
+  int64_t vocab_off, V_total;
+  const float* logp;
+  const float* entropy;
+  const float* lse;
+};
+
 inline rl_status cuda_ok() { return cudaGetLastError() == cudaSuccess ? RL_OK : RL_ERR_CUDA; }
+
+// Which part of the forward stage a call needs, and where its rows of W sit in the vocabulary.
+struct FwdPlan {
+  bool scan = true;          // mask scan (false: the row map of an earlier call on this workspace is reused)
+  bool stats = true;         // tensor-core pass that leaves per-range statistics in the workspace
+  int64_t vocab_off = 0;     // first vocabulary id of W's rows (vocabulary-parallel head)
+  int64_t V_total = 0;       // size of the whole vocabulary for the token-range check (0: V)
+};
 
 // Mask scan + row compaction + forward statistics.  Leaves per-range partials in the workspace.
 rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, const void* W, int64_t ldW,
                       const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
-                      GemmShape* shape_out, const KlRef* kl = nullptr) {
+                      GemmShape* shape_out, const KlRef* kl = nullptr, const FwdPlan& plan = FwdPlan()) {
   char* ws = static_cast<char*>(c->ws);
   int* row_map = reinterpret_cast<int*>(ws + L.row_map);
   int* tokens_c = reinterpret_cast<int*>(ws + L.tokens_c);
   __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + L.Hc);
-  {
+  if (plan.scan) {
     const int pr = prof_begin(c, 4);
     int* block_counts = reinterpret_cast<int*>(ws + L.scan_counts);
     const int n_blocks = (int)((T + kScanRowsPerBlock - 1) / kScanRowsPerBlock);
@@ -294,12 +311,18 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
     mask_offsets_kernel<<<1, 1024, 0, c->stream>>>(block_counts, n_blocks, c->dstatus);
     mask_write_kernel<<<n_blocks, kScanThreads, 0, c->stream>>>(mask, (int)T, block_counts, row_map);
     prof_end(c, pr, 4);
+    c->launches += 3;
   }
   const int pr_gather = prof_begin(c, 5);
   gather_rows_kernel<<<c->n_sm * 4, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16*>(H), ldH, (int)d, row_map,
-                                                         tokens, (int)V, Hc, tokens_c, c->dstatus);
+                                                         tokens, (int)(plan.V_total > 0 ? plan.V_total : V),
+                                                         (int)plan.vocab_off, Hc, tokens_c, c->dstatus);
   prof_end(c, pr_gather, 5);
-  c->launches += 4;
+  c->launches += 1;
+  if (!plan.stats) {
+    memset(shape_out, 0, sizeof(*shape_out));
+    return cuda_ok();
+  }
   CUtensorMap tmA, tmB;
   if (!map_kmajor(c, &tmA, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, BM)) return RL_ERR_CUDA;
   if (!map_kmajor(c, &tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)ldW, b_box_rows(c))) return RL_ERR_CUDA;
@@ -631,11 +654,12 @@ rl_status rl_token_logprobs(rl_ctx* c, const void* H, int64_t ldH, const void* W
   return cuda_ok();
 }
 
-rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const void* W, int64_t ldW,
-                                    const int32_t* tokens, const float* old_logp, const float* ref_logp,
-                                    const float* adv, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
-                                    float eps_low, float eps_high, float beta, float* loss, void* dH, float* dW,
-                                    const rl_loss_opts* opts) {
+// Body of rl_policy_loss_fwd_bwd_ex (shard == NULL) and of rl_policy_loss_shard_bwd.
+static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const void* W, int64_t ldW,
+                                   const int32_t* tokens, const float* old_logp, const float* ref_logp,
+                                   const float* adv, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
+                                   float eps_low, float eps_high, float beta, float* loss, void* dH, float* dW,
+                                   const rl_loss_opts* opts, const ShardArgs* shard) {
   if (!c) return RL_ERR_INVALID_ARG;
   rl_status s = check_hw(H, ldH, W, ldW, T, d, V);
   if (s != RL_OK) return s;
@@ -659,6 +683,12 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   const bool seq_path = o.sequence_level || (o.agg_mode != 0 && !o.token_weight);
   KlRef klref;
   memset(&klref, 0, sizeof(klref));
+  if (shard) {
+    if (o.kl_full) return RL_ERR_INVALID_ARG;
+    if (shard->vocab_off < 0 || shard->V_total < shard->vocab_off + V || shard->V_total >= (int64_t(1) << 30))
+      return RL_ERR_SHAPE;
+    if (T > 0 && (!shard->logp || !shard->entropy || !shard->lse)) return RL_ERR_INVALID_ARG;
+  }
   if (o.kl_full) {
     if (seq_path) return RL_ERR_INVALID_ARG;
     if (!o.W_ref || (T > 0 && !o.H_ref) || o.d_ref <= 0) return RL_ERR_INVALID_ARG;
@@ -687,7 +717,14 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
 
   // ---- forward: statistics per (row, vocabulary range)
   GemmShape fwd_shape;
-  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &fwd_shape, o.kl_full ? &klref : nullptr)) !=
+  FwdPlan plan;
+  if (shard) {
+    // the statistics of the whole vocabulary are given: only the row compaction is needed
+    plan.stats = false;
+    plan.vocab_off = shard->vocab_off;
+    plan.V_total = shard->V_total;
+  }
+  if ((s = run_forward(c, L, H, ldH, W, ldW, tokens, mask, T, d, V, &fwd_shape, o.kl_full ? &klref : nullptr, plan)) !=
       RL_OK)
     return s;
 
@@ -716,6 +753,11 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
   p.logp_out = o.logp_out;
   p.ent_out = o.entropy_out;
   p.block_sums = reinterpret_cast<double*>(ws + L.block_sums);
+  if (shard) {
+    p.ext_logp = shard->logp;
+    p.ext_ent = shard->entropy;
+    p.ext_lse = shard->lse;
+  }
   if (o.kl_full) {
     p.kl_full = 1;
     p.partials2 = reinterpret_cast<const float4*>(ws + L.partials2);
@@ -872,6 +914,132 @@ rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const
                                                      c->grid[c->cta_group] / c->cta_group, (long long)L.Ts * d, row_map,
                                                      static_cast<__nv_bfloat16*>(dH), c->dstatus);
     prof_end(c, pr_sc, 7);
+    c->launches++;
+  }
+  return cuda_ok();
+}
+
+rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* c, const void* H, int64_t ldH, const void* W, int64_t ldW,
+                                    const int32_t* tokens, const float* old_logp, const float* ref_logp,
+                                    const float* adv, const uint8_t* mask, int64_t T, int64_t d, int64_t V,
+                                    float eps_low, float eps_high, float beta, float* loss, void* dH, float* dW,
+                                    const rl_loss_opts* opts) {
+  return loss_fwd_bwd_impl(c, H, ldH, W, ldW, tokens, old_logp, ref_logp, adv, mask, T, d, V, eps_low, eps_high, beta,
+                           loss, dH, dW, opts, nullptr);
+}
+
+rl_status rl_policy_loss_shard_bwd(rl_ctx* c, const void* H, int64_t ldH, const void* W_shard, int64_t ldW,
+                                   const int32_t* tokens, const float* old_logp, const float* ref_logp,
+                                   const float* adv, const uint8_t* mask, int64_t T, int64_t d, int64_t V_shard,
+                                   int64_t vocab_offset, int64_t V_total, const float* logp, const float* entropy,
+                                   const float* lse, float eps_low, float eps_high, float beta, float* loss,
+                                   void* dH_partial, float* dW_shard, const rl_loss_opts* opts) {
+  ShardArgs sh;
+  sh.vocab_off = vocab_offset;
+  sh.V_total = V_total;
+  sh.logp = logp;
+  sh.entropy = entropy;
+  sh.lse = lse;
+  return loss_fwd_bwd_impl(c, H, ldH, W_shard, ldW, tokens, old_logp, ref_logp, adv, mask, T, d, V_shard, eps_low,
+                           eps_high, beta, loss, dH_partial, dW_shard, opts, &sh);
+}
+
+rl_status rl_shard_logit_stats(rl_ctx* c, const void* H, int64_t ldH, const void* W_shard, int64_t ldW,
+                               const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t d, int64_t V_shard,
+                               int64_t vocab_offset, int64_t V_total, float* stats) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  rl_status s = check_hw(H, ldH, W_shard, ldW, T, d, V_shard);
+  if (s != RL_OK) return s;
+  if (vocab_offset < 0 || V_total < vocab_offset + V_shard || V_total >= (int64_t(1) << 30)) return RL_ERR_SHAPE;
+  if (T == 0) return RL_OK;
+  if (!tokens || !stats) return RL_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(stats) & 15) return RL_ERR_ALIGNMENT;
+  const WsLayout L = ws_layout(c, T, d, V_shard, false);
+  if ((s = check_ws(c, L)) != RL_OK) return s;
+  char* ws = static_cast<char*>(c->ws);
+  cudaMemsetAsync(stats, 0, (size_t)T * 16, c->stream);
+  GemmShape fwd_shape;
+  FwdPlan plan;
+  plan.vocab_off = vocab_offset;
+  plan.V_total = V_total;
+  if ((s = run_forward(c, L, H, ldH, W_shard, ldW, tokens, mask, T, d, V_shard, &fwd_shape, nullptr, plan)) != RL_OK)
+    return s;
+  LossParams p;
+  memset(&p, 0, sizeof(p));
+  p.partials = reinterpret_cast<const float4*>(ws + L.partials);
+  p.part_stride = L.Tpad;
+  p.fwd_shape = fwd_shape;
+  p.fwd_cg = c->cta_group;
+  p.fwd_workers = c->grid[c->cta_group] / c->cta_group;
+  p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
+  p.stats_out = reinterpret_cast<float4*>(stats);
+  int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
+  if (blocks > 1024) blocks = 1024;
+  const int pr = prof_begin(c, 6);
+  combine_loss_kernel<<<blocks, kLossThreads, 0, c->stream>>>(p, c->dstatus);
+  prof_end(c, pr, 6);
+  c->launches++;
+  return cuda_ok();
+}
+
+rl_status rl_merge_logit_stats(rl_ctx* c, const float* stats, int n_shards, const uint8_t* mask, int64_t T,
+                               float* logp, float* entropy, float* lse) {
+  if (!c || T < 0 || n_shards < 1 || n_shards > 4096) return RL_ERR_INVALID_ARG;
+  if (T == 0) return RL_OK;
+  if (!stats || !logp) return RL_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(stats) & 15) return RL_ERR_ALIGNMENT;
+  int blocks = (int)((T + 255) / 256);
+  if (blocks > 4096) blocks = 4096;
+  const int pr = prof_begin(c, 6);
+  merge_shard_stats_kernel<<<blocks, 256, 0, c->stream>>>(reinterpret_cast<const float4*>(stats), n_shards,
+                                                          (long long)T, mask, logp, entropy, lse);
+  prof_end(c, pr, 6);
+  c->launches++;
+  return cuda_ok();
+}
+
+rl_status rl_token_logprobs_multi(rl_ctx* c, int n_models, const void* const* H, const int64_t* ldH,
+                                  const void* const* W, const int64_t* ldW, const int64_t* d,
+                                  const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t V,
+                                  float* const* logp, float* const* entropy) {
+  if (!c || n_models < 1 || n_models > 16 || !H || !ldH || !W || !ldW || !d || !logp) return RL_ERR_INVALID_ARG;
+  int64_t d_max = 0;
+  for (int i = 0; i < n_models; ++i) {
+    rl_status s = check_hw(H[i], ldH[i], W[i], ldW[i], T, d[i], V);
+    if (s != RL_OK) return s;
+    if (T > 0 && !logp[i]) return RL_ERR_INVALID_ARG;
+    d_max = d[i] > d_max ? d[i] : d_max;
+  }
+  if (T == 0) return RL_OK;
+  if (!tokens) return RL_ERR_INVALID_ARG;
+  // one layout for all models: the compacted rows of the widest model fix the offsets
+  const WsLayout L = ws_layout(c, T, d_max, V, false);
+  rl_status s = check_ws(c, L);
+  if (s != RL_OK) return s;
+  char* ws = static_cast<char*>(c->ws);
+  for (int i = 0; i < n_models; ++i) {
+    cudaMemsetAsync(logp[i], 0, (size_t)T * 4, c->stream);
+    if (entropy && entropy[i]) cudaMemsetAsync(entropy[i], 0, (size_t)T * 4, c->stream);
+    GemmShape fwd_shape;
+    FwdPlan plan;
+    plan.scan = i == 0;   // the mask is scanned once; every model reuses the row map
+    if ((s = run_forward(c, L, H[i], ldH[i], W[i], ldW[i], tokens, mask, T, d[i], V, &fwd_shape, nullptr, plan)) != RL_OK)
+      return s;
+    LossParams p;
+    memset(&p, 0, sizeof(p));
+    p.partials = reinterpret_cast<const float4*>(ws + L.partials);
+    p.part_stride = L.Tpad;
+    p.fwd_shape = fwd_shape;
+    p.fwd_cg = c->cta_group;
+    p.fwd_workers = c->grid[c->cta_group] / c->cta_group;
+    p.row_map = reinterpret_cast<const int*>(ws + L.row_map);
+    p.lse_c = reinterpret_cast<float*>(ws + L.lse_c);
+    p.ent_c = reinterpret_cast<float*>(ws + L.ent_c);
+    p.logp_out = logp[i];
+    p.ent_out = entropy ? entropy[i] : nullptr;
+    int blocks = (int)((T + kLossThreads - 1) / kLossThreads);
+    if (blocks > 1024) blocks = 1024;
+    combine_loss_kernel<<<blocks, kLossThreads, 0, c->stream>>>(p, c->dstatus);
     c->launches++;
   }
   return cuda_ok();

@@ -110,10 +110,13 @@ __global__ void __launch_bounds__(kScanThreads) mask_write_kernel(const uint8_t*
 // ------------------------------------------------------------------------------------------
 // Row compaction: Hc[i,:] = H[row_map[i],:] for i < n_valid, zero rows up to the next multiple
 // of 128 (so that tensor-core tiles never see stale data), compact token ids, and the
-// token-range check.  One warp per row, 16-byte loads.
+// token-range check.  One warp per row, 16-byte loads.  Token ids are checked against the whole
+// vocabulary [0, V) and stored relative to vocab_off, the first id of the rows of W this call
+// holds (0 unless the head is split by vocabulary): an id outside the held slice becomes a
+// negative or too large column that no tile ever matches.
 __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* __restrict__ H, long long ldH, int d,
                                                           const int* __restrict__ row_map,
-                                                          const int* __restrict__ tokens, int V,
+                                                          const int* __restrict__ tokens, int V, int vocab_off,
                                                           __nv_bfloat16* __restrict__ Hc,
                                                           int* __restrict__ tokens_c, DevStatus* st) {
   const int n = st->n_valid;
@@ -129,8 +132,9 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
       for (int v = lane; v < vec_per_row; v += 32) dst[v] = __ldg(src + v);
       if (lane == 0) {
         const int y = tokens[r];
-        tokens_c[i] = y;
-        if (y < 0 || y >= V) latch_status(st, kStatusTokenRange, r);
+        const bool in_range = y >= 0 && y < V;
+        tokens_c[i] = in_range ? y - vocab_off : -1;
+        if (!in_range) latch_status(st, kStatusTokenRange, r);
       }
     } else {
       for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
@@ -313,31 +317,50 @@ struct LossParams {
   float* kl_out;
   // reduction scratch: [gridDim.x][kLossSums] doubles
   double* block_sums;
+  // vocabulary-parallel head: stats_out != NULL -> only merge the ranges of this call's slice and
+  // write (M, S, A, z_y) per original row; ext_lse != NULL -> the statistics of the whole
+  // vocabulary come from the caller ([T], original rows) instead of the partials
+  float4* stats_out;
+  const float* ext_logp;
+  const float* ext_ent;
+  const float* ext_lse;
 };
 constexpr int kLossSums = 8;  // loss, pg, kl, ent, clip, ratio, ratio_max, unused
 constexpr int kLossThreads = 256;
 
 __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossParams p, DevStatus* st) {
   const int n = st->n_valid;
-  const int n_ranges = gemm_extents(p.fwd_shape, n, p.fwd_cg, p.fwd_workers).n_ranges;
+  const int n_ranges = p.ext_lse ? 0 : gemm_extents(p.fwd_shape, n, p.fwd_cg, p.fwd_workers).n_ranges;
   double acc[kLossSums];
 #pragma unroll
   for (int k = 0; k < kLossSums; ++k) acc[k] = 0.0;
   const float w_mean = n > 0 ? 1.f / (float)n : 0.f;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-    float M = -CUDART_INF_F;
-    for (int r = 0; r < n_ranges; ++r) M = fmaxf(M, p.partials[(size_t)r * p.part_stride + i].x);
-    float S = 0.f, A = 0.f, zy = 0.f;
-    for (int r = 0; r < n_ranges; ++r) {
-      const float4 q = p.partials[(size_t)r * p.part_stride + i];
-      const float sc = exp2f((q.x - M) * kLog2e);
-      S = fmaf(q.y, sc, S);
-      A = fmaf(q.z, sc, A);
-      zy += q.w;
+    float lse, logp, ent;
+    float M = -CUDART_INF_F, S = 0.f, A = 0.f;
+    if (p.ext_lse) {
+      const int row = p.row_map[i];
+      lse = p.ext_lse[row];
+      logp = p.ext_logp[row];
+      ent = p.ext_ent[row];
+    } else {
+      for (int r = 0; r < n_ranges; ++r) M = fmaxf(M, p.partials[(size_t)r * p.part_stride + i].x);
+      float zy = 0.f;
+      for (int r = 0; r < n_ranges; ++r) {
+        const float4 q = p.partials[(size_t)r * p.part_stride + i];
+        const float sc = exp2f((q.x - M) * kLog2e);
+        S = fmaf(q.y, sc, S);
+        A = fmaf(q.z, sc, A);
+        zy += q.w;
+      }
+      if (p.stats_out) {
+        p.stats_out[p.row_map[i]] = make_float4(M, S, A, zy);
+        continue;
+      }
+      lse = M + logf(S);
+      logp = zy - lse;
+      ent = lse - A / S;
     }
-    const float lse = M + logf(S);
-    const float logp = zy - lse;
-    const float ent = lse - A / S;
     float kl = 0.f;
     if (p.kl_full) {
       float Mr = -CUDART_INF_F;
@@ -563,6 +586,38 @@ __global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restr
   if (metrics) {
     if (k >= 1 && k <= 6) metrics[k - 1] = (float)v;
     if (k == 7) { metrics[6] = (float)st->n_valid; metrics[7] = 0.f; }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Vocabulary-parallel head: merge of the per-row statistics (M, S, A, z_y) of the n_shards slices
+// of a partition of the vocabulary (stats[s][t], original rows) into the log-probability of the
+// sampled token, the entropy and the log-sum-exp over the whole vocabulary.  Rows with mask 0
+// get 0.  One thread per row; the slices are visited in order, so the result is reproducible.
+__global__ void __launch_bounds__(256) merge_shard_stats_kernel(const float4* __restrict__ stats, int n_shards,
+                                                                long long T, const uint8_t* __restrict__ mask,
+                                                                float* __restrict__ logp, float* __restrict__ ent,
+                                                                float* __restrict__ lse) {
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < T; t += (long long)gridDim.x * blockDim.x) {
+    float o_logp = 0.f, o_ent = 0.f, o_lse = 0.f;
+    if (!mask || mask[t]) {
+      float M = -CUDART_INF_F;
+      for (int s = 0; s < n_shards; ++s) M = fmaxf(M, __ldg(&stats[(size_t)s * T + t]).x);
+      float S = 0.f, A = 0.f, zy = 0.f;
+      for (int s = 0; s < n_shards; ++s) {
+        const float4 q = __ldg(&stats[(size_t)s * T + t]);
+        const float sc = exp2f((q.x - M) * kLog2e);
+        S = fmaf(q.y, sc, S);
+        A = fmaf(q.z, sc, A);
+        zy += q.w;
+      }
+      o_lse = M + logf(S);
+      o_logp = zy - o_lse;
+      o_ent = o_lse - A / S;
+    }
+    logp[t] = o_logp;
+    if (ent) ent[t] = o_ent;
+    if (lse) lse[t] = o_lse;
   }
 }
 

@@ -42,3 +42,47 @@ def allreduce_gradients(dW: torch.Tensor, loss: torch.Tensor, group=None):
         dist.all_reduce(dW, op=dist.ReduceOp.SUM, group=group)
         dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=group)
     return dW, loss
+
+
+# ---------------------------------------------------------------------------------------------
+# Vocabulary-parallel head: the rows of the LM-head weight are partitioned over the ranks of a
+# group (rank r holds vocabulary ids [offsets[r], offsets[r+1])), every rank sees the same token
+# rows.  Two exchanges are real: an all-gather of 16 bytes of softmax statistics per row and an
+# all-reduce (sum) of the partial dH.  `compute` is the object that runs the three per-rank calls
+# (a binding.Context on a GPU); it is a parameter so that the plumbing can be exercised on CPU
+# ranks with a stand-in.
+def shard_vocab(V: int, world: int, rank: int, multiple: int = 256):
+    """Contiguous slice of the vocabulary for `rank`: (offset, size).  Slices are whole multiples of
+    `multiple` rows (one tensor-core column tile) except the last, which takes the remainder."""
+    tiles = -(-V // multiple)
+    base, extra = divmod(tiles, world)
+    start = (rank * base + min(rank, extra)) * multiple
+    stop = ((rank + 1) * base + min(rank + 1, extra)) * multiple
+    start, stop = min(start, V), min(stop, V)
+    return start, stop - start
+
+
+def vocab_parallel_logprobs(compute, H, W_shard, tokens, mask, vocab_offset, V_total, group=None):
+    """(logp, entropy, lse) over the whole vocabulary, identical on every rank of the group."""
+    stats = compute.rl_shard_logit_stats(H, W_shard, tokens, mask, vocab_offset, V_total)
+    world = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
+    if world > 1:
+        gathered = torch.empty((world,) + tuple(stats.shape), dtype=stats.dtype, device=stats.device)
+        dist.all_gather(list(gathered.unbind(0)), stats.contiguous(), group=group)
+    else:
+        gathered = stats.reshape((1,) + tuple(stats.shape))
+    return compute.rl_merge_logit_stats(gathered, mask)
+
+
+def vocab_parallel_loss_fwd_bwd(compute, H, W_shard, tokens, old_logp, ref_logp, adv, mask, vocab_offset, V_total,
+                                eps_low, eps_high, beta, group=None, **kw):
+    """Forward and backward with the head split by vocabulary.  Returns dict(loss, dH, dW, logp,
+    entropy): loss and dH (fp32, summed over the group) are the same on every rank; dW holds this
+    rank's rows of the head gradient."""
+    logp, ent, lse = vocab_parallel_logprobs(compute, H, W_shard, tokens, mask, vocab_offset, V_total, group)
+    out = compute.rl_policy_loss_shard_bwd(H, W_shard, tokens, old_logp, ref_logp, adv, mask, vocab_offset, V_total,
+                                           logp, ent, lse, eps_low, eps_high, beta, **kw)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(out["dH"], op=dist.ReduceOp.SUM, group=group)
+    out["logp"], out["entropy"] = logp, ent
+    return out

@@ -96,3 +96,77 @@ def test_two_rank_data_parallel_matches_single_process():
     # weights travel as fp32 (1/N rounded), hence the 1e-6 relative tolerance
     assert abs(loss - ref["loss"]) <= 1e-6 * abs(ref["loss"])
     assert np.abs(dW - ref["dW"]).max() <= 1e-6 * np.abs(ref["dW"]).max()
+
+
+# ----------------------------------------------------------------------------- vocabulary-parallel head
+class _OracleCompute:
+    """Stands in for the GPU context on CPU ranks: the three per-rank calls, from the float64 oracle."""
+
+    def rl_shard_logit_stats(self, H, W_shard, tokens, mask, vocab_offset, V_total):
+        return torch.from_numpy(O.shard_logit_stats(H.numpy(), W_shard.numpy(), tokens.numpy(), vocab_offset, mask.numpy()))
+
+    def rl_merge_logit_stats(self, stats, mask):
+        return tuple(torch.from_numpy(x) for x in O.merge_logit_stats(stats.numpy(), mask.numpy()))
+
+    def rl_policy_loss_shard_bwd(self, H, W_shard, tokens, old, ref, adv, mask, vocab_offset, V_total, logp, ent, lse,
+                                 eps_low, eps_high, beta, **kw):
+        o = O.policy_loss_shard_bwd(H.numpy(), W_shard.numpy(), tokens.numpy(), vocab_offset, logp.numpy(), ent.numpy(),
+                                    lse.numpy(), old.numpy(), ref.numpy(), adv.numpy(), mask.numpy(), eps_low, eps_high,
+                                    beta, **kw)
+        return dict(loss=torch.tensor([o["loss"]], dtype=torch.float64), dH=torch.from_numpy(o["dH_partial"]), dW=torch.from_numpy(o["dW_shard"]))
+
+
+def _vocab_worker(rank, world, port, q):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2512_21450_b200 import parallel as par
+    P = _problem()
+    V = P["W"].shape[0]
+    off, size = par.shard_vocab(V, world, rank, multiple=8)
+    T = P["H"].shape[0]
+    adv = O.broadcast_to_tokens(O.grpo_advantages(P["rewards"], P["G"]), np.arange(0, T + 1, P["L"]), T)
+    t = torch.from_numpy
+    out = par.vocab_parallel_loss_fwd_bwd(_OracleCompute(), t(P["H"]), t(P["W"][off:off + size].copy()), t(P["tok"]),
+                                          t(P["old"]), t(P["ref"]), t(adv), t(P["mask"]), off, V, 0.2, 0.28, 0.04,
+                                          ent_coef=0.01)
+    q.put((rank, off, size, out["dW"].numpy(), out["dH"].numpy(), float(out["loss"].item()), out["logp"].numpy()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_shard_vocab_partition():
+    from paper_2512_21450_b200 import parallel as par
+    for V in (1, 255, 256, 4096, 151936, 152064):
+        for world in (1, 2, 3, 8):
+            pos = 0
+            for r in range(world):
+                off, size = par.shard_vocab(V, world, r)
+                assert off == pos and size >= 0 and (off % 256 == 0 or size == 0)
+                pos += size
+            assert pos == V
+
+
+def test_two_rank_vocab_parallel_matches_single_process():
+    world = 2
+    port = _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_vocab_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted([q.get(timeout=120) for _ in range(world)], key=lambda x: x[0])
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    P = _problem()
+    T = P["H"].shape[0]
+    adv = O.broadcast_to_tokens(O.grpo_advantages(P["rewards"], P["G"]), np.arange(0, T + 1, P["L"]), T)
+    ref = O.policy_loss_fwd_bwd(P["H"], P["W"], P["tok"], P["old"], P["ref"], adv, P["mask"], 0.2, 0.28, 0.04,
+                                ent_coef=0.01)
+    assert got[0][1] == 0 and got[0][2] > 0 and got[1][1] == got[0][2] and got[1][1] + got[1][2] == P["W"].shape[0]
+    for rank, off, size, dW, dH, loss, logp in got:
+        assert abs(loss - ref["loss"]) <= 1e-13 * max(1.0, abs(ref["loss"]))
+        assert np.abs(logp - ref["logp"]).max() <= 1e-12
+        assert np.abs(dW - ref["dW"][off:off + size]).max() <= 1e-13
+        assert np.abs(dH - ref["dH"]).max() <= 1e-13          # summed over the two ranks
