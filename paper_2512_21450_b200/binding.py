@@ -76,6 +76,8 @@ def load_library():
     lib.rl_set_slab_limits.argtypes = [P, c_int, c_int]
     lib.rl_set_dh_k_slices.argtypes = [P, c_int]
     lib.rl_set_dh_k_slices.restype = c_int
+    lib.rl_set_dh_stream_k.argtypes = [P, c_int]
+    lib.rl_set_dh_stream_k.restype = c_int
     lib.rl_set_cta_group.argtypes = [P, c_int]
     lib.rl_set_cta_group.restype = c_int
     lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
@@ -180,6 +182,9 @@ class Context:
 
     def set_dh_k_slices(self, max_slices):
         _check(self.lib.rl_set_dh_k_slices(self.handle, max_slices), "rl_set_dh_k_slices")
+
+    def set_dh_stream_k(self, on):
+        _check(self.lib.rl_set_dh_stream_k(self.handle, int(on)), "rl_set_dh_stream_k")
 
     def set_cta_group(self, cta_group):
         _check(self.lib.rl_set_cta_group(self.handle, cta_group), "rl_set_cta_group")

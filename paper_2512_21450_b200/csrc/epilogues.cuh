@@ -231,6 +231,7 @@ struct EpiAcc {
     int n_cols;
     int accumulate;
     int row_base;
+    int slice_add;   // stream-K launches: output slices past the first are always added to
   };
   struct State {
     int k_slice;
@@ -266,7 +267,7 @@ struct EpiAcc {
     fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) {
-      if (p.accumulate) tma_reduce_add_3d(tmC, buf, col0, p.row_base + row0, st.k_slice);
+      if (p.accumulate || (p.slice_add && st.k_slice > 0)) tma_reduce_add_3d(tmC, buf, col0, p.row_base + row0, st.k_slice);
       else              tma_store_3d(tmC, buf, col0, p.row_base + row0, st.k_slice);
       bulk_commit_group();
     }

@@ -90,6 +90,16 @@ struct GemmShape {
   // the K range, each a work unit of its own that adds into its own output buffer (the epilogue
   // gets the slice index); the slice count is chosen on the device to even out the last wave.
   int k_split_max;
+  // Stream-K: when set (and the tiles are not cut by k_split, n_range == 1) and the tile count is
+  // not a multiple of the worker count, the tiles of the last full wave and of the ragged wave
+  // after it are balanced: their (tile, k-block) iterations, tile-major, are cut into one
+  // contiguous share per worker, so every worker gets the same amount of tensor-core work.  A
+  // tile that straddles two shares is finished by two workers: the part that starts at k-block 0
+  // goes to output slice 0, the part that ends the tile is ADDED to output slice 1 (which the
+  // caller zeroes beforehand), so each output element still has exactly one writer per slice and
+  // launch.  Every share holds at least one whole tile's worth of iterations, so a tile has at
+  // most two parts.
+  int stream_k;
   // coordinate offsets into the operands' global tensors
   int a_mn_off, a_k_off, b_mn_off, b_k_off;
 };
@@ -110,7 +120,7 @@ __host__ __device__ inline int choose_split(int m_units, int n_tiles, int n_work
 }
 
 struct GemmExtents {
-  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units, slab_off, k_split, kb_per;
+  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units, slab_off, k_split, kb_per, stream_k;
 };
 
 // Number of K slices per tile (1..smax) that minimises the number of waves the tiles take on
@@ -172,6 +182,8 @@ __host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_v
   e.kb_per = (e.k_blocks + e.k_split - 1) / e.k_split;
   e.n_units *= e.k_split;
   if (sh.skip_if_k0 && e.k_blocks == 0) e.n_units = 0;
+  e.stream_k = (sh.stream_k && e.k_split == 1 && e.n_range == 1 && e.k_blocks > 0 && e.n_units >= n_workers &&
+                e.n_units % n_workers != 0) ? 1 : 0;
   return e;
 }
 
@@ -185,6 +197,46 @@ __device__ __forceinline__ void unit_coords(const GemmShape& sh, const GemmExten
   if (sh.n_fastest) { nr = u % ex.n_ranges; mu = u / ex.n_ranges; }
   else              { mu = u % ex.m_units;  nr = u / ex.m_units; }
 }
+
+// The work units of one worker, in the order all three roles of a CTA walk them.
+// Plain: units worker, worker + n_workers, ... decoded by unit_coords.  Stream-K: all full waves
+// but the last are walked the same way (CTAs that run together then share operand panels); the
+// remaining tiles (between one and two per worker) are balanced: their (tile, k-block) iterations,
+// tile-major, are cut into one contiguous share per worker, one unit per tile a share touches; ks
+// is then the output slice of the part: 0 when it starts at k-block 0, else 1.
+struct UnitWalk {
+  const GemmShape& sh;
+  const GemmExtents& ex;
+  int n_workers, u, plain_units;
+  long long it, it_end;
+  __device__ __forceinline__ UnitWalk(const GemmShape& sh_, const GemmExtents& ex_, int worker, int n_workers_)
+      : sh(sh_), ex(ex_), n_workers(n_workers_), u(worker), plain_units(ex_.n_units), it(0), it_end(0) {
+    if (ex.stream_k) {
+      plain_units = (ex.n_units / n_workers - 1) * n_workers;
+      const long long total = (long long)(ex.n_units - plain_units) * ex.k_blocks;
+      it = total * worker / n_workers;
+      it_end = total * (worker + 1) / n_workers;
+    }
+  }
+  __device__ __forceinline__ bool next(int& mu, int& nr, int& ks, int& kb0, int& kb1) {
+    if (u < plain_units) {
+      unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
+      u += n_workers;
+      return true;
+    }
+    if (it >= it_end) return false;
+    const int t_rel = (int)(it / ex.k_blocks);
+    kb0 = (int)(it - (long long)t_rel * ex.k_blocks);
+    const long long left = it_end - it;
+    kb1 = (left < (long long)(ex.k_blocks - kb0)) ? kb0 + (int)left : ex.k_blocks;
+    ks = kb0 > 0 ? 1 : 0;
+    it += kb1 - kb0;
+    const int tile = plain_units + t_rel;
+    if (sh.n_fastest) { nr = tile % ex.n_ranges; mu = tile / ex.n_ranges; }
+    else              { mu = tile % ex.m_units;  nr = tile / ex.m_units; }
+    return true;
+  }
+};
 
 // Epilogue functor contract (all methods run in the 128 epilogue threads, one tile row each):
 //   struct Epi { struct Params; struct State;
@@ -246,9 +298,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = worker; u < ex.n_units && ok; u += n_workers) {
-        int mu, nr, ks, kb0, kb1;
-        unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
+      UnitWalk walk(sh, ex, worker, n_workers);
+      int mu, nr, ks, kb0, kb1;
+      while (ok && walk.next(mu, nr, ks, kb0, kb1)) {
         const int m = mu * CG + (int)rank;
         const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
         for (int n = n0; n < n1 && ok; ++n) {
@@ -306,9 +358,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t t = 0;
       bool ok = true;
       if (ex.k_blocks > 0) {
-        for (int u = worker; u < ex.n_units && ok; u += n_workers) {
-          int mu, nr, ks, kb0, kb1;
-          unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
+        UnitWalk walk(sh, ex, worker, n_workers);
+        int mu, nr, ks, kb0, kb1;
+        while (ok && walk.next(mu, nr, ks, kb0, kb1)) {
           if (kb1 <= kb0) continue;   // empty K slice: the epilogue handles it without an accumulator
           const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
           for (int n = n0; n < n1 && ok; ++n, ++t) {
@@ -362,9 +414,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     Epi::init(st);
     uint32_t t = 0;
     bool ok = true;
-    for (int u = worker; u < ex.n_units && ok; u += n_workers) {
-      int mu, nr, ks, kb0, kb1;
-      unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
+    UnitWalk walk(sh, ex, worker, n_workers);
+    int mu, nr, ks, kb0, kb1;
+    while (ok && walk.next(mu, nr, ks, kb0, kb1)) {
       const bool has_k = kb1 > kb0;   // an empty K slice contributes zeros
       const int m = mu * CG + (int)rank;
       const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);

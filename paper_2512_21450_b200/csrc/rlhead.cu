@@ -34,6 +34,7 @@ struct rl_ctx {
   int slab_cols;  // vocabulary columns of one gradient slab (multiple of 256)
   int cta_group;  // 1: one CTA per 128x256 tile; 2: CTA pairs on 256x256 tiles
   int dh_k_slices;  // upper bound on the K slices of the dH pass (1 = tiles are not cut)
+  int dh_stream_k;  // 1: the dH pass balances its tiles over the SMs by stream-K (needs a second accumulator buffer)
   int grid[3];    // persistent grid for cta_group 1 and 2 (index = cta_group)
   long long launches;  // kernels launched by this context so far
   // optional per-kernel timing: event pairs around every tensor-core launch, by kernel kind
@@ -50,6 +51,10 @@ constexpr int kDhSplitMax = 4;             // most K slices (separate fp32 accum
 constexpr int kSlabColsMax = 148 * 128;    // vocabulary columns of one gradient slab (74 tiles of 256)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// fp32 accumulator buffers of the dH pass: one per K slice, or two when stream-K balancing is on
+inline bool dh_uses_stream_k(const rl_ctx* c) { return c->dh_stream_k && c->dh_k_slices == 1; }
+inline int dh_buffers(const rl_ctx* c) { return dh_uses_stream_k(c) ? 2 : c->dh_k_slices; }
 
 struct WsLayout {
   int Tpad, Ts, Vs;
@@ -93,7 +98,7 @@ WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_s
   L.block_sums = take((size_t)1024 * kLossSums * sizeof(double));
   L.Hc = take((size_t)L.Tpad * d * 2);
   L.G = take((size_t)L.Ts * L.Vs * 2);
-  L.dH_acc = take((size_t)c->dh_k_slices * L.Ts * d * 4);
+  L.dH_acc = take((size_t)dh_buffers(c) * L.Ts * d * 4);
   L.Hc_ref = L.partials2 = L.lse_ref_c = L.kl_c = L.cb_c = 0;
   if (d_ref > 0) {
     L.Hc_ref = take((size_t)L.Tpad * d_ref * 2);
@@ -401,6 +406,7 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->slab_cols = kSlabColsMax;
   c->cta_group = 1;
   c->dh_k_slices = 1;
+  c->dh_stream_k = 1;
   c->grid[0] = 0;
   c->grid[1] = c->n_sm;
   c->grid[2] = c->n_sm / 2 * 2;
@@ -499,6 +505,12 @@ rl_status rl_set_dh_k_slices(rl_ctx* c, int max_slices) {
   if (!c) return RL_ERR_INVALID_ARG;
   if (max_slices < 1 || max_slices > kDhSplitMax) return RL_ERR_INVALID_ARG;
   c->dh_k_slices = max_slices;
+  return RL_OK;
+}
+
+rl_status rl_set_dh_stream_k(rl_ctx* c, int on) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  c->dh_stream_k = on ? 1 : 0;
   return RL_OK;
 }
 
@@ -829,7 +841,7 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
             map_mnmajor(c, &tmG_mn, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs, BM / 64) &&
             map_mnmajor(c, &tmHc_mn, Hc, (uint64_t)L.Tpad, (uint64_t)d, (uint64_t)d, b_box_panels(c)) &&
             map_out_bf16(c, &tm_G_out, G, (uint64_t)L.Ts, (uint64_t)L.Vs, (uint64_t)L.Vs) &&
-            map_out_f32(c, &tm_dH, dH_acc, (uint64_t)L.Ts, (uint64_t)d, (uint64_t)d, (uint64_t)c->dh_k_slices, (uint64_t)L.Ts) &&
+            map_out_f32(c, &tm_dH, dH_acc, (uint64_t)L.Ts, (uint64_t)d, (uint64_t)d, (uint64_t)dh_buffers(c), (uint64_t)L.Ts) &&
             map_out_f32(c, &tm_dW, dW, (uint64_t)V, (uint64_t)d, (uint64_t)d, 1, (uint64_t)V);
   if (!ok) return RL_ERR_CUDA;
 
@@ -840,6 +852,8 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
     GemmShape dh_shape;
     memset(&dh_shape, 0, sizeof(dh_shape));
     const int rows_cap = L.Ts;   // the valid rows are cut into equal slabs of at most Ts rows on the device
+    // stream-K parts that finish a tile are added to the second accumulator buffer: it starts at zero
+    if (dh_uses_stream_k(c)) cudaMemsetAsync(dH_acc + (size_t)L.Ts * d, 0, (size_t)L.Ts * d * 4, st);
     for (int cs = 0; cs < n_col_slabs; ++cs) {
       const int vocab_base = cs * L.Vs;
       const int cols = (int)((V - vocab_base) < L.Vs ? (V - vocab_base) : L.Vs);
@@ -881,9 +895,10 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
         sh.b_k_off = vocab_base;
         sh.n_fastest = 1;   // the CTAs that share a panel of G rows run together
         sh.k_split_max = c->dh_k_slices;
+        sh.stream_k = dh_uses_stream_k(c) ? 1 : 0;
         dh_shape = sh;      // the slice count depends only on rows, d tiles and grid: same for every slab
         EpiAcc::Params ep;
-        ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0;
+        ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0; ep.slice_add = sh.stream_k;
         launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, tm_dH, sh, ep);
       }
       // (3) dW_slab (+)= G^T * H_slab      [vocabulary rows x d], K = valid rows of the slab
@@ -900,7 +915,7 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
         sh.n_fastest = 1;
         EpiAcc::Params ep;
         ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
-        ep.row_base = vocab_base;
+        ep.row_base = vocab_base; ep.slice_add = 0;
         launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, tm_dW, sh, ep);
       }
     }
@@ -1141,7 +1156,7 @@ rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, in
   CUtensorMap tc;
   if (!map_out_f32(c, &tc, C, (uint64_t)M, (uint64_t)N, (uint64_t)N, 1, (uint64_t)M)) return RL_ERR_CUDA;
   EpiAcc::Params ep;
-  ep.n_cols = (int)N; ep.accumulate = accumulate; ep.row_base = 0;
+  ep.n_cols = (int)N; ep.accumulate = accumulate; ep.row_base = 0; ep.slice_add = 0;
   if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, -1, ta, tb, tc, sh, ep);
   else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, -1, ta, tb, tc, sh, ep);
   else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, -1, ta, tb, tc, sh, ep);
@@ -1204,6 +1219,7 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
     c.slab_cols = kSlabColsMax;
     c.cta_group = 1;
     c.dh_k_slices = 1;
+    c.dh_stream_k = 0;
     c.grid[1] = c.n_sm;
     slot.ready = true;
   }

@@ -643,7 +643,8 @@ __global__ void __launch_bounds__(256) scatter_dH_f32_kernel(const float* __rest
                                                              float* __restrict__ dH, const DevStatus* st) {
   int slab_base, rows;
   slab_extent(st->n_valid, dh_shape.slab_cap, dh_shape.slab_index, slab_base, rows);
-  const int n_slices = gemm_extents(dh_shape, st->n_valid, dh_cg, dh_workers).k_split;
+  // stream-K launches always keep two buffers (the second holds the parts that finished a tile)
+  const int n_slices = dh_shape.stream_k ? 2 : gemm_extents(dh_shape, st->n_valid, dh_cg, dh_workers).k_split;
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
@@ -659,7 +660,8 @@ __global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict
                                                          __nv_bfloat16* __restrict__ dH, const DevStatus* st) {
   int slab_base, rows;
   slab_extent(st->n_valid, dh_shape.slab_cap, dh_shape.slab_index, slab_base, rows);
-  const int n_slices = gemm_extents(dh_shape, st->n_valid, dh_cg, dh_workers).k_split;
+  // stream-K launches always keep two buffers (the second holds the parts that finished a tile)
+  const int n_slices = dh_shape.stream_k ? 2 : gemm_extents(dh_shape, st->n_valid, dh_cg, dh_workers).k_split;
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {

@@ -345,6 +345,37 @@ def test_dh_k_slices(slices):
         c2.close()
 
 
+@pytest.mark.parametrize("cta_group", [2, 1])
+def test_dh_stream_k(cta_group):
+    # dH tiles balanced over the SMs by stream-K: a case with more tiles than workers and a ragged last
+    # wave (10 row tiles of 256 x 8 column tiles = 80 tiles on 74 pairs; 160 on 148 single CTAs), several
+    # vocabulary slabs (parts are added to what earlier slabs left) - against the oracle, against the
+    # plain tile loop, and bitwise reproducible
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(1, prompts=1, L_max=640, V=1200, seed=83)
+    assert 2304 < w.n_valid <= 2560
+    c2 = Context(0)
+    try:
+        c2.set_cta_group(cta_group)
+        c2.set_slab_limits(32768, 512)
+        out, _ = _check_against_oracle(c2, w)
+        first = out["dH"].clone()
+        again, _ = _check_against_oracle(c2, w)
+        assert torch.equal(first, again["dH"])
+        c2.set_dh_stream_k(False)
+        plain, _ = _check_against_oracle(c2, w)
+        assert _rel(_np64(first), _np64(plain["dH"])) <= 1e-2
+        # fp32 dH leaves the two accumulator buffers without a bf16 rounding in between
+        c2.set_dh_stream_k(True)
+        a32, _ = _check_against_oracle(c2, w, dH_fp32=True)
+        c2.set_dh_stream_k(False)
+        b32, _ = _check_against_oracle(c2, w, dH_fp32=True)
+        assert _rel(_np64(a32["dH"]), _np64(b32["dH"])) <= 1e-5
+    finally:
+        c2.close()
+
+
 def test_token_weight_accumulate_and_strides(ctx):
     from paper_2512_21450_b200.workloads import make_workload
     w = make_workload(0, seed=31)
