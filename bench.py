@@ -83,7 +83,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], None, set()
+        sm, smax, reasons, power = [], None, set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             if len(r) < 7:
@@ -93,12 +93,17 @@ class ClockSampler:
                 smax = float(r[1])
             except ValueError:
                 continue
+            try:
+                power.append(float(r[2]))
+            except ValueError:
+                pass
             for n, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         sm.sort()
+        power.sort()
         return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=smax, reasons=sorted(reasons),
-                    samples=len(sm))
+                    samples=len(sm), power_w=power[len(power) // 2] if power else None)
 
 
 def oracle_sample_time(w, n_rows, repeat=1):

@@ -86,14 +86,17 @@ rl_status rl_set_cta_group(rl_ctx* ctx, int cta_group);
  * (max_slices - 1) extra [slab rows x d] fp32 buffers of workspace: call before
  * rl_workspace_bytes().  On the measured workloads the gain was within 1 %. */
 rl_status rl_set_dh_k_slices(rl_ctx* ctx, int max_slices);
-/* Load balancing of the dH pass (default on).  The pass has (row tiles x d/256) output tiles; when
- * that count is not a multiple of the number of SM pairs the last wave of tiles would leave most
- * SMs idle (7.14 waves at d = 2048 with 16896 rows).  With stream-K on, the tile x k-block
- * iterations are instead cut into equal contiguous shares, one per SM pair; a tile that straddles
- * two shares is completed in a second fp32 accumulator buffer, summed when dH is written.  Every
- * element still has one writer per buffer and launch, so results stay reproducible run to run.
- * Costs one extra [slab rows x d] fp32 buffer of workspace: call before rl_workspace_bytes().
- * Ignored while rl_set_dh_k_slices() asks for more than one slice. */
+/* Load balancing of the dH pass (default off).  The pass has (row tiles x d/256) output tiles; when
+ * that count is not a multiple of the number of SM pairs the last wave of tiles leaves most SMs
+ * idle (7.14 waves at d = 2048 with 16896 rows).  With stream-K on, the last full wave and the
+ * ragged wave are instead cut, by tile x k-block iterations, into equal contiguous shares, one per
+ * SM pair; a tile that straddles two shares is completed in a second fp32 accumulator buffer,
+ * summed when dH is written.  Every element still has one writer per buffer and launch, so
+ * results stay reproducible run to run.  Costs one extra [slab rows x d] fp32 buffer of
+ * workspace: call before rl_workspace_bytes().  Ignored while rl_set_dh_k_slices() asks for more
+ * than one slice.  Measured: the dH pass itself gets about 7 % faster at 16896 rows, but a
+ * whole step on a board that sits at its power limit does not (the other passes slow down by as
+ * much), which is why it is opt-in. */
 rl_status rl_set_dh_stream_k(rl_ctx* ctx, int on);
 /* Caller-owned device scratch, 256-byte aligned; must outlive the calls that use it. */
 rl_status rl_set_workspace(rl_ctx* ctx, void* dev_ptr, size_t bytes);

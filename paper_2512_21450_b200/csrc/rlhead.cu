@@ -406,7 +406,7 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->slab_cols = kSlabColsMax;
   c->cta_group = 1;
   c->dh_k_slices = 1;
-  c->dh_stream_k = 1;
+  c->dh_stream_k = 0;
   c->grid[0] = 0;
   c->grid[1] = c->n_sm;
   c->grid[2] = c->n_sm / 2 * 2;

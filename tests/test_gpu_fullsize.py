@@ -171,3 +171,74 @@ def test_full_size_full_kl():
     finally:
         ctx.close()
         torch.cuda.empty_cache()
+
+
+def test_full_size_vocab_parallel():
+    """Config 1 at full size with the head cut into two vocabulary slices (one GPU plays both ranks
+    in turn): merged log-prob / entropy and the summed dH on sampled rows, sampled dW rows on both
+    sides of the cut, the loss, and the two identities on the assembled gradients."""
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    ctx = Context(0)
+    try:
+        w = make_workload(1)
+        cut = 296 * 256            # 75776: the first slice ends on a column-tile boundary, the second is ragged
+        cuts = (0, cut, w.V)
+        _, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+        stats = torch.stack([ctx.rl_shard_logit_stats(w.H, w.W[a:b], w.tokens, w.mask, a, w.V)
+                             for a, b in zip(cuts[:-1], cuts[1:])]).contiguous()
+        logp, ent, lse = ctx.rl_merge_logit_stats(stats, w.mask)
+        dH = torch.zeros(w.T, w.d, dtype=torch.float32, device=w.H.device)
+        dW = torch.empty(w.V, w.d, dtype=torch.float32, device=w.H.device)
+        losses = []
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            o = ctx.rl_policy_loss_shard_bwd(w.H, w.W[a:b], w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, a, w.V,
+                                             logp, ent, lse, w.eps_low, w.eps_high, w.beta, dW=dW[a:b])
+            dH += o["dH"]
+            losses.append(o["loss"].item())
+        status, detail = ctx.last_device_status()
+        assert status == 0, (status, hex(detail & 0xffffffff))
+        assert losses[0] == losses[1]
+
+        o_adv_tok = O.broadcast_to_tokens(O.grpo_advantages(w.rewards.cpu().numpy(), w.G),
+                                          w.seq_offsets.cpu().numpy(), w.T)
+        valid = torch.nonzero(w.mask, as_tuple=False)[:, 0].cpu().numpy()
+        N = valid.size
+        rng = np.random.default_rng(991)
+        special = [0, 127, 128, 255, 256, N - 129, N - 1]
+        idx = np.unique(np.concatenate([np.array(special), rng.choice(N, size=128, replace=False)]))
+        rows = valid[idx]
+        W64 = _np64(w.W)
+        r = O.dH_rows(_np64(w.H[rows]), W64, w.tokens[rows].cpu().numpy(), _np64(w.old_logp[rows]),
+                      _np64(w.ref_logp[rows]), o_adv_tok[rows], np.full(rows.size, 1.0 / N), w.eps_low, w.eps_high,
+                      w.beta)
+        assert np.abs(_np64(logp[rows]) - r["logp"]).max() <= TOL_LOGP
+        assert np.abs(_np64(ent[rows]) - r["entropy"]).max() <= TOL_ENT
+        assert np.abs(_np64(lse[rows]) - r["lse"]).max() <= TOL_LOGP
+        assert _rel(_np64(dH[rows]), r["dH"]) <= TOL_GRAD_REL
+        masked = torch.nonzero(w.mask == 0, as_tuple=False)[:, 0]
+        assert not dH[masked[:4096]].any() and not logp[masked[:4096]].any()
+
+        lp, en, ls = _np64(logp)[valid], _np64(ent)[valid], _np64(lse)[valid]
+        s, k3, rho, active, dlogp = O.per_token_terms(lp, _np64(w.old_logp)[valid], _np64(w.ref_logp)[valid],
+                                                      o_adv_tok[valid], w.eps_low, w.eps_high, w.beta)
+        loss64 = float(((-s + w.beta * k3) / N).sum())
+        assert abs(losses[0] - loss64) <= TOL_LOSS_REL * abs(loss64) + 1e-7
+
+        tok_valid = w.tokens.cpu().numpy()[valid]
+        sel = np.unique(np.concatenate([rng.choice(w.V, size=48, replace=False),
+                                        np.array([0, cut - 2, cut - 1, cut, cut + 1, w.V - 2, w.V - 1])]))
+        Hv = _np64(w.H[torch.from_numpy(valid).to(w.H.device)])
+        dWs = O.dW_rows(Hv, W64[sel], sel, tok_valid, ls, en, dlogp / N, np.zeros(N))
+        del Hv, W64
+        assert _rel(_np64(dW[torch.from_numpy(sel).to(w.H.device)]), dWs) <= TOL_GRAD_REL
+
+        col_sum = dW.double().sum(dim=0)
+        col_abs = dW.double().abs().sum(dim=0)
+        assert (col_sum.abs() <= 1e-3 * col_abs + 1e-12).all()
+        rowdot = (dH.double() * w.H.double()).sum(dim=1)
+        rhs = (dW.double() * w.W.double()).sum().item()
+        assert abs(rowdot.sum().item() - rhs) <= 1e-2 * rowdot.abs().sum().item()
+    finally:
+        ctx.close()
+        torch.cuda.empty_cache()

@@ -359,6 +359,7 @@ def test_dh_stream_k(cta_group):
     try:
         c2.set_cta_group(cta_group)
         c2.set_slab_limits(32768, 512)
+        c2.set_dh_stream_k(True)
         out, _ = _check_against_oracle(c2, w)
         first = out["dH"].clone()
         again, _ = _check_against_oracle(c2, w)
