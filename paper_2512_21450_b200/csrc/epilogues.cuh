@@ -168,10 +168,21 @@ struct EpiGrad {
           g[i + 1] = g2.y;
         }
       } else {
+        // entropy term as well, still two columns per instruction:
+        // g = p * (ce * (z - lse) + (ce * Ent + cp))
+        const float2 l2 = make_float2(kLog2e, kLog2e), nl2 = make_float2(-st.lse * kLog2e, -st.lse * kLog2e);
+        const float2 nlse2 = make_float2(-st.lse, -st.lse), ce2 = make_float2(st.ce, st.ce);
+        const float k = fmaf(st.ce, st.ent, st.cp);
+        const float2 k2 = make_float2(k, k);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float lp = v[i] - st.lse;
-          g[i] = ex2_approx(lp * kLog2e) * fmaf(st.ce, lp + st.ent, st.cp);
+        for (int i = 0; i < 32; i += 2) {
+          const float2 z2 = make_float2(v[i], v[i + 1]);
+          const float2 t2 = __ffma2_rn(z2, l2, nl2);
+          const float2 e2 = make_float2(ex2_approx(t2.x), ex2_approx(t2.y));
+          const float2 w2 = __ffma2_rn(ce2, __fadd2_rn(z2, nlse2), k2);
+          const float2 g2 = __fmul2_rn(e2, w2);
+          g[i] = g2.x;
+          g[i + 1] = g2.y;
         }
       }
       const unsigned rel = (unsigned)(st.y - col_g);
