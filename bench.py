@@ -25,12 +25,17 @@ METRIC = "fused LM-head logprob+GRPO loss fwd+bwd tokens/s; % of bf16 tensor pea
 KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad> (dlogits slab)",
               "gemm_kernel<EpiAcc,K,MN> (dH)", "gemm_kernel<EpiAcc,MN,MN> (dW)"]
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant
-# kernel from an ncu capture, valid only for the sources of that kernel (main loop, its epilogue,
-# the PTX wrappers) whose hash is recorded with it.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core kernels from one ncu
+# capture of config 1 (profiles/gemm_kernels_config1_ncu_full.md), valid only for the sources of those
+# kernels (main loop, epilogues, PTX wrappers) whose hash is recorded with it.  Kind 0 is the forward
+# launch (whole vocabulary); kinds 1-3 were captured on a full slab of 18944 vocabulary columns and their
+# traffic grows with the slab's columns, so an average launch of a step (the last slab is short) carries
+# bytes x (V / 18944) / launches-per-step.
 KERNEL_SOURCES = ("epilogues.cuh", "gemm_engine.cuh", "ptx.cuh")
-NCU_TRAFFIC = {"sources_sha256": "08d32b81de7297c58b9a8584da760398c3bb1cfe36befa4b194947ea6eb2c0ce", "kind": 2, "config": 1,
-               "bytes_per_launch": 1334359000 + 137476608}   # profiles/gemm_kernels_config1_ncu_full.md
+NCU_TRAFFIC = {"sources_sha256": "c11a8ee356dc6cdd9722a1e8f346dbc4a2922aa2beef331e18a4dbdddda76b43", "config": 1,
+               "slab_cols": 18944,
+               "bytes": {0: 3003288000 + 23964160, 1: 1051839000 + 623447552, 2: 1352570000 + 140417280,
+                         3: 1278569000 + 141344768}}
 
 
 def sources_hash():
@@ -366,9 +371,10 @@ def main():
     dom = max(range(4), key=lambda k: kind_ms[k])
     achieved = flops_pass / (kind_ms[dom] / 1e3) / 1e12
     traffic = None
-    if (NCU_TRAFFIC["sources_sha256"] == sources_hash() and NCU_TRAFFIC["kind"] == dom
-            and NCU_TRAFFIC["config"] == args.config):
-        traffic = NCU_TRAFFIC["bytes_per_launch"]
+    if NCU_TRAFFIC["sources_sha256"] == sources_hash() and NCU_TRAFFIC["config"] == args.config:
+        traffic = float(NCU_TRAFFIC["bytes"][dom])
+        if dom != 0:
+            traffic *= (w.V / NCU_TRAFFIC["slab_cols"]) / (kind_n[dom] / args.steps)
     roofline = {
         "bound": "tensor", "kernel": KIND_NAMES[dom], "achieved": achieved, "peak": peaks["sustained"],
         "unit": "TFLOP/s", "frac": achieved / peaks["sustained"], "peak_source": f"of {peaks['source']} (sustained)",
