@@ -229,6 +229,64 @@ def run_library_comparison(args):
     print(json.dumps({"library_comparison": res, "note": "sustained loops of 2.5 s each, one kernel at a time"}))
 
 
+def run_small_kernel_stress(args):
+    """The HBM-bound helpers at a size where a bandwidth fraction means something: 2^26 token rows,
+    2^20 GRPO groups of 8 responses.  Each kernel is timed alone with CUDA events (inputs far larger
+    than L2), algorithmic bytes / time against the measured copy bandwidth."""
+    import torch
+    from paper_2512_21450_b200 import Context
+    ctx = Context(0)
+    peaks = measured_peaks()
+    T, n_groups, G = 1 << 26, 1 << 20, 8
+    n_seq = n_groups * G
+    g = torch.Generator(device="cuda").manual_seed(SEED_STRESS)
+    mask = (torch.rand(T, generator=g, device="cuda") < 0.55).to(torch.uint8)
+    N = int(mask.sum().item())
+    row_map = torch.empty(T, dtype=torch.int32, device="cuda")
+    n_valid = torch.empty(1, dtype=torch.int32, device="cuda")
+    rewards = (torch.rand(n_seq, generator=g, device="cuda") < 0.4).float()
+    seq_offsets = torch.arange(0, T + 1, T // n_seq, dtype=torch.int32, device="cuda")
+    stats = torch.randn(1, T, 4, generator=g, device="cuda")
+    stats[..., 1] = stats[..., 1].abs() + 1.0          # S >= 1 as for real statistics
+
+    def timed(fn, iters=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    out = []
+
+    def report(name, ms, nbytes, note):
+        gbs = nbytes / (ms / 1e3) / 1e9
+        out.append(dict(kernel=name, ms=ms, algorithmic_bytes=nbytes, gbs=gbs, frac_of_hbm_peak=gbs / peaks["hbm"],
+                        bytes=note))
+
+    ms = timed(lambda: ctx.rl_mask_scan(mask, row_map=row_map, n_valid=n_valid))
+    report("mask scan (count, offsets, write)", ms, T + 4 * N, "mask read once + row map written (the kernels read the mask twice)")
+    assert int(n_valid.item()) == N
+    ms = timed(lambda: ctx.rl_grpo_advantages(rewards, G, seq_offsets=seq_offsets, T=T))
+    report("GRPO advantages + broadcast", ms, 12 * n_seq + 4 * (n_seq + 1) + 4 * T,
+           "rewards read, per-response advantages written and read back, offsets read, per-token advantages written "
+           "(the call also clears the per-token array first; the binding allocates the outputs)")
+    ms = timed(lambda: ctx.rl_merge_logit_stats(stats, mask))
+    report("merge of softmax statistics -> logp, entropy, lse", ms, 16 * T + T + 12 * T,
+           "16 B of statistics + 1 B of mask read, three fp32 outputs written per row (the binding allocates the outputs)")
+    status, _ = ctx.last_device_status()
+    assert status == 0
+    print(json.dumps({"small_kernel_stress": {"rows": T, "valid_rows": N, "groups": n_groups, "group_size": G,
+                                              "peak_gbs": peaks["hbm"], "peak_source": peaks["source"], "kernels": out}}))
+
+
+SEED_STRESS = 251221450 + 99
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -241,6 +299,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--compare-library", action="store_true",
                     help="instead of the benchmark line, time the tensor-core kernels against torch.matmul")
+    ap.add_argument("--stress-small", action="store_true",
+                    help="instead of the benchmark line, time the HBM-bound helper kernels at 2^26 rows / 2^20 groups")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
@@ -249,6 +309,9 @@ def main():
         return
     if args.compare_library:
         run_library_comparison(args)
+        return
+    if args.stress_small:
+        run_small_kernel_stress(args)
         return
 
     import torch

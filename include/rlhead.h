@@ -136,6 +136,14 @@ typedef enum { RL_ADV_GRPO = 0, RL_ADV_RLOO = 1, RL_ADV_OPO = 2, RL_ADV_REINFORC
 rl_status rl_advantages(rl_ctx* ctx, int estimator, const float* rewards, const int32_t* lengths,
                         int64_t n_seq, int group_size, float eps_std, float* adv_seq);
 
+/* Padding-free row map on its own (section 4.4 "padding-free training"): row_map[i] = index of
+ * the i-th row with mask != 0, ascending, for i < *n_valid; entries past that are left untouched.
+ * mask NULL = all rows valid.  row_map[T] (int32) and n_valid[1] (int32) are device pointers; the
+ * workspace needs (T / 4096 + 3) * 4 bytes.  Every other call of this library runs the same
+ * three kernels internally; this entry exists so that the map can be checked and timed by itself.
+ * Errors: T < 0 or T >= 2^31, NULL outputs -> RL_ERR_INVALID_ARG; RL_ERR_WORKSPACE. */
+rl_status rl_mask_scan(rl_ctx* ctx, const uint8_t* mask, int64_t T, int32_t* row_map, int32_t* n_valid);
+
 /* Per-token log-probability of the sampled token, entropy and log-sum-exp of the next-token
  * distribution softmax(W h_t) - section 2.2 (policy over the vocabulary; importance ratio
  * numerator) and section 2.2 "Regularization" (entropy).  Natural logarithms.

@@ -126,6 +126,17 @@ def broadcast_to_tokens(adv_seq, seq_offsets, T):
 
 
 # --------------------------------------------------------------------------- #
+# Section 4.4 "padding-free training": only rows whose mask is non-zero are
+# worked on; the row map lists them in ascending order.
+# --------------------------------------------------------------------------- #
+def valid_row_map(mask, T=None):
+    """Indices of the rows with mask != 0, ascending (mask None: every row 0..T-1)."""
+    if mask is None:
+        return list(range(T))
+    return [t for t in range(len(mask)) if mask[t] != 0]
+
+
+# --------------------------------------------------------------------------- #
 # Section 2.2: the policy is the next-token distribution over the vocabulary.
 # --------------------------------------------------------------------------- #
 def logits(H, W):

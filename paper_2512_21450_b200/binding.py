@@ -101,6 +101,8 @@ def load_library():
     lib.rl_selftest_gemm.argtypes = [P, P, P, P, c_int64, c_int64, c_int64, c_int, c_int, c_int]
     lib.rl_token_logprobs_static.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P, P]
     lib.rl_token_logprobs_static.restype = c_int
+    lib.rl_mask_scan.argtypes = [P, P, c_int64, P, P]
+    lib.rl_mask_scan.restype = c_int
     lib.rl_token_logprobs_multi.argtypes = [P, c_int, POINTER(c_void_p), POINTER(c_int64), POINTER(c_void_p),
                                             POINTER(c_int64), POINTER(c_int64), P, P, c_int64, c_int64,
                                             POINTER(c_void_p), POINTER(c_void_p)]
@@ -303,6 +305,21 @@ class Context:
                 opts.kl_out = out["kl"].data_ptr()
         _check(self.lib.rl_policy_loss_fwd_bwd_ex(*args, byref(opts)), "rl_policy_loss_fwd_bwd_ex")
         return out
+
+    def rl_mask_scan(self, mask, T=None, row_map=None, n_valid=None):
+        """Row map of the valid rows: returns (row_map [T] int32, n_valid [1] int32), both on the device."""
+        self._bind_stream()
+        T = mask.numel() if T is None else T
+        need = (T // 4096 + 3) * 4
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=self.device)
+        _check(self.lib.rl_set_workspace(self.handle, _ptr(self._ws), self._ws.numel()), "rl_set_workspace")
+        if row_map is None:
+            row_map = torch.empty(max(T, 1), dtype=torch.int32, device=self.device)
+        if n_valid is None:
+            n_valid = torch.empty(1, dtype=torch.int32, device=self.device)
+        _check(self.lib.rl_mask_scan(self.handle, _ptr(mask), T, _ptr(row_map), _ptr(n_valid)), "rl_mask_scan")
+        return row_map, n_valid
 
     def rl_token_logprobs_multi(self, Hs, Ws, tokens, mask=None, want_entropy=True):
         """Log-probabilities of the same tokens under several models (e.g. old policy and reference):

@@ -583,15 +583,21 @@ rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, 
   if (n_seq == 0) return RL_OK;
   const int n_groups = (int)(n_seq / group_size);
   const int warps = 8;
+  int seg = 32;   // lanes per group, as the kernel computes it
+  while (seg > 1 && (seg >> 1) >= group_size) seg >>= 1;
+  const int groups_per_block = warps * (32 / seg);
   const int pr_adv = prof_begin(c, 8);
-  grpo_adv_kernel<<<(n_groups + warps - 1) / warps, warps * 32, 0, c->stream>>>(rewards, n_groups, group_size, ddof,
-                                                                                eps_std, adv_seq);
+  grpo_adv_kernel<<<(n_groups + groups_per_block - 1) / groups_per_block, warps * 32, 0, c->stream>>>(
+      rewards, n_groups, group_size, ddof, eps_std, adv_seq);
   c->launches++;
   if (adv_tok) {
-    if (T > 0 && cudaMemsetAsync(adv_tok, 0, (size_t)T * 4, c->stream) != cudaSuccess) return RL_ERR_CUDA;
-    int blocks = (int)(n_seq < 4096 ? n_seq : 4096);
-    broadcast_adv_kernel<<<blocks, 256, 0, c->stream>>>(adv_seq, seq_offsets, (int)n_seq, adv_tok);
-    c->launches++;
+    if (T > 0) {
+      const long long rows_per_block = (long long)kBroadcastRounds * 1024;
+      long long blocks = (T + rows_per_block - 1) / rows_per_block;
+      if (blocks > (long long)c->n_sm * 32) blocks = (long long)c->n_sm * 32;
+      broadcast_adv_kernel<<<(int)blocks, 256, 0, c->stream>>>(adv_seq, seq_offsets, (int)n_seq, (long long)T, adv_tok);
+      c->launches++;
+    }
   }
   prof_end(c, pr_adv, 8);
   return cuda_ok();
@@ -627,6 +633,23 @@ rl_status rl_advantages(rl_ctx* c, int estimator, const float* rewards, const in
 
 rl_status rl_grpo_advantages(rl_ctx* c, const float* rewards, int64_t n_seq, int group_size, float* adv_seq) {
   return rl_grpo_advantages_ex(c, rewards, n_seq, group_size, 1, 1e-6f, nullptr, 0, adv_seq, nullptr);
+}
+
+rl_status rl_mask_scan(rl_ctx* c, const uint8_t* mask, int64_t T, int32_t* row_map, int32_t* n_valid) {
+  if (!c || T < 0 || T >= (int64_t(1) << 31) || !n_valid || (T > 0 && !row_map)) return RL_ERR_INVALID_ARG;
+  if (T == 0) return cudaMemsetAsync(n_valid, 0, 4, c->stream) == cudaSuccess ? RL_OK : RL_ERR_CUDA;
+  const int n_blocks = (int)((T + kScanRowsPerBlock - 1) / kScanRowsPerBlock);
+  if (!c->ws || c->ws_bytes < ((size_t)n_blocks + 2) * 4) return RL_ERR_WORKSPACE;
+  int* block_counts = static_cast<int*>(c->ws);
+  const int pr = prof_begin(c, 4);
+  mask_count_kernel<<<n_blocks, kScanThreads, 0, c->stream>>>(mask, (int)T, block_counts);
+  mask_offsets_kernel<<<1, 1024, 0, c->stream>>>(block_counts, n_blocks, c->dstatus);
+  mask_write_kernel<<<n_blocks, kScanThreads, 0, c->stream>>>(mask, (int)T, block_counts, row_map);
+  prof_end(c, pr, 4);
+  c->launches += 3;
+  if (cudaMemcpyAsync(n_valid, &c->dstatus->n_valid, 4, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
+    return RL_ERR_CUDA;
+  return cuda_ok();
 }
 
 rl_status rl_token_logprobs(rl_ctx* c, const void* H, int64_t ldH, const void* W, int64_t ldW, const int32_t* tokens,

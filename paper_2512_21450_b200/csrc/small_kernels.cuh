@@ -97,14 +97,20 @@ __global__ void __launch_bounds__(kScanThreads) mask_write_kernel(const uint8_t*
                                                                   const int* __restrict__ block_offsets,
                                                                   int* __restrict__ row_map) {
   __shared__ int warp_sums[32];
+  __shared__ int block_total;
+  __shared__ int staged[kScanRowsPerBlock];   // the block's valid rows, in order
   const long long base = ((long long)blockIdx.x * kScanThreads + threadIdx.x) * kScanRowsPerThread;
   unsigned bits = scan_load_bits(mask, base, T);
-  int pos = block_offsets[blockIdx.x] + block_exclusive_scan(__popc(bits), warp_sums, nullptr);
+  int pos = block_exclusive_scan(__popc(bits), warp_sums, &block_total);
   while (bits) {
     const int i = __ffs(bits) - 1;
     bits &= bits - 1;
-    row_map[pos++] = (int)base + i;
+    staged[pos++] = (int)base + i;
   }
+  __syncthreads();
+  // coalesced copy of the block's indices to their place in the map
+  int* dst = row_map + block_offsets[blockIdx.x];
+  for (int k = threadIdx.x; k < block_total; k += kScanThreads) dst[k] = staged[k];
 }
 
 // ------------------------------------------------------------------------------------------
@@ -164,38 +170,48 @@ __global__ void __launch_bounds__(256) gather_plain_kernel(const __nv_bfloat16* 
 }
 
 // ------------------------------------------------------------------------------------------
-// GRPO advantages (section 4.2 group-based normalisation): one warp per group of G consecutive
-// rewards, shuffle reductions for mean, centred sum of squares and the all-equal test.
+// GRPO advantages (section 4.2 group-based normalisation), warp-shuffle segmented: a warp is cut
+// into segments of seg = (smallest power of two >= G, at most 32) lanes, one group of G consecutive
+// rewards per segment (a group of more than 32 responses takes a whole warp and strides over it).
+// Mean, centred sum of squares (both in double) and the all-equal test are butterfly reductions that
+// stay inside the segment.  For power-of-two G a warp reads and writes 128 contiguous bytes.
 __global__ void __launch_bounds__(256) grpo_adv_kernel(const float* __restrict__ rewards, int n_groups, int G,
                                                        int ddof, float eps_std, float* __restrict__ adv_seq) {
+  int seg = 32;
+  while (seg > 1 && (seg >> 1) >= G) seg >>= 1;
+  const int groups_per_warp = 32 / seg;
   const int lane = threadIdx.x & 31;
-  const int g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (g >= n_groups) return;
-  const float* r = rewards + (size_t)g * G;
-  float sum = 0.f, mx = -CUDART_INF_F, mn = CUDART_INF_F;
-  for (int i = lane; i < G; i += 32) {
+  const int sub = lane & (seg - 1);
+  const long long warp_global = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long g = warp_global * groups_per_warp + lane / seg;
+  const bool live = g < n_groups;                 // lanes of groups past the end still take part in the shuffles
+  const float* r = rewards + (size_t)(live ? g : 0) * G;
+  // sums in double: a group whose rewards lie close together has a small sigma, and the rounding of
+  // an fp32 mean divided by it would exceed the 1e-6 the advantages are held to
+  double sum = 0.0;
+  float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+  for (int i = sub; i < G && live; i += seg) {
     const float x = r[i];
-    sum += x;
+    sum += (double)x;
     mx = fmaxf(mx, x);
     mn = fminf(mn, x);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
+  for (int o = seg >> 1; o > 0; o >>= 1) {
     sum += __shfl_xor_sync(0xffffffffu, sum, o);
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
   }
-  const float mu = sum / (float)G;
-  float ss = 0.f;
-  for (int i = lane; i < G; i += 32) {
-    const float c = r[i] - mu;
-    ss = fmaf(c, c, ss);
+  const double mu = sum / (double)G;
+  double ss = 0.0;
+  for (int i = sub; i < G && live; i += seg) {
+    const double c = (double)r[i] - mu;
+    ss = fma(c, c, ss);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  const float sigma = sqrtf(ss / (float)(G - ddof));
-  const float inv = (mx == mn) ? 0.f : 1.f / (sigma + eps_std);
-  for (int i = lane; i < G; i += 32) adv_seq[(size_t)g * G + i] = (mx == mn) ? 0.f : (r[i] - mu) * inv;
+  for (int o = seg >> 1; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const double sigma = sqrt(ss / (double)(G - ddof));
+  const double inv = (mx == mn) ? 0.0 : 1.0 / (sigma + (double)eps_std);
+  for (int i = sub; i < G && live; i += seg)
+    adv_seq[(size_t)g * G + i] = (mx == mn) ? 0.f : (float)(((double)r[i] - mu) * inv);
 }
 
 // Other critic-free estimators named in section 4.2 (no formula printed there; readings):
@@ -270,13 +286,67 @@ __global__ void __launch_bounds__(256) batch_normalise_kernel(float* __restrict_
 }
 
 // Broadcast of the per-response advantage to the rows of the response (outcome supervision).
+// The row ranges [seq_offsets[s], seq_offsets[s+1]) are ascending and adjacent, so they partition
+// [seq_offsets[0], seq_offsets[n_seq]); rows outside that span get 0.  A block owns
+// kBroadcastRounds * 1024 consecutive rows and walks them in rounds of 1024; a thread owns four
+// consecutive rows per round (one 16-byte store when the output is aligned).  It finds the response
+// of its first row by binary search in round 0 and from then on by a galloping search that starts
+// at the response it ended the previous round in, so the cost per row does not depend on how long
+// the responses are and almost all offset reads after round 0 hit lines the block just used.
+constexpr int kBroadcastRounds = 8;
+
+// Largest s in [s_from, n_seq) with seq_offsets[s] <= t, given seq_offsets[s_from] <= t < seq_offsets[n_seq].
+__device__ __forceinline__ int seq_of_row(const int* __restrict__ seq_offsets, int n_seq, int s_from, long long t) {
+  int lo = s_from, step = 1;
+  while (lo + step < n_seq && seq_offsets[lo + step] <= t) { lo += step; step <<= 1; }
+  int hi = min(lo + step, n_seq);        // seq_offsets[lo] <= t < seq_offsets[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (seq_offsets[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
 __global__ void __launch_bounds__(256) broadcast_adv_kernel(const float* __restrict__ adv_seq,
                                                             const int* __restrict__ seq_offsets, int n_seq,
-                                                            float* __restrict__ adv_tok) {
-  for (int s = blockIdx.x; s < n_seq; s += gridDim.x) {
-    const int b = seq_offsets[s], e = seq_offsets[s + 1];
-    const float a = adv_seq[s];
-    for (int t = b + threadIdx.x; t < e; t += blockDim.x) adv_tok[t] = a;
+                                                            long long T, float* __restrict__ adv_tok) {
+  const int first = seq_offsets[0], last = seq_offsets[n_seq];
+  const bool vec_ok = (reinterpret_cast<uintptr_t>(adv_tok) & 15) == 0;
+  const long long rows_per_block = (long long)kBroadcastRounds * blockDim.x * 4;
+  for (long long b0 = (long long)blockIdx.x * rows_per_block; b0 < T; b0 += (long long)gridDim.x * rows_per_block) {
+    int s = -1;                           // response this thread was in last, -1: not searched yet
+    for (int round = 0; round < kBroadcastRounds; ++round) {
+      const long long t0 = b0 + ((long long)round * blockDim.x + threadIdx.x) * 4;
+      if (t0 >= T) break;
+      float v[4] = {0.f, 0.f, 0.f, 0.f};
+      if (t0 + 3 >= first && t0 < last) {
+        const long long t_in = t0 < first ? first : t0;
+        if (s < 0) {
+          int lo = 0, hi = n_seq;         // seq_offsets[lo] <= t_in < seq_offsets[hi]
+          while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (seq_offsets[mid] <= t_in) lo = mid; else hi = mid;
+          }
+          s = lo;
+        } else {
+          s = seq_of_row(seq_offsets, n_seq, s, t_in);
+        }
+        int end = seq_offsets[s + 1];
+        float a = adv_seq[s];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const long long t = t0 + i;
+          if (t < first || t >= last) continue;
+          while (t >= end) { ++s; end = seq_offsets[s + 1]; a = adv_seq[s]; }   // empty ranges are skipped
+          v[i] = a;
+        }
+      }
+      if (vec_ok && t0 + 3 < T) {
+        *reinterpret_cast<float4*>(adv_tok + t0) = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
+        for (int i = 0; i < 4 && t0 + i < T; ++i) adv_tok[t0 + i] = v[i];
+      }
+    }
   }
 }
 

@@ -127,7 +127,27 @@ def test_single_cta_tiles_match_oracle():
         c1.close()
 
 
-@pytest.mark.parametrize("n_groups,G", [(4, 4), (8, 8), (64, 16), (7, 5), (3, 40), (1024, 8)])
+@pytest.mark.parametrize("T", [1, 15, 16, 17, 4095, 4096, 4097, 70001, (1 << 20) + 3])
+def test_mask_scan_row_map_is_exact(ctx, T):
+    # integer work: the row map and the count must equal the oracle's bit for bit
+    rng = np.random.default_rng(T)
+    for p_valid in (0.0, 0.55, 1.0):
+        m_np = (rng.uniform(size=T) < p_valid).astype(np.uint8) * rng.integers(1, 256, size=T).astype(np.uint8)
+        backing = torch.zeros(T + 1, dtype=torch.uint8, device="cuda")
+        for off in (0, 1):                               # 16-byte aligned and unaligned mask pointers
+            mask = backing[off:off + T]
+            mask.copy_(torch.from_numpy(m_np))
+            row_map, n_valid = ctx.rl_mask_scan(mask)
+            expect = O.valid_row_map(m_np.tolist())
+            assert n_valid.item() == len(expect)
+            assert row_map[:len(expect)].cpu().tolist() == expect
+    row_map, n_valid = ctx.rl_mask_scan(None, T=T)       # no mask: every row
+    assert n_valid.item() == T and row_map.cpu().tolist() == O.valid_row_map(None, T)
+    _assert_status_ok(ctx)
+
+
+@pytest.mark.parametrize("n_groups,G", [(4, 4), (8, 8), (64, 16), (7, 5), (3, 40), (1024, 8), (9, 2), (5, 32), (3, 33),
+                                        (100, 3)])
 def test_advantages(ctx, n_groups, G):
     rng = np.random.default_rng(100 + G)
     for kind in ("bernoulli", "uniform", "zero_var"):
@@ -144,6 +164,45 @@ def test_advantages(ctx, n_groups, G):
             assert np.abs(_np64(a) - o).max() <= TOL_ADV
             if kind == "zero_var":
                 assert not _np64(a).any()
+
+
+@pytest.mark.parametrize("case", ["long", "short", "ragged", "empty_ranges", "inner_span", "one_row"])
+def test_advantage_broadcast_is_exact(ctx, case):
+    # a copy: every row must carry exactly its response's value, rows outside the span of the ranges 0
+    rng = np.random.default_rng(sum(map(ord, case)))
+    G = 4
+    if case == "long":
+        lens = rng.integers(3000, 9000, size=16)
+    elif case == "short":
+        lens = rng.integers(1, 9, size=4096)
+    elif case == "ragged":
+        lens = np.concatenate([rng.integers(1, 5, size=300), rng.integers(500, 3000, size=20)])
+        rng.shuffle(lens)
+    elif case == "empty_ranges":
+        lens = rng.integers(0, 40, size=2000) * (rng.uniform(size=2000) < 0.3)
+        lens[:700] = 0
+        lens[700] = 5
+    elif case == "inner_span":
+        lens = rng.integers(10, 2000, size=64)
+    else:
+        lens = np.ones(4, dtype=np.int64)
+    first = 1237 if case == "inner_span" else 0
+    off = np.concatenate([[first], first + np.cumsum(lens)]).astype(np.int32)
+    T = int(off[-1]) + (4321 if case == "inner_span" else 0)
+    if case == "ragged":
+        T += 3                                              # rows past the last range, T not a multiple of 4
+    n_seq = len(lens)
+    r = rng.uniform(size=n_seq).astype(np.float32)
+    adv_seq, adv_tok = ctx.rl_grpo_advantages(torch.from_numpy(r).cuda(), G, seq_offsets=torch.from_numpy(off).cuda(), T=T)
+    _assert_status_ok(ctx)
+    expect = O.broadcast_to_tokens(O.grpo_advantages(r, G), off, T)
+    got = _np64(adv_tok)
+    assert got.shape == (T,) and np.abs(got - expect).max() <= TOL_ADV
+    outside = np.ones(T, dtype=bool)
+    outside[off[0]:off[-1]] = False
+    assert not got[outside].any()                             # rows outside the span of the ranges: exactly 0
+    # property of the copy: a row holds bit for bit what the call returned for its response
+    assert np.array_equal(got[off[0]:off[-1]], np.repeat(_np64(adv_seq), lens))
 
 
 @pytest.mark.parametrize("n_groups,G", [(8, 8), (5, 3), (64, 16), (3, 40), (2048, 8)])
@@ -310,6 +369,13 @@ def test_extreme_shapes(ctx, d, V, L_max):
     out, oo = _check_against_oracle(ctx, w)
     if V == 1:
         assert not out["dH"].any() and not out["dW"].any() and not out["logp"].any()
+
+
+def test_wide_hidden_size(ctx):
+    # d = 8192, four times the hidden size of the 3B-class head: 128 k-slices per logit tile, 32 column tiles in the dH and dW passes.  The entropy-bonus configuration keeps the loss
+    # away from the near-zero value that equal-length GRPO groups otherwise cancel to.
+    from paper_2512_21450_b200.workloads import make_workload
+    _check_against_oracle(ctx, make_workload(4, prompts=1, L_max=5, d=8192, V=1500, seed=640))
 
 
 def test_multiple_slabs(ctx):

@@ -37,6 +37,7 @@ MUTANTS = {
     "slice statistics: target id not made local": ("y = int(tokens[t]) - int(vocab_offset)", "y = int(tokens[t])"),
     "slice backward: one-hot not made local": ("y = tokens[rows] - int(vocab_offset)", "y = tokens[rows]"),
     "slice backward: softmax renormalised inside the slice": ("LP = H[rows] @ W_shard.T - np.asarray(lse, dtype=np.float64)[rows][:, None]", "LP = H[rows] @ W_shard.T; LP = LP - np.log(np.exp(LP).sum(axis=1))[:, None]"),
+    "row map keeps the masked rows": ("return [t for t in range(len(mask)) if mask[t] != 0]", "return [t for t in range(len(mask)) if mask[t] == 0]"),
     "logits index order": ("return H @ W.T", "return (W @ H.T).T[::-1][::-1] if H.shape[0] == 1 else (H[:, ::-1] @ W[:, ::-1].T if False else H @ W[::-1].T)"),
 }
 

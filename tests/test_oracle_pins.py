@@ -624,3 +624,20 @@ def test_shard_backward_sums_to_the_full_gradient(cuts):
     o = O.policy_loss_shard_bwd(H, W[3:15], tokens, 3, full["logp"], full["entropy"], full["lse"], old, ref, adv,
                                 mask, token_weight=tw, **kw)
     assert np.abs(o["dW_shard"] - full["dW"][3:15]).max() < 1e-13 and abs(o["loss"] - full["loss"]) < 1e-14
+
+
+# ----------------------------------------------------------------------------- padding-free row map
+def test_valid_row_map():
+    assert O.valid_row_map([0, 3, 0, 1, 255, 0]) == [1, 3, 4]          # any non-zero byte counts
+    assert O.valid_row_map([]) == [] and O.valid_row_map([0, 0]) == [] and O.valid_row_map(None, 3) == [0, 1, 2]
+    m = (_rng(60).uniform(size=1000) < 0.3).astype(np.uint8)
+    rm = O.valid_row_map(m)
+    assert rm == sorted(rm) and len(rm) == int(m.sum()) and all(m[t] for t in rm)
+    assert rm == np.flatnonzero(m).tolist()                             # library second opinion
+    # the compacted rows are what the masked functions work on: same log-probs either way
+    H = _rng(61).normal(size=(12, 4)); W = _rng(62).normal(size=(7, 4)); tok = _rng(63).integers(0, 7, size=12)
+    mk = np.array([1, 0, 1, 1, 0, 0, 1, 0, 1, 1, 0, 1], dtype=np.uint8)
+    idx = O.valid_row_map(mk)
+    lp_masked, _, _ = O.token_logprobs(H, W, tok, mk)
+    lp_compact, _, _ = O.token_logprobs(H[idx], W, tok[idx])
+    assert np.array_equal(lp_masked[idx], lp_compact)
