@@ -317,7 +317,7 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
 
 /* Instrumentation.  rl_launch_count: kernels this context has launched so far.
  * rl_set_profiling(on): when on, every kernel (or group of small kernels) is bracketed by a pair of CUDA events
- * on the context's stream (at most 2048 launches are kept between two reads).
+ * on the context's stream (at most 65536 launch groups are kept between two reads; later ones go untimed).
  * rl_profile_read: synchronises the stream and returns, per kernel kind (0 forward statistics,
  * 1 gradient-of-logits slab, 2 dH, 3 dW, 4 mask scan, 5 row gather, 6 merge + per-token loss,
  * 7 dH scatter, 8 advantages), the summed device time in milliseconds ms[9] (host) and the number

@@ -18,7 +18,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kProfMax = 2048;   // timed launches kept between two rl_profile_read calls
+constexpr int kProfMax = 1 << 16;   // timed launch groups kept between two rl_profile_read calls
 constexpr int kProfKinds = 9;    // 0 forward statistics, 1 dlogits, 2 dH, 3 dW, 4 mask scan, 5 row gather,
                                  // 6 merge + loss, 7 dH scatter, 8 advantages
 
@@ -40,8 +40,8 @@ struct rl_ctx {
   // optional per-kernel timing: event pairs around every tensor-core launch, by kernel kind
   int prof_on;
   int prof_used;
-  int prof_kind[kProfMax];
-  cudaEvent_t prof_ev[kProfMax][2];
+  int* prof_kind;                 // [kProfMax], allocated when profiling is first switched on
+  cudaEvent_t (*prof_ev)[2];      // [kProfMax][2], events created on first use
 };
 
 namespace {
@@ -196,7 +196,7 @@ inline uint32_t b_box_panels(const rl_ctx* c) { return BN / 64 / c->cta_group; }
 
 // Optional timing of a group of launches: event pair on the context's stream, tagged with a kind.
 int prof_begin(rl_ctx* c, int kind) {
-  if (!(c->prof_on && kind >= 0 && kind < kProfKinds && c->prof_used < kProfMax)) return -1;
+  if (!(c->prof_on && c->prof_ev && kind >= 0 && kind < kProfKinds && c->prof_used < kProfMax)) return -1;
   const int i = c->prof_used;
   for (int e = 0; e < 2; ++e)
     if (!c->prof_ev[i][e]) cudaEventCreate(&c->prof_ev[i][e]);
@@ -413,7 +413,8 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->launches = 0;
   c->prof_on = 0;
   c->prof_used = 0;
-  memset(c->prof_ev, 0, sizeof(c->prof_ev));
+  c->prof_kind = nullptr;
+  c->prof_ev = nullptr;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -461,9 +462,13 @@ rl_status rl_create(rl_ctx** out, int device) {
 
 rl_status rl_destroy(rl_ctx* c) {
   if (!c) return RL_ERR_INVALID_ARG;
-  for (int i = 0; i < kProfMax; ++i)
-    for (int e = 0; e < 2; ++e)
-      if (c->prof_ev[i][e]) cudaEventDestroy(c->prof_ev[i][e]);
+  if (c->prof_ev) {
+    for (int i = 0; i < kProfMax; ++i)
+      for (int e = 0; e < 2; ++e)
+        if (c->prof_ev[i][e]) cudaEventDestroy(c->prof_ev[i][e]);
+    delete[] c->prof_ev;
+    delete[] c->prof_kind;
+  }
   cudaFree(c->dstatus);
   delete c;
   return RL_OK;
@@ -522,6 +527,18 @@ rl_status rl_launch_count(rl_ctx* c, int64_t* n) {
 
 rl_status rl_set_profiling(rl_ctx* c, int on) {
   if (!c) return RL_ERR_INVALID_ARG;
+  if (on && !c->prof_ev) {
+    c->prof_kind = new (std::nothrow) int[kProfMax];
+    c->prof_ev = new (std::nothrow) cudaEvent_t[kProfMax][2];
+    if (!c->prof_kind || !c->prof_ev) {
+      delete[] c->prof_kind;
+      delete[] c->prof_ev;
+      c->prof_kind = nullptr;
+      c->prof_ev = nullptr;
+      return RL_ERR_CUDA;
+    }
+    memset(c->prof_ev, 0, sizeof(cudaEvent_t) * 2 * kProfMax);
+  }
   c->prof_on = on ? 1 : 0;
   c->prof_used = 0;
   return RL_OK;

@@ -735,15 +735,20 @@ __global__ void __launch_bounds__(256) scatter_dH_kernel(const float* __restrict
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < rows; i += gridDim.x * warps_per_block) {
+    // eight elements per lane: two 16-byte loads, one 16-byte store (d is a multiple of 64)
     const float4* src = reinterpret_cast<const float4*>(acc + (size_t)i * d);
-    uint2* dst = reinterpret_cast<uint2*>(dH + (size_t)row_map[slab_base + i] * d);
-    for (int v = lane; v < d / 4; v += 32) {
-      const float4 x = sum_k_slices(src + v, n_slices, split_stride);
-      __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
-      uint2 o;
-      o.x = *reinterpret_cast<uint32_t*>(&lo);
-      o.y = *reinterpret_cast<uint32_t*>(&hi);
-      dst[v] = o;
+    uint4* dst = reinterpret_cast<uint4*>(dH + (size_t)row_map[slab_base + i] * d);
+    for (int v = lane; v < d / 8; v += 32) {
+      const float4 x = sum_k_slices(src + 2 * v, n_slices, split_stride);
+      const float4 y = sum_k_slices(src + 2 * v + 1, n_slices, split_stride);
+      __nv_bfloat162 b0 = __floats2bfloat162_rn(x.x, x.y), b1 = __floats2bfloat162_rn(x.z, x.w);
+      __nv_bfloat162 b2 = __floats2bfloat162_rn(y.x, y.y), b3 = __floats2bfloat162_rn(y.z, y.w);
+      uint4 o;
+      o.x = *reinterpret_cast<uint32_t*>(&b0);
+      o.y = *reinterpret_cast<uint32_t*>(&b1);
+      o.z = *reinterpret_cast<uint32_t*>(&b2);
+      o.w = *reinterpret_cast<uint32_t*>(&b3);
+      __stcs(dst + v, o);
     }
   }
 }
