@@ -86,6 +86,15 @@ rl_status rl_set_cta_group(rl_ctx* ctx, int cta_group);
  * (max_slices - 1) extra [slab rows x d] fp32 buffers of workspace: call before
  * rl_workspace_bytes().  On the measured workloads the gain was within 1 %. */
 rl_status rl_set_dh_k_slices(rl_ctx* ctx, int max_slices);
+/* L2 working set of the two passes that walk their tiles rows-first (forward statistics and the
+ * gradient-of-logits slab).  Every CTA of such a pass re-reads its panel of compacted hidden rows
+ * (256 rows x d, bf16) once per vocabulary tile; when the panels of all row tiles together exceed
+ * what L2 keeps (126 MB shared with the streamed operand), each re-read goes to DRAM.  The row
+ * tiles are therefore taken in equal groups whose panels fit `bytes` (default 36 MiB), and all
+ * vocabulary tiles are walked for one group before the next group starts; the rows of W are then
+ * read once per group instead of once per launch.  0 = one group.  Results do not depend on it.
+ * Measured: 2 % (16896 rows, d = 2048) to 11 % (32768-row slabs, d = 2560 / 3584) of a step. */
+rl_status rl_set_row_group_bytes(rl_ctx* ctx, int64_t bytes);
 /* Load balancing of the dH pass (default off).  The pass has (row tiles x d/256) output tiles; when
  * that count is not a multiple of the number of SM pairs the last wave of tiles leaves most SMs
  * idle (7.14 waves at d = 2048 with 16896 rows).  With stream-K on, the last full wave and the

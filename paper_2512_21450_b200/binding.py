@@ -76,6 +76,8 @@ def load_library():
     lib.rl_set_slab_limits.argtypes = [P, c_int, c_int]
     lib.rl_set_dh_k_slices.argtypes = [P, c_int]
     lib.rl_set_dh_k_slices.restype = c_int
+    lib.rl_set_row_group_bytes.argtypes = [P, c_int64]
+    lib.rl_set_row_group_bytes.restype = c_int
     lib.rl_set_dh_stream_k.argtypes = [P, c_int]
     lib.rl_set_dh_stream_k.restype = c_int
     lib.rl_set_cta_group.argtypes = [P, c_int]
@@ -184,6 +186,9 @@ class Context:
 
     def set_dh_k_slices(self, max_slices):
         _check(self.lib.rl_set_dh_k_slices(self.handle, max_slices), "rl_set_dh_k_slices")
+
+    def set_row_group_bytes(self, nbytes):
+        _check(self.lib.rl_set_row_group_bytes(self.handle, int(nbytes)), "rl_set_row_group_bytes")
 
     def set_dh_stream_k(self, on):
         _check(self.lib.rl_set_dh_stream_k(self.handle, int(on)), "rl_set_dh_stream_k")

@@ -100,6 +100,11 @@ struct GemmShape {
   // launch.  Every share holds at least one whole tile's worth of iterations, so a tile has at
   // most two parts.
   int stream_k;
+  // Row groups (only when the units are walked rows-first, n_fastest == 0): when m_group > 0 the row
+  // tiles are taken at most m_group at a time (in groups of equal size) and all column ranges are
+  // walked for one group before the next group starts, so that the A panels the CTAs running at any
+  // moment keep re-reading stay in L2; B is then fetched once per group instead of once per launch.
+  int m_group;
   // coordinate offsets into the operands' global tensors
   int a_mn_off, a_k_off, b_mn_off, b_k_off;
 };
@@ -120,7 +125,7 @@ __host__ __device__ inline int choose_split(int m_units, int n_tiles, int n_work
 }
 
 struct GemmExtents {
-  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units, slab_off, k_split, kb_per, stream_k;
+  int m_rows, m_units, k_blocks, n_range, n_ranges, n_units, slab_off, k_split, kb_per, stream_k, m_group;
 };
 
 // Number of K slices per tile (1..smax) that minimises the number of waves the tiles take on
@@ -182,6 +187,12 @@ __host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_v
   e.kb_per = (e.k_blocks + e.k_split - 1) / e.k_split;
   e.n_units *= e.k_split;
   if (sh.skip_if_k0 && e.k_blocks == 0) e.n_units = 0;
+  // row groups of equal size: as few groups as the budget of sh.m_group row tiles allows
+  e.m_group = 0;
+  if (sh.m_group > 0 && !sh.n_fastest && sh.m_group < e.m_units) {
+    const int n_groups = (e.m_units + sh.m_group - 1) / sh.m_group;
+    e.m_group = (e.m_units + n_groups - 1) / n_groups;
+  }
   e.stream_k = (sh.stream_k && e.k_split == 1 && e.n_range == 1 && e.k_blocks > 0 && e.n_units >= n_workers &&
                 e.n_units % n_workers != 0) ? 1 : 0;
   return e;
@@ -194,8 +205,17 @@ __device__ __forceinline__ void unit_coords(const GemmShape& sh, const GemmExten
   u /= ex.k_split;
   kb0 = ks * ex.kb_per;
   kb1 = min(kb0 + ex.kb_per, ex.k_blocks);
-  if (sh.n_fastest) { nr = u % ex.n_ranges; mu = u / ex.n_ranges; }
-  else              { mu = u % ex.m_units;  nr = u / ex.m_units; }
+  if (sh.n_fastest) {
+    nr = u % ex.n_ranges; mu = u / ex.n_ranges;
+  } else if (ex.m_group > 0) {
+    const int per_group = ex.m_group * ex.n_ranges;
+    const int gi = u / per_group, r = u - gi * per_group;
+    const int m0 = gi * ex.m_group;
+    const int gsz = min(ex.m_group, ex.m_units - m0);
+    mu = m0 + r % gsz; nr = r / gsz;
+  } else {
+    mu = u % ex.m_units;  nr = u / ex.m_units;
+  }
 }
 
 // The work units of one worker, in the order all three roles of a CTA walk them.

@@ -34,6 +34,7 @@ struct rl_ctx {
   int slab_cols;  // vocabulary columns of one gradient slab (multiple of 256)
   int cta_group;  // 1: one CTA per 128x256 tile; 2: CTA pairs on 256x256 tiles
   int dh_k_slices;  // upper bound on the K slices of the dH pass (1 = tiles are not cut)
+  long long row_group_bytes;  // forward / dlogits: bytes of A panels walked together (0 = all row tiles at once)
   int dh_stream_k;  // 1: the dH pass balances its tiles over the SMs by stream-K (needs a second accumulator buffer)
   int grid[3];    // persistent grid for cta_group 1 and 2 (index = cta_group)
   long long launches;  // kernels launched by this context so far
@@ -46,6 +47,7 @@ struct rl_ctx {
 
 namespace {
 
+constexpr long long kRowGroupBytes = 36ll << 20;   // A panels walked together by the rows-first passes (L2 is 126 MB)
 constexpr int kSlabRowsMax = 32768;        // rows of one gradient slab
 constexpr int kDhSplitMax = 4;             // most K slices (separate fp32 accumulators) of the dH pass
 constexpr int kSlabColsMax = 148 * 128;    // vocabulary columns of one gradient slab (74 tiles of 256)
@@ -290,6 +292,14 @@ struct ShardArgs {
   const float* lse;
 };
 
+// Row tiles per group for the rows-first passes: as many A panels (one row tile x K, bf16) as fit the byte budget.
+inline int row_group_tiles(const rl_ctx* c, int64_t k) {
+  if (c->row_group_bytes <= 0) return 0;
+  const long long panel = (long long)BM * c->cta_group * k * 2;
+  const long long n = c->row_group_bytes / panel;
+  return n < 1 ? 1 : (n > (1 << 20) ? (1 << 20) : (int)n);
+}
+
 inline rl_status cuda_ok() { return cudaGetLastError() == cudaSuccess ? RL_OK : RL_ERR_CUDA; }
 
 // Which part of the forward stage a call needs, and where its rows of W sit in the vocabulary.
@@ -339,6 +349,7 @@ rl_status run_forward(rl_ctx* c, const WsLayout& L, const void* H, int64_t ldH, 
   sh.k_cap = (int)d;
   sh.n_tiles = (int)((V + BN - 1) / BN);
   sh.n_range = 0;  // split chosen on the device from the number of valid rows
+  sh.m_group = row_group_tiles(c, d + (kl ? kl->d_ref : 0));
   EpiStats::Params ep;
   ep.tokens_c = tokens_c;
   ep.partials = reinterpret_cast<float4*>(ws + L.partials);
@@ -407,6 +418,7 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->cta_group = 1;
   c->dh_k_slices = 1;
   c->dh_stream_k = 0;
+  c->row_group_bytes = kRowGroupBytes;
   c->grid[0] = 0;
   c->grid[1] = c->n_sm;
   c->grid[2] = c->n_sm / 2 * 2;
@@ -510,6 +522,12 @@ rl_status rl_set_dh_k_slices(rl_ctx* c, int max_slices) {
   if (!c) return RL_ERR_INVALID_ARG;
   if (max_slices < 1 || max_slices > kDhSplitMax) return RL_ERR_INVALID_ARG;
   c->dh_k_slices = max_slices;
+  return RL_OK;
+}
+
+rl_status rl_set_row_group_bytes(rl_ctx* c, int64_t bytes) {
+  if (!c || bytes < 0) return RL_ERR_INVALID_ARG;
+  c->row_group_bytes = bytes;
   return RL_OK;
 }
 
@@ -908,6 +926,7 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
         sh.n_range = 1;
         sh.a_mn_slab = 1;
         sh.b_mn_off = vocab_base;
+        sh.m_group = row_group_tiles(c, d + (o.kl_full ? o.d_ref : 0));
         if (!o.kl_full) {
           EpiGrad::Params ep;
           ep.tokens_c = reinterpret_cast<const int*>(ws + L.tokens_c);
@@ -1260,6 +1279,7 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
     c.cta_group = 1;
     c.dh_k_slices = 1;
     c.dh_stream_k = 0;
+    c.row_group_bytes = kRowGroupBytes;
     c.grid[1] = c.n_sm;
     slot.ready = true;
   }

@@ -371,6 +371,32 @@ def test_extreme_shapes(ctx, d, V, L_max):
         assert not out["dH"].any() and not out["dW"].any() and not out["logp"].any()
 
 
+@pytest.mark.parametrize("cta_group", [2, 1])
+def test_row_groups(cta_group):
+    # the rows-first passes take the row tiles in groups that fit an L2 budget: any grouping must give
+    # bit for bit what one group gives (only the order in which tiles are visited changes), several
+    # groups, a ragged last group, several vocabulary slabs and ranges
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(1, prompts=1, L_max=400, d=256, V=3000, seed=87)
+    assert w.n_valid > 1400                                   # at least 6 row tiles of 256 / 11 of 128
+    panel = 128 * cta_group * w.d * 2
+    c2 = Context(0)
+    try:
+        c2.set_cta_group(cta_group)
+        c2.set_slab_limits(32768, 1024)
+        c2.set_row_group_bytes(0)
+        base, _ = _check_against_oracle(c2, w)
+        base = {k: v.clone() for k, v in base.items()}
+        for tiles in (1, 2, 4, 5, 1000):
+            c2.set_row_group_bytes(tiles * panel)
+            out, _ = _check_against_oracle(c2, w)
+            for k in ("loss", "dH", "dW", "logp", "entropy"):
+                assert torch.equal(out[k], base[k]), (tiles, k)
+    finally:
+        c2.close()
+
+
 def test_wide_hidden_size(ctx):
     # d = 8192, four times the hidden size of the 3B-class head: 128 k-slices per logit tile, 32 column tiles in the dH and dW passes.  The entropy-bonus configuration keeps the loss
     # away from the near-zero value that equal-length GRPO groups otherwise cancel to.
