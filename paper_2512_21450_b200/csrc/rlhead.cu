@@ -627,7 +627,7 @@ rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, 
   c->launches++;
   if (adv_tok) {
     if (T > 0) {
-      const long long rows_per_block = (long long)kBroadcastRounds * 1024;
+      const long long rows_per_block = (long long)kBroadcastSweeps * 1024;
       long long blocks = (T + rows_per_block - 1) / rows_per_block;
       if (blocks > (long long)c->n_sm * 32) blocks = (long long)c->n_sm * 32;
       broadcast_adv_kernel<<<(int)blocks, 256, 0, c->stream>>>(adv_seq, seq_offsets, (int)n_seq, (long long)T, adv_tok);

@@ -288,12 +288,12 @@ __global__ void __launch_bounds__(256) batch_normalise_kernel(float* __restrict_
 // Broadcast of the per-response advantage to the rows of the response (outcome supervision).
 // The row ranges [seq_offsets[s], seq_offsets[s+1]) are ascending and adjacent, so they partition
 // [seq_offsets[0], seq_offsets[n_seq]); rows outside that span get 0.  A block owns
-// kBroadcastRounds * 1024 consecutive rows and walks them in rounds of 1024; a thread owns four
-// consecutive rows per round (one 16-byte store when the output is aligned).  It finds the response
-// of its first row by binary search in round 0 and from then on by a galloping search that starts
-// at the response it ended the previous round in, so the cost per row does not depend on how long
-// the responses are and almost all offset reads after round 0 hit lines the block just used.
-constexpr int kBroadcastRounds = 8;
+// kBroadcastSweeps * 1024 consecutive rows and walks them in sweeps of 1024; a thread owns four
+// consecutive rows per sweep (one 16-byte store when the output is aligned).  It finds the response
+// of its first row by binary search in its first sweep and from then on by a galloping search that starts
+// at the response it ended the previous sweep in, so the cost per row does not depend on how long
+// the responses are and almost all offset reads after the first sweep hit lines the block just used.
+constexpr int kBroadcastSweeps = 8;
 
 // Largest s in [s_from, n_seq) with seq_offsets[s] <= t, given seq_offsets[s_from] <= t < seq_offsets[n_seq].
 __device__ __forceinline__ int seq_of_row(const int* __restrict__ seq_offsets, int n_seq, int s_from, long long t) {
@@ -312,11 +312,11 @@ __global__ void __launch_bounds__(256) broadcast_adv_kernel(const float* __restr
                                                             long long T, float* __restrict__ adv_tok) {
   const int first = seq_offsets[0], last = seq_offsets[n_seq];
   const bool vec_ok = (reinterpret_cast<uintptr_t>(adv_tok) & 15) == 0;
-  const long long rows_per_block = (long long)kBroadcastRounds * blockDim.x * 4;
+  const long long rows_per_block = (long long)kBroadcastSweeps * blockDim.x * 4;
   for (long long b0 = (long long)blockIdx.x * rows_per_block; b0 < T; b0 += (long long)gridDim.x * rows_per_block) {
     int s = -1;                           // response this thread was in last, -1: not searched yet
-    for (int round = 0; round < kBroadcastRounds; ++round) {
-      const long long t0 = b0 + ((long long)round * blockDim.x + threadIdx.x) * 4;
+    for (int sweep = 0; sweep < kBroadcastSweeps; ++sweep) {
+      const long long t0 = b0 + ((long long)sweep * blockDim.x + threadIdx.x) * 4;
       if (t0 >= T) break;
       float v[4] = {0.f, 0.f, 0.f, 0.f};
       if (t0 + 3 >= first && t0 < last) {
