@@ -23,7 +23,7 @@ if ROOT not in sys.path:
 
 METRIC = "fused LM-head logprob+GRPO loss fwd+bwd tokens/s; % of bf16 tensor peak"
 KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad> (dlogits slab)",
-              "gemm_kernel<EpiAcc,K,MN> (dH)", "gemm_kernel<EpiAcc,MN,MN> (dW)"]
+              "gemm_wide_kernel<EpiAcc,K,MN> (dH)", "gemm_wide_kernel<EpiAcc,MN,MN> (dW)"]
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core kernels from one ncu
 # capture of config 1 (profiles/gemm_kernels_config1_ncu_full.md), valid only for the sources of those
@@ -31,7 +31,7 @@ KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad
 # launch (whole vocabulary); kinds 1-3 were captured on a full slab of 18944 vocabulary columns and their
 # traffic grows with the slab's columns, so an average launch of a step (the last slab is short) carries
 # bytes x (V / 18944) / launches-per-step.
-KERNEL_SOURCES = ("epilogues.cuh", "gemm_engine.cuh", "ptx.cuh")
+KERNEL_SOURCES = ("epilogues.cuh", "gemm_engine.cuh", "wide_engine.cuh", "ptx.cuh")
 NCU_TRAFFIC = {"sources_sha256": "7220a2adb687c3c524e517c841f7fb1f468fd9ce018b1086ea8fb0b6153c9bdf", "config": 1,
                "slab_cols": 18944,
                "bytes": {0: 2337157000 + 24326400, 1: 356552000 + 612814336, 2: 1429694000 + 137084160,

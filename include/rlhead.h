@@ -86,6 +86,14 @@ rl_status rl_set_cta_group(rl_ctx* ctx, int cta_group);
  * (max_slices - 1) extra [slab rows x d] fp32 buffers of workspace: call before
  * rl_workspace_bytes().  On the measured workloads the gain was within 1 %. */
 rl_status rl_set_dh_k_slices(rl_ctx* ctx, int max_slices);
+/* Tile shape of the two long-K gradient products, dH = G W and dW = G^T H (default on, used when the
+ * tensor-core passes run as CTA pairs and neither rl_set_dh_k_slices nor rl_set_dh_stream_k is in
+ * effect): 256 x 512 output tiles that fill both accumulators of tensor memory, so a CTA pulls a
+ * quarter fewer operand bytes from L2 per flop, at the price of not overlapping a tile's epilogue
+ * with the next tile's main loop (about 1 % of a tile at K of 17-19 thousand).  Off: 256 x 256 tiles
+ * with a double-buffered accumulator, as the forward and gradient-of-logits passes always use.
+ * Results are bit-identical either way.  Measured: 3.4-4.1 % of a step on the four large workloads. */
+rl_status rl_set_wide_tiles(rl_ctx* ctx, int on);
 /* L2 working set of the two passes that walk their tiles rows-first (forward statistics and the
  * gradient-of-logits slab).  Every CTA of such a pass re-reads its panel of compacted hidden rows
  * (256 rows x d, bf16) once per vocabulary tile; when the panels of all row tiles together exceed

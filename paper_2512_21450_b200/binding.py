@@ -78,6 +78,8 @@ def load_library():
     lib.rl_set_dh_k_slices.restype = c_int
     lib.rl_set_row_group_bytes.argtypes = [P, c_int64]
     lib.rl_set_row_group_bytes.restype = c_int
+    lib.rl_set_wide_tiles.argtypes = [P, c_int]
+    lib.rl_set_wide_tiles.restype = c_int
     lib.rl_set_dh_stream_k.argtypes = [P, c_int]
     lib.rl_set_dh_stream_k.restype = c_int
     lib.rl_set_cta_group.argtypes = [P, c_int]
@@ -189,6 +191,9 @@ class Context:
 
     def set_row_group_bytes(self, nbytes):
         _check(self.lib.rl_set_row_group_bytes(self.handle, int(nbytes)), "rl_set_row_group_bytes")
+
+    def set_wide_tiles(self, on):
+        _check(self.lib.rl_set_wide_tiles(self.handle, int(on)), "rl_set_wide_tiles")
 
     def set_dh_stream_k(self, on):
         _check(self.lib.rl_set_dh_stream_k(self.handle, int(on)), "rl_set_dh_stream_k")

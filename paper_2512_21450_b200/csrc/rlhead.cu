@@ -11,6 +11,7 @@
 
 #include "rlhead.h"
 #include "small_kernels.cuh"
+#include "wide_engine.cuh"
 
 using namespace rlh;
 
@@ -35,6 +36,7 @@ struct rl_ctx {
   int cta_group;  // 1: one CTA per 128x256 tile; 2: CTA pairs on 256x256 tiles
   int dh_k_slices;  // upper bound on the K slices of the dH pass (1 = tiles are not cut)
   long long row_group_bytes;  // forward / dlogits: bytes of A panels walked together (0 = all row tiles at once)
+  int wide_tiles;   // 1: dH and dW run on 256 x 512 tiles (both accumulators hold one tile)
   int dh_stream_k;  // 1: the dH pass balances its tiles over the SMs by stream-K (needs a second accumulator buffer)
   int grid[3];    // persistent grid for cta_group 1 and 2 (index = cta_group)
   long long launches;  // kernels launched by this context so far
@@ -239,6 +241,33 @@ void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b
   prof_end(c, prof, kind);
 }
 
+// 256 x 512 tiles on CTA pairs; sh.n_tiles counts 512-wide column tiles.
+inline bool use_wide(const rl_ctx* c) {
+  return c->wide_tiles && c->cta_group == 2 && c->dh_k_slices == 1 && !c->dh_stream_k;
+}
+
+template <class Epi, int A_MN, int B_MN>
+void launch_wide(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& out,
+                 const GemmShape& sh, const typename Epi::Params& ep) {
+  const int prof = prof_begin(c, kind);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(c->grid[2]);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = kGemmSmemBytes;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, gemm_wide_kernel<Epi, A_MN, B_MN>, a, b, out, sh, ep, c->dstatus);
+  c->launches++;
+  prof_end(c, prof, kind);
+}
+
 template <class Epi>
 void launch_dual(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
                  const CUtensorMap& b2, const CUtensorMap& out, const GemmShape& sh, int k2_len,
@@ -418,6 +447,7 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->cta_group = 1;
   c->dh_k_slices = 1;
   c->dh_stream_k = 0;
+  c->wide_tiles = 1;
   c->row_group_bytes = kRowGroupBytes;
   c->grid[0] = 0;
   c->grid[1] = c->n_sm;
@@ -441,7 +471,11 @@ rl_status rl_create(rl_ctx** out, int device) {
   bool ok = set_smem_attr<EpiStats, 0, 0>() == cudaSuccess && set_smem_attr<EpiGrad, 0, 0>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 0, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 0, 1>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess &&
-            set_smem_attr_dual<EpiStatsKL>() == cudaSuccess && set_smem_attr_dual<EpiGradKL>() == cudaSuccess;
+            set_smem_attr_dual<EpiStatsKL>() == cudaSuccess && set_smem_attr_dual<EpiGradKL>() == cudaSuccess &&
+            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess;
   if (!ok) { cudaFree(c->dstatus); delete c; return RL_ERR_CUDA; }
   {
     // how many CTA pairs can be resident at once (pairs must share a TPC): the persistent grid
@@ -528,6 +562,12 @@ rl_status rl_set_dh_k_slices(rl_ctx* c, int max_slices) {
 rl_status rl_set_row_group_bytes(rl_ctx* c, int64_t bytes) {
   if (!c || bytes < 0) return RL_ERR_INVALID_ARG;
   c->row_group_bytes = bytes;
+  return RL_OK;
+}
+
+rl_status rl_set_wide_tiles(rl_ctx* c, int on) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  c->wide_tiles = on ? 1 : 0;
   return RL_OK;
 }
 
@@ -958,7 +998,13 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
         dh_shape = sh;      // the slice count depends only on rows, d tiles and grid: same for every slab
         EpiAcc::Params ep;
         ep.n_cols = (int)d; ep.accumulate = cs > 0; ep.row_base = 0; ep.slice_add = sh.stream_k;
-        launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, tm_dH, sh, ep);
+        if (use_wide(c)) {
+          sh.n_tiles = (int)((d + 2 * BN - 1) / (2 * BN));
+          dh_shape = sh;
+          launch_wide<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, tm_dH, sh, ep);
+        } else {
+          launch_gemm<EpiAcc, 0, 1>(c, 2, tmG_k, tmW_mn, tm_dH, sh, ep);
+        }
       }
       // (3) dW_slab (+)= G^T * H_slab      [vocabulary rows x d], K = valid rows of the slab
       {
@@ -975,7 +1021,12 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
         EpiAcc::Params ep;
         ep.n_cols = (int)d; ep.accumulate = (r > 0 || o.accumulate_dW) ? 1 : 0;
         ep.row_base = vocab_base; ep.slice_add = 0;
-        launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, tm_dW, sh, ep);
+        if (use_wide(c)) {
+          sh.n_tiles = (int)((d + 2 * BN - 1) / (2 * BN));
+          launch_wide<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, tm_dW, sh, ep);
+        } else {
+          launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, tm_dW, sh, ep);
+        }
       }
     }
     const int pr_sc = prof_begin(c, 7);
@@ -1216,7 +1267,13 @@ rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, in
   if (!map_out_f32(c, &tc, C, (uint64_t)M, (uint64_t)N, (uint64_t)N, 1, (uint64_t)M)) return RL_ERR_CUDA;
   EpiAcc::Params ep;
   ep.n_cols = (int)N; ep.accumulate = accumulate; ep.row_base = 0; ep.slice_add = 0;
-  if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, -1, ta, tb, tc, sh, ep);
+  if (use_wide(c)) {
+    sh.n_tiles = (int)((N + 2 * BN - 1) / (2 * BN));
+    if (!a_mn && !b_mn) launch_wide<EpiAcc, 0, 0>(c, -1, ta, tb, tc, sh, ep);
+    else if (!a_mn && b_mn) launch_wide<EpiAcc, 0, 1>(c, -1, ta, tb, tc, sh, ep);
+    else if (a_mn && !b_mn) launch_wide<EpiAcc, 1, 0>(c, -1, ta, tb, tc, sh, ep);
+    else launch_wide<EpiAcc, 1, 1>(c, -1, ta, tb, tc, sh, ep);
+  } else if (!a_mn && !b_mn) launch_gemm<EpiAcc, 0, 0>(c, -1, ta, tb, tc, sh, ep);
   else if (!a_mn && b_mn) launch_gemm<EpiAcc, 0, 1>(c, -1, ta, tb, tc, sh, ep);
   else if (a_mn && !b_mn) launch_gemm<EpiAcc, 1, 0>(c, -1, ta, tb, tc, sh, ep);
   else launch_gemm<EpiAcc, 1, 1>(c, -1, ta, tb, tc, sh, ep);
@@ -1279,6 +1336,7 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
     c.cta_group = 1;
     c.dh_k_slices = 1;
     c.dh_stream_k = 0;
+    c.wide_tiles = 0;
     c.row_group_bytes = kRowGroupBytes;
     c.grid[1] = c.n_sm;
     slot.ready = true;

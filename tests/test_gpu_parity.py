@@ -114,6 +114,42 @@ def test_gemm_engine_layouts(cta_group):
     ctx.close()
 
 
+def test_wide_and_square_gradient_tiles():
+    # dH and dW run on 256 x 512 tiles by default; the 256 x 256 tiles must give the same bits (every
+    # output element is the same sum in the same order), on shapes where the last wide tile is half
+    # empty (d = 256, 768, 2304) and where several slabs accumulate
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    wide, square = Context(0), Context(0)
+    try:
+        square.set_wide_tiles(False)
+        g = torch.Generator(device="cuda").manual_seed(5)
+        for (M, N, K) in [(256, 512, 64), (256, 256, 200), (384, 768, 2048), (1280, 1280, 72)]:
+            A = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+            B = torch.randn(N, K, generator=g, device="cuda").to(torch.bfloat16)
+            ref = A.float() @ B.float().T
+            for a_mn in (0, 1):
+                for b_mn in (0, 1):
+                    args = (A.T.contiguous() if a_mn else A, B.T.contiguous() if b_mn else B, M, N, K, a_mn, b_mn)
+                    C = wide.rl_selftest_gemm(*args)
+                    _assert_status_ok(wide)
+                    assert (C - ref).abs().max().item() <= 1e-4 * ref.abs().max().item()
+                    assert torch.equal(C, square.rl_selftest_gemm(*args))
+                    C2 = wide.rl_selftest_gemm(*args, C=C.clone(), accumulate=True)
+                    assert (C2 - 2 * ref).abs().max().item() <= 2e-4 * ref.abs().max().item()
+        for kw in (dict(cfg_id=0, L_max=13, V=4100, seed=710), dict(cfg_id=1, prompts=1, L_max=40, d=768, V=30000, seed=711),
+                   dict(cfg_id=1, prompts=1, L_max=24, d=2304, V=5000, seed=712)):
+            w = make_workload(kw.pop("cfg_id"), **kw)
+            a, _ = _check_against_oracle(wide, w)
+            a = {k: v.clone() for k, v in a.items()}
+            b, _ = _check_against_oracle(square, w)
+            for k in ("loss", "dH", "dW"):
+                assert torch.equal(a[k], b[k]), k
+    finally:
+        wide.close()
+        square.close()
+
+
 def test_single_cta_tiles_match_oracle():
     # the default context runs CTA pairs; the single-CTA tile shape must give the same results
     from paper_2512_21450_b200 import Context
