@@ -353,6 +353,20 @@ rl_status rl_selftest_gemm(rl_ctx* ctx, const void* A, const void* B, float* C,
                            int64_t M, int64_t N, int64_t K, int a_mn_major, int b_mn_major,
                            int accumulate);
 
+/* Host-only view of how a tensor-core pass distributes its work (no GPU is touched; the paper has
+ * no counterpart).  For a pass over n_valid rows (at most rows_cap), K extent k_len, n_tiles column
+ * tiles walked n_range at a time (0: chosen as the forward pass does), with the ordering options
+ * of the library (n_fastest, row groups of m_group row tiles, stream-K, K slices) on n_workers
+ * workers of cta_group CTAs each, writes one record of eight int32 per work unit, worker by worker
+ * in the order the worker walks them: {worker, row tile, first column tile, end column tile,
+ * output slice, first k-block, end k-block, k-blocks per tile}.  units (host, may be NULL when
+ * max_units is 0) receives at most max_units records, *n_units (host) the total.  It runs the very
+ * functions the kernels run, so that a test without a GPU can check that every (tile, k-block) is
+ * covered exactly once. */
+rl_status rl_debug_schedule(int64_t n_valid, int64_t rows_cap, int64_t k_len, int64_t n_tiles, int n_range,
+                            int n_fastest, int m_group, int stream_k, int k_split_max, int cta_group,
+                            int n_workers, int32_t* units, int64_t max_units, int64_t* n_units);
+
 /* Self-test of the bounded waits every kernel of this library uses: launches one warp that waits,
  * for at most limit_ms (1..1000) milliseconds, on a barrier nothing ever signals.  The kernel
  * returns by itself with RL_ERR_TIMEOUT latched (detail 0x70000000); rl_last_device_status()

@@ -105,6 +105,9 @@ def load_library():
     lib.rl_selftest_gemm.argtypes = [P, P, P, P, c_int64, c_int64, c_int64, c_int, c_int, c_int]
     lib.rl_token_logprobs_static.argtypes = [P, P, c_int64, P, c_int64, P, P, c_int64, c_int64, c_int64, P, P, P, P]
     lib.rl_token_logprobs_static.restype = c_int
+    lib.rl_debug_schedule.argtypes = [c_int64, c_int64, c_int64, c_int64, c_int, c_int, c_int, c_int, c_int, c_int, c_int,
+                                      P, c_int64, POINTER(c_int64)]
+    lib.rl_debug_schedule.restype = c_int
     lib.rl_mask_scan.argtypes = [P, P, c_int64, P, P]
     lib.rl_mask_scan.restype = c_int
     lib.rl_token_logprobs_multi.argtypes = [P, c_int, POINTER(c_void_p), POINTER(c_int64), POINTER(c_void_p),
@@ -464,6 +467,21 @@ class Context:
         _check(self.lib.rl_selftest_gemm(self.handle, _ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn_major),
                                          int(b_mn_major), int(accumulate)), "rl_selftest_gemm")
         return C
+
+
+def debug_schedule(n_valid, rows_cap, k_len, n_tiles, n_range=1, n_fastest=0, m_group=0, stream_k=0, k_split_max=1,
+                   cta_group=2, n_workers=74):
+    """Work units of one tensor-core pass as the kernels would walk them (host only, needs no GPU):
+    int32 array [n_units, 8] = worker, row tile, first / end column tile, output slice, first / end
+    k-block, k-blocks per tile."""
+    import numpy as np
+    lib = load_library()
+    n = c_int64()
+    args = (n_valid, rows_cap, k_len, n_tiles, n_range, n_fastest, m_group, stream_k, k_split_max, cta_group, n_workers)
+    _check(lib.rl_debug_schedule(*args, None, 0, byref(n)), "rl_debug_schedule")
+    out = np.zeros((n.value, 8), dtype=np.int32)
+    _check(lib.rl_debug_schedule(*args, out.ctypes.data_as(c_void_p), n.value, byref(n)), "rl_debug_schedule")
+    return out
 
 
 _default_ctx = {}

@@ -199,19 +199,19 @@ __host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_v
 }
 
 // Unit u -> row tile mu, column range nr and the K-block range [kb0, kb1) of its K slice ks.
-__device__ __forceinline__ void unit_coords(const GemmShape& sh, const GemmExtents& ex, int u, int& mu, int& nr,
+__host__ __device__ inline void unit_coords(const GemmShape& sh, const GemmExtents& ex, int u, int& mu, int& nr,
                                             int& ks, int& kb0, int& kb1) {
   ks = u % ex.k_split;
   u /= ex.k_split;
   kb0 = ks * ex.kb_per;
-  kb1 = min(kb0 + ex.kb_per, ex.k_blocks);
+  kb1 = kb0 + ex.kb_per < ex.k_blocks ? kb0 + ex.kb_per : ex.k_blocks;
   if (sh.n_fastest) {
     nr = u % ex.n_ranges; mu = u / ex.n_ranges;
   } else if (ex.m_group > 0) {
     const int per_group = ex.m_group * ex.n_ranges;
     const int gi = u / per_group, r = u - gi * per_group;
     const int m0 = gi * ex.m_group;
-    const int gsz = min(ex.m_group, ex.m_units - m0);
+    const int gsz = ex.m_group < ex.m_units - m0 ? ex.m_group : ex.m_units - m0;
     mu = m0 + r % gsz; nr = r / gsz;
   } else {
     mu = u % ex.m_units;  nr = u / ex.m_units;
@@ -229,7 +229,7 @@ struct UnitWalk {
   const GemmExtents& ex;
   int n_workers, u, plain_units;
   long long it, it_end;
-  __device__ __forceinline__ UnitWalk(const GemmShape& sh_, const GemmExtents& ex_, int worker, int n_workers_)
+  __host__ __device__ inline UnitWalk(const GemmShape& sh_, const GemmExtents& ex_, int worker, int n_workers_)
       : sh(sh_), ex(ex_), n_workers(n_workers_), u(worker), plain_units(ex_.n_units), it(0), it_end(0) {
     if (ex.stream_k) {
       plain_units = (ex.n_units / n_workers - 1) * n_workers;
@@ -238,7 +238,7 @@ struct UnitWalk {
       it_end = total * (worker + 1) / n_workers;
     }
   }
-  __device__ __forceinline__ bool next(int& mu, int& nr, int& ks, int& kb0, int& kb1) {
+  __host__ __device__ inline bool next(int& mu, int& nr, int& ks, int& kb0, int& kb1) {
     if (u < plain_units) {
       unit_coords(sh, ex, u, mu, nr, ks, kb0, kb1);
       u += n_workers;

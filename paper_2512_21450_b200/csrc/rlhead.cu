@@ -1239,6 +1239,44 @@ rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* c, const void* H_host, int64_t ldH
   return RL_OK;
 }
 
+rl_status rl_debug_schedule(int64_t n_valid, int64_t rows_cap, int64_t k_len, int64_t n_tiles, int n_range,
+                            int n_fastest, int m_group, int stream_k, int k_split_max, int cta_group,
+                            int n_workers, int32_t* units, int64_t max_units, int64_t* n_units) {
+  if (!n_units || n_valid < 0 || rows_cap <= 0 || k_len < 0 || n_tiles <= 0 || n_workers <= 0 || max_units < 0 ||
+      (cta_group != 1 && cta_group != 2) || (max_units > 0 && !units))
+    return RL_ERR_INVALID_ARG;
+  const int nv = (int)n_valid;
+  GemmShape sh;
+  memset(&sh, 0, sizeof(sh));
+  sh.n_valid = &nv;
+  sh.m_rows_cap = (int)rows_cap;
+  sh.m_dyn = 1;
+  sh.k_cap = (int)k_len;
+  sh.n_tiles = (int)n_tiles;
+  sh.n_range = n_range;
+  sh.n_fastest = n_fastest;
+  sh.m_group = m_group;
+  sh.stream_k = stream_k;
+  sh.k_split_max = k_split_max;
+  const GemmExtents ex = gemm_extents(sh, nv, cta_group, n_workers);
+  int64_t n = 0;
+  for (int worker = 0; worker < n_workers; ++worker) {
+    UnitWalk walk(sh, ex, worker, n_workers);
+    int mu, nr, ks, kb0, kb1;
+    while (walk.next(mu, nr, ks, kb0, kb1)) {
+      if (n < max_units) {
+        int32_t* o = units + n * 8;
+        o[0] = worker; o[1] = mu; o[2] = nr * ex.n_range;
+        o[3] = (nr + 1) * ex.n_range < sh.n_tiles ? (nr + 1) * ex.n_range : sh.n_tiles;
+        o[4] = ks; o[5] = kb0; o[6] = kb1; o[7] = ex.k_blocks;
+      }
+      ++n;
+    }
+  }
+  *n_units = n;
+  return RL_OK;
+}
+
 rl_status rl_selftest_wait_timeout(rl_ctx* c, int limit_ms) {
   if (!c || limit_ms < 1 || limit_ms > 1000) return RL_ERR_INVALID_ARG;
   wait_timeout_probe_kernel<<<1, 32, 0, c->stream>>>((unsigned long long)limit_ms * 1000000ull, c->dstatus);

@@ -81,3 +81,70 @@ def test_workload_structure_cpu():
     zero_var = (r.max(1).values == r.min(1).values).float().mean().item()
     assert 0.1 < zero_var < 0.45 and w4.ref_logp is None and w4.ent_coef == 1e-3 and w4.eps_high == 0.28
     assert CONFIGS[2]["V"] == 152064 and CONFIGS[2]["d"] == 3584
+
+
+def _check_schedule(n_valid, rows_cap, k_len, n_tiles, cta_group, n_workers, **kw):
+    """Every (row tile, column tile, k-block) of the pass is covered exactly once."""
+    from paper_2512_21450_b200.binding import debug_schedule
+    u = debug_schedule(n_valid, rows_cap, k_len, n_tiles, cta_group=cta_group, n_workers=n_workers, **kw)
+    rows = min(n_valid, rows_cap)
+    m_units = -(-rows // (128 * cta_group))
+    kb = -(-k_len // 64)
+    cover = np.zeros((m_units, n_tiles, max(kb, 1)), dtype=np.int32)
+    for worker, mu, c0, c1, ks, kb0, kb1, kpt in u:
+        assert 0 <= worker < n_workers and 0 <= mu < m_units and 0 <= c0 < c1 <= n_tiles and kpt == kb
+        assert 0 <= kb0 and kb1 <= kb               # kb1 <= kb0: an empty K slice, which the kernels fill with zeros
+        cover[mu, c0:c1, kb0:kb1] += 1
+        if kw.get("stream_k"):
+            assert ks == (1 if kb0 > 0 else 0) and kb1 > kb0
+    if kb > 0:
+        assert (cover == 1).all(), (n_valid, k_len, n_tiles, kw)
+    else:
+        assert len(u) == m_units * len({(r[2], r[3]) for r in u}) or len(u) == 0
+    return u
+
+
+def test_tile_schedules_cover_every_tile_once():
+    # the functions the kernels use to hand out work, run on the host: plain round-robin, column ranges,
+    # row groups (equal groups, ragged last group), stream-K (last full wave + ragged wave cut by k-blocks,
+    # at most two parts per tile) and K slices - on pairs and single CTAs, many sizes
+    rng = np.random.default_rng(0)
+    for _ in range(60):
+        cg = int(rng.integers(1, 3))
+        workers = int(rng.choice([3, 7, 74, 148]))
+        n_valid = int(rng.integers(1, 40000))
+        k_len = int(rng.choice([64, 72, 2048, 18944, 384]))
+        n_tiles = int(rng.integers(1, 80))
+        _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers)
+        _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_fastest=1)
+        _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_range=0)
+        _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_range=int(rng.integers(1, 9)),
+                        m_group=int(rng.integers(1, 40)))
+        _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_fastest=1, k_split_max=int(rng.integers(2, 5)))
+        u = _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_fastest=1, stream_k=1)
+        parts = {}
+        for worker, mu, c0, c1, ks, kb0, kb1, kpt in u:
+            parts.setdefault((mu, c0), []).append((kb0, kb1))
+        assert max(len(v) for v in parts.values()) <= 2
+    # the benchmark's dH pass with 256 x 256 tiles: 66 row tiles x 8 column tiles on 74 pairs, stream-K on
+    u = _check_schedule(16896, 32768, 18944, 8, 2, 74, n_fastest=1, stream_k=1)
+    work = np.zeros(74, dtype=np.int64)
+    for worker, mu, c0, c1, ks, kb0, kb1, kpt in u:
+        work[worker] += kb1 - kb0
+    assert work.max() - work.min() <= 1 and work.sum() == 66 * 8 * 296
+    # row groups: 66 row tiles with a budget of 36 tiles become two groups of 33; within a group all
+    # column ranges are walked before the next group starts
+    u = _check_schedule(16896, 32768, 2048, 74, 2, 74, m_group=36)
+    assert {int(r[1]) for r in u} == set(range(66))
+    for worker in (0, 37, 73):
+        seen_second = False
+        for r in u[u[:, 0] == worker]:
+            if r[1] >= 33:
+                seen_second = True
+            else:
+                assert not seen_second                 # a worker never returns to the first group
+        assert seen_second
+    # argument errors
+    from paper_2512_21450_b200.binding import RLHeadError, debug_schedule
+    with pytest.raises(RLHeadError):
+        debug_schedule(10, 0, 64, 1)
