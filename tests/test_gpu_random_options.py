@@ -1,0 +1,69 @@
+"""Seeded random sweep over shapes and over every ordering / tiling option of the library at once (CTA
+pairs or single CTAs, 256 x 512 or 256 x 256 gradient tiles, stream-K, K slices, row-group budgets, slab
+limits, fp32 or bf16 dH), each case against the float64 oracle within the stated tolerances.  The single
+options have tests of their own; this one looks for interactions between them on odd sizes."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import grpo_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _np64(t):
+    return t.detach().double().cpu().numpy()
+
+
+def _rel(a, b):
+    nb = np.linalg.norm(b)
+    return np.linalg.norm(a - b) / nb if nb > 0 else np.linalg.norm(a)
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_shapes_and_options(seed):
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    rng = np.random.default_rng(seed)
+    for _ in range(8):
+        cfg = int(rng.choice([0, 1, 3, 4]))
+        d = int(rng.choice([64, 128, 192, 256, 320, 512, 576, 1024, 1280]))
+        V = int(rng.integers(1, 6000))
+        w = make_workload(cfg, prompts=int(rng.integers(1, 3)), L_max=int(rng.integers(1, 300 if cfg != 3 else 120)),
+                          d=d, V=V, seed=int(rng.integers(1 << 30)), sigma_old=float(rng.choice([0.05, 0.3])))
+        opts = dict(cta_group=int(rng.choice([1, 2])), wide=int(rng.integers(0, 2)), stream_k=int(rng.integers(0, 2)),
+                    k_slices=int(rng.choice([1, 1, 2, 3])), group=int(rng.choice([0, 1 << 16, 1 << 19, 36 << 20])),
+                    slab=(int(rng.choice([128, 256, 1024, 32768])), int(rng.choice([256, 512, 2048, 18944]))),
+                    dH_fp32=bool(rng.integers(0, 2)))
+        c = Context(0)
+        try:
+            c.set_cta_group(opts["cta_group"])
+            c.set_wide_tiles(opts["wide"])
+            c.set_dh_stream_k(opts["stream_k"])
+            c.set_dh_k_slices(opts["k_slices"])
+            c.set_row_group_bytes(opts["group"])
+            c.set_slab_limits(*opts["slab"])
+            _, adv_tok = c.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+            out = c.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, w.eps_low,
+                                           w.eps_high, w.beta, ent_coef=w.ent_coef, dH_fp32=opts["dH_fp32"])
+            status, detail = c.last_device_status()
+            assert status == 0, (status, hex(detail & 0xffffffff), opts)
+        finally:
+            c.close()
+        o_adv = O.broadcast_to_tokens(O.grpo_advantages(w.rewards.cpu().numpy(), w.G), w.seq_offsets.cpu().numpy(), w.T)
+        oo = O.policy_loss_fwd_bwd(_np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), _np64(w.old_logp),
+                                   None if w.ref_logp is None else _np64(w.ref_logp), o_adv, w.mask.cpu().numpy(),
+                                   w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef)
+        where = (cfg, d, V, w.T, w.n_valid, opts)
+        assert np.abs(_np64(out["logp"]) - oo["logp"]).max() <= 2e-3, where
+        assert np.abs(_np64(out["entropy"]) - oo["entropy"]).max() <= 2e-3, where
+        rho = oo.get("rho", np.ones(1))
+        on_boundary = rho.size and np.minimum(np.abs(rho - (1 - w.eps_low)), np.abs(rho - (1 + w.eps_high))).min() <= 1e-5
+        if not on_boundary:      # a ratio on a clip boundary within fp32 rounding may fall on either side
+            # tiny batches of equal-length groups cancel to a loss near zero: the floor is that of the other tests, scaled
+            # to the handful of tokens a case here may have
+            assert abs(out["loss"].item() - oo["loss"]) <= 1e-3 * abs(oo["loss"]) + 1e-6, where
+            assert _rel(_np64(out["dH"]), oo["dH"]) <= 1e-2, where
+            assert _rel(_np64(out["dW"]), oo["dW"]) <= 1e-2, where
+        m = w.mask.cpu().numpy().astype(bool)
+        assert not _np64(out["dH"])[~m].any() and not _np64(out["logp"])[~m].any(), where
