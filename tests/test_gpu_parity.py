@@ -429,6 +429,19 @@ def test_row_groups(cta_group):
             out, _ = _check_against_oracle(c2, w)
             for k in ("loss", "dH", "dW", "logp", "entropy"):
                 assert torch.equal(out[k], base[k]), (tiles, k)
+        # the two-product passes of the full-distribution KL walk their tiles through the same function
+        from paper_2512_21450_b200.workloads import make_reference_model
+        H_ref, W_ref = make_reference_model(w, d_ref=128)
+        _, adv_tok = c2.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+        kl = []
+        for nbytes in (0, 2 * 128 * cta_group * (w.d + 128) * 2):
+            c2.set_row_group_bytes(nbytes)
+            o = c2.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, None, adv_tok, w.mask, w.eps_low, w.eps_high,
+                                          0.05, H_ref=H_ref, W_ref=W_ref)
+            _assert_status_ok(c2)
+            kl.append({k: v.clone() for k, v in o.items()})
+        for k in ("loss", "dH", "dW", "kl"):
+            assert torch.equal(kl[0][k], kl[1][k]), k
     finally:
         c2.close()
 
