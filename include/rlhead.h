@@ -314,8 +314,10 @@ rl_status rl_policy_loss_shard_bwd(rl_ctx* ctx, const void* H, int64_t ldH, cons
  * rl_token_logprobs; everything in between (compacted rows, row map, per-range softmax
  * statistics, the status word) lives in a fixed 16 MiB device array that is part of the library
  * image, so every GPU on which the library is loaded holds those 16 MiB until the process exits.
- *   Limit: the forward scratch, about Tpad*(2*d + 280) + 70 KB bytes with Tpad = T rounded up to
- *   128, must fit in 16 MiB - 256 B (e.g. T <= 3712 at d = 2048, T <= 1920 at d = 4096); larger
+ *   Limit: the forward scratch, about Tpad*(2*d + 28 + 16*R) + 70 KB bytes with Tpad = T rounded up
+ *   to 128 and R = max(16, ceil(ceil(V/256)/8)) vocabulary ranges, must fit in 16 MiB - 256 B (e.g.
+ *   T <= 3712 at d = 2048 for V <= 32768; T <= 3072 at d = 2048 and T <= 1664 at d = 4096 for the
+ *   151936-word vocabulary, where R = 75); larger
  *   sizes are rejected with RL_ERR_WORKSPACE before anything is enqueued.
  *   The call runs on the CURRENT device (device ordinal < 16) and enqueues on cuda_stream.  The
  *   first call on each device looks up the array's device address and configures the kernel; make
