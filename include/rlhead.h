@@ -305,6 +305,32 @@ rl_status rl_policy_loss_shard_bwd(rl_ctx* ctx, const void* H, int64_t ldH, cons
                                    float* loss, void* dH_partial, float* dW_shard,
                                    const rl_loss_opts* opts);
 
+/* The same step split in two, so that the host-to-device copies of one step overlap the kernels of
+ * the step before it (a trainer that receives rollout batches in host memory: Algorithm 1 runs
+ * mu policy updates per sampled batch).  rl_policy_loss_fwd_bwd_host_submit copies the inputs of a
+ * step on a copy stream that belongs to the context into staging slot `slot` (0 or 1), makes the
+ * context's stream wait for them, enqueues the step there and returns without synchronising;
+ * rl_policy_loss_fwd_bwd_host_wait blocks until the step submitted to that slot has finished and
+ * returns its loss and metrics.  A slot must be waited for before it is submitted to again
+ * (RL_ERR_INVALID_ARG otherwise); steps run in submission order and share dH / dW as the caller
+ * passes them, so a step's dH and dW are valid between its wait and the submit after next at the
+ * latest - with one dH / dW pair, read them before submitting the next step, or alternate two pairs.
+ * The host buffers of a step must stay untouched until its wait returns; pinned memory is needed for
+ * the copies to be asynchronous.  Workspace: rl_workspace_bytes_host_pipelined() (two staging
+ * slots).  The first submit on a context creates the copy stream, four events and 128 bytes of
+ * pinned memory, released by rl_destroy. */
+rl_status rl_workspace_bytes_host_pipelined(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_t* bytes);
+rl_status rl_policy_loss_fwd_bwd_host_submit(rl_ctx* ctx, int slot, const void* H_host, int64_t ldH,
+                                             const void* W, int64_t ldW, const int32_t* tokens_host,
+                                             const float* old_logp_host, const float* ref_logp_host,
+                                             const float* adv_host, const float* rewards_host,
+                                             int64_t n_seq, int group_size,
+                                             const int32_t* seq_offsets_host, const uint8_t* mask_host,
+                                             int64_t T, int64_t d, int64_t V,
+                                             float eps_low, float eps_high, float beta, float ent_coef,
+                                             void* dH, float* dW);
+rl_status rl_policy_loss_fwd_bwd_host_wait(rl_ctx* ctx, int slot, float* loss_host, float* metrics_host);
+
 /* rl_token_logprobs without any device allocation and without a context (the paper has no
  * counterpart).  It is meant for callers that cannot allocate GPU memory when they need
  * log-probabilities: a scoring pass that shares the GPU with a rollout engine which has already

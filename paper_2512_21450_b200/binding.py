@@ -99,6 +99,13 @@ def load_library():
     lib.rl_policy_loss_fwd_bwd_host.argtypes = [P, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int, P, P,
                                                 c_int64, c_int64, c_int64,
                                                 c_float, c_float, c_float, c_float, P, P, P, P]
+    lib.rl_workspace_bytes_host_pipelined.argtypes = [P, c_int64, c_int64, c_int64, POINTER(c_size_t)]
+    lib.rl_workspace_bytes_host_pipelined.restype = c_int
+    lib.rl_policy_loss_fwd_bwd_host_submit.argtypes = [P, c_int, P, c_int64, P, c_int64, P, P, P, P, P, c_int64, c_int, P, P,
+                                                       c_int64, c_int64, c_int64, c_float, c_float, c_float, c_float, P, P]
+    lib.rl_policy_loss_fwd_bwd_host_submit.restype = c_int
+    lib.rl_policy_loss_fwd_bwd_host_wait.argtypes = [P, c_int, P, P]
+    lib.rl_policy_loss_fwd_bwd_host_wait.restype = c_int
     lib.rl_launch_count.argtypes = [P, POINTER(c_int64)]
     lib.rl_set_profiling.argtypes = [P, c_int]
     lib.rl_profile_read.argtypes = [P, POINTER(ctypes.c_double), POINTER(c_int64)]
@@ -154,6 +161,7 @@ class Context:
         _check(self.lib.rl_create(byref(self.handle), device), "rl_create")
         self._ws = None
         self._ws_key = None
+        self._slot_busy = [False, False]
 
     def close(self):
         if self.handle:
@@ -458,6 +466,38 @@ class Context:
             _ptr(seq_offsets_host), _ptr(mask_host), T, d, V, eps_low, eps_high, beta, ent_coef,
             ctypes.cast(loss, c_void_p), ctypes.cast(metrics, c_void_p), _ptr(dH), _ptr(dW)),
             "rl_policy_loss_fwd_bwd_host")
+        return loss[0], list(metrics)
+
+    def rl_policy_loss_fwd_bwd_host_submit(self, slot, H_host, W, tokens_host, old_host, ref_host, adv_host, mask_host,
+                                           eps_low, eps_high, beta, ent_coef, dH, dW, rewards_host=None, group_size=0,
+                                           seq_offsets_host=None):
+        """First half of a pipelined host-buffer step: enqueue copies and kernels, do not wait."""
+        self._bind_stream()
+        T, d = H_host.shape
+        V = W.shape[0]
+        need = c_size_t()
+        _check(self.lib.rl_workspace_bytes_host_pipelined(self.handle, T, d, V, byref(need)),
+               "rl_workspace_bytes_host_pipelined")
+        if self._ws is None or self._ws.numel() < need.value:
+            assert not any(self._slot_busy), "workspace must not be replaced while a step is in flight"
+            self._ws = None
+            self._ws = torch.empty(need.value, dtype=torch.uint8, device=self.device)
+        _check(self.lib.rl_set_workspace(self.handle, _ptr(self._ws), self._ws.numel()), "rl_set_workspace")
+        _check(self.lib.rl_policy_loss_fwd_bwd_host_submit(
+            self.handle, slot, _ptr(H_host), d, _ptr(W), W.stride(0), _ptr(tokens_host), _ptr(old_host), _ptr(ref_host),
+            _ptr(adv_host), _ptr(rewards_host), rewards_host.numel() if rewards_host is not None else 0, group_size,
+            _ptr(seq_offsets_host), _ptr(mask_host), T, d, V, eps_low, eps_high, beta, ent_coef, _ptr(dH), _ptr(dW)),
+            "rl_policy_loss_fwd_bwd_host_submit")
+        self._slot_busy[slot] = True
+
+    def rl_policy_loss_fwd_bwd_host_wait(self, slot):
+        """Second half: block until the step submitted to `slot` is done; returns (loss, metrics)."""
+        loss = (c_float * 1)()
+        metrics = (c_float * 8)()
+        _check(self.lib.rl_policy_loss_fwd_bwd_host_wait(self.handle, slot, ctypes.cast(loss, c_void_p),
+                                                         ctypes.cast(metrics, c_void_p)),
+               "rl_policy_loss_fwd_bwd_host_wait")
+        self._slot_busy[slot] = False
         return loss[0], list(metrics)
 
     def rl_selftest_gemm(self, A, B, M, N, K, a_mn_major, b_mn_major, C=None, accumulate=False):

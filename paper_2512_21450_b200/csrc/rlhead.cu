@@ -43,6 +43,11 @@ struct rl_ctx {
   // optional per-kernel timing: event pairs around every tensor-core launch, by kernel kind
   int prof_on;
   int prof_used;
+  // pipelined host-buffer steps: a copy stream, per-slot events and pinned result words (created on first use)
+  cudaStream_t copy_stream;
+  cudaEvent_t copy_done[2], step_done[2];
+  float* pinned_out[2];
+  int slot_busy[2];
   int* prof_kind;                 // [kProfMax], allocated when profiling is first switched on
   cudaEvent_t (*prof_ev)[2];      // [kProfMax][2], events created on first use
 };
@@ -75,8 +80,36 @@ struct KlRef {
   int64_t d_ref;
 };
 
-// staging_T > 0 adds room for host-call inputs (H, tokens, old, ref, adv, mask).
-WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_staging, int64_t d_ref = 0) {
+// Device copies of one step's host inputs (H, tokens, old, ref, adv, mask, rewards, offsets) and its result words.
+struct HostStage {
+  void* H;
+  int32_t* tok;
+  float *old_lp, *ref_lp, *adv;
+  uint8_t* mask;
+  float* out;       // [16]: loss, 7 unused, 8 metrics
+  float *rew, *advseq;
+  int32_t* off;
+};
+inline size_t carve_stage(char* base, int64_t T, int64_t d, HostStage* hs) {
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 1024); return base ? base + at : nullptr; };
+  HostStage h;
+  h.H = take((size_t)T * d * 2);
+  h.tok = reinterpret_cast<int32_t*>(take((size_t)T * 4));
+  h.old_lp = reinterpret_cast<float*>(take((size_t)T * 4));
+  h.ref_lp = reinterpret_cast<float*>(take((size_t)T * 4));
+  h.adv = reinterpret_cast<float*>(take((size_t)T * 4));
+  h.mask = reinterpret_cast<uint8_t*>(take((size_t)T));
+  h.out = reinterpret_cast<float*>(take(64));
+  h.rew = reinterpret_cast<float*>(take((size_t)T * 4));
+  h.advseq = reinterpret_cast<float*>(take((size_t)T * 4));
+  h.off = reinterpret_cast<int32_t*>(take((size_t)(T + 1) * 4));
+  if (hs) *hs = h;
+  return o;
+}
+
+// host_slots > 0 adds room for that many sets of host-call inputs behind the scratch proper.
+WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, int host_slots, int64_t d_ref = 0) {
   WsLayout L;
   L.Tpad = (int)align_up((size_t)(T > 0 ? T : 1), 128);
   L.Ts = L.Tpad < c->slab_rows ? L.Tpad : c->slab_rows;
@@ -112,18 +145,7 @@ WsLayout ws_layout(const rl_ctx* c, int64_t T, int64_t d, int64_t V, bool host_s
     L.cb_c = take((size_t)L.Tpad * 4);
   }
   L.staging = o;
-  if (host_staging) {
-    take((size_t)T * d * 2);  // H
-    take((size_t)T * 4);      // tokens
-    take((size_t)T * 4);      // old
-    take((size_t)T * 4);      // ref
-    take((size_t)T * 4);      // adv
-    take((size_t)T);          // mask
-    take(64);                 // loss + metrics
-    take((size_t)T * 4);      // rewards
-    take((size_t)T * 4);      // per-response advantages
-    take((size_t)(T + 1) * 4);  // seq_offsets
-  }
+  o += (size_t)host_slots * carve_stage(nullptr, T, d, nullptr);
   L.total = o;
   return L;
 }
@@ -457,6 +479,8 @@ rl_status rl_create(rl_ctx** out, int device) {
   c->prof_used = 0;
   c->prof_kind = nullptr;
   c->prof_ev = nullptr;
+  c->copy_stream = nullptr;
+  for (int i = 0; i < 2; ++i) { c->copy_done[i] = nullptr; c->step_done[i] = nullptr; c->pinned_out[i] = nullptr; c->slot_busy[i] = 0; }
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -514,6 +538,15 @@ rl_status rl_destroy(rl_ctx* c) {
         if (c->prof_ev[i][e]) cudaEventDestroy(c->prof_ev[i][e]);
     delete[] c->prof_ev;
     delete[] c->prof_kind;
+  }
+  if (c->copy_stream) {
+    cudaStreamSynchronize(c->copy_stream);
+    cudaStreamDestroy(c->copy_stream);
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(c->copy_done[i]);
+      cudaEventDestroy(c->step_done[i]);
+      cudaFreeHost(c->pinned_out[i]);
+    }
   }
   cudaFree(c->dstatus);
   delete c;
@@ -1178,6 +1211,71 @@ rl_status rl_policy_loss_fwd_bwd(rl_ctx* c, const void* H, int64_t ldH, const vo
                                    eps_high, beta, loss, dH, dW, nullptr);
 }
 
+// Arguments of one host-buffer step (all per-step inputs are host pointers).
+struct HostStepArgs {
+  const void* H_host;
+  int64_t ldH;
+  const void* W;
+  int64_t ldW;
+  const int32_t* tokens_host;
+  const float *old_host, *ref_host, *adv_host, *rewards_host;
+  int64_t n_seq;
+  int group_size;
+  const int32_t* seq_offsets_host;
+  const uint8_t* mask_host;
+  int64_t T, d, V;
+  float eps_low, eps_high, beta, ent_coef;
+  void* dH;
+  float* dW;
+};
+
+static rl_status host_step_check(const rl_ctx* c, const HostStepArgs& a) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  if (a.T < 0 || a.d <= 0 || a.V <= 0) return RL_ERR_INVALID_ARG;
+  if (a.T > 0 && (!a.H_host || !a.tokens_host || !a.old_host)) return RL_ERR_INVALID_ARG;
+  if (a.T > 0 && !a.adv_host && (!a.rewards_host || !a.seq_offsets_host || a.n_seq <= 0 || a.n_seq > a.T))
+    return RL_ERR_INVALID_ARG;
+  if (a.ldH != a.d) return RL_ERR_SHAPE;  // host rows are copied as one block
+  return RL_OK;
+}
+
+// Copies the step's inputs into the stage on `copy` (the context's stream itself, or the copy stream, in
+// which case the context's stream waits for copy_done) and enqueues advantages + loss forward/backward on
+// the context's stream; the result words end up in hs.out.
+static rl_status host_step_enqueue(rl_ctx* c, const HostStage& hs, cudaStream_t copy, cudaEvent_t copy_done,
+                                   const HostStepArgs& a) {
+  const int64_t T = a.T;
+  if (T > 0) {
+    cudaMemcpyAsync(hs.H, a.H_host, (size_t)T * a.d * 2, cudaMemcpyHostToDevice, copy);
+    cudaMemcpyAsync(hs.tok, a.tokens_host, (size_t)T * 4, cudaMemcpyHostToDevice, copy);
+    cudaMemcpyAsync(hs.old_lp, a.old_host, (size_t)T * 4, cudaMemcpyHostToDevice, copy);
+    if (a.ref_host) cudaMemcpyAsync(hs.ref_lp, a.ref_host, (size_t)T * 4, cudaMemcpyHostToDevice, copy);
+    if (a.adv_host) {
+      cudaMemcpyAsync(hs.adv, a.adv_host, (size_t)T * 4, cudaMemcpyHostToDevice, copy);
+    } else {
+      cudaMemcpyAsync(hs.rew, a.rewards_host, (size_t)a.n_seq * 4, cudaMemcpyHostToDevice, copy);
+      cudaMemcpyAsync(hs.off, a.seq_offsets_host, (size_t)(a.n_seq + 1) * 4, cudaMemcpyHostToDevice, copy);
+    }
+    if (a.mask_host) cudaMemcpyAsync(hs.mask, a.mask_host, (size_t)T, cudaMemcpyHostToDevice, copy);
+  }
+  if (copy != c->stream) {
+    if (cudaEventRecord(copy_done, copy) != cudaSuccess || cudaStreamWaitEvent(c->stream, copy_done, 0) != cudaSuccess)
+      return RL_ERR_CUDA;
+  }
+  if (T > 0 && !a.adv_host) {
+    rl_status sa = rl_grpo_advantages_ex(c, hs.rew, a.n_seq, a.group_size, 1, 1e-6f, hs.off, T, hs.advseq, hs.adv);
+    if (sa != RL_OK) return sa;
+  }
+  rl_loss_opts opts;
+  memset(&opts, 0, sizeof(opts));
+  opts.struct_size = sizeof(opts);
+  opts.ent_coef = a.ent_coef;
+  opts.metrics_out = hs.out + 8;
+  return rl_policy_loss_fwd_bwd_ex(c, hs.H, a.d, a.W, a.ldW, hs.tok, hs.old_lp, a.ref_host ? hs.ref_lp : nullptr, hs.adv,
+                                   a.mask_host ? hs.mask : nullptr, T, a.d, a.V, a.eps_low, a.eps_high, a.beta, hs.out,
+                                   a.dH, a.dW, &opts);
+}
+
 rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* c, const void* H_host, int64_t ldH, const void* W, int64_t ldW,
                                       const int32_t* tokens_host, const float* old_host, const float* ref_host,
                                       const float* adv_host, const float* rewards_host, int64_t n_seq,
@@ -1185,57 +1283,71 @@ rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* c, const void* H_host, int64_t ldH
                                       const uint8_t* mask_host, int64_t T, int64_t d,
                                       int64_t V, float eps_low, float eps_high, float beta, float ent_coef,
                                       float* loss_host, float* metrics_host, void* dH, float* dW) {
-  if (!c || !loss_host) return RL_ERR_INVALID_ARG;
-  if (T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
-  if (T > 0 && (!H_host || !tokens_host || !old_host)) return RL_ERR_INVALID_ARG;
-  if (T > 0 && !adv_host && (!rewards_host || !seq_offsets_host || n_seq <= 0 || n_seq > T)) return RL_ERR_INVALID_ARG;
-  if (ldH != d) return RL_ERR_SHAPE;  // host rows are copied as one block
-  const WsLayout L = ws_layout(c, T, d, V, true);
-  rl_status s = check_ws(c, L);
+  if (!loss_host) return RL_ERR_INVALID_ARG;
+  const HostStepArgs a = {H_host, ldH, W, ldW, tokens_host, old_host, ref_host, adv_host, rewards_host, n_seq, group_size,
+                          seq_offsets_host, mask_host, T, d, V, eps_low, eps_high, beta, ent_coef, dH, dW};
+  rl_status s = host_step_check(c, a);
   if (s != RL_OK) return s;
-  char* ws = static_cast<char*>(c->ws);
-  size_t o = L.staging;
-  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 1024); return ws + at; };
-  void* dH_in = take((size_t)T * d * 2);
-  int32_t* d_tok = reinterpret_cast<int32_t*>(take((size_t)T * 4));
-  float* d_old = reinterpret_cast<float*>(take((size_t)T * 4));
-  float* d_ref = reinterpret_cast<float*>(take((size_t)T * 4));
-  float* d_adv = reinterpret_cast<float*>(take((size_t)T * 4));
-  uint8_t* d_mask = reinterpret_cast<uint8_t*>(take((size_t)T));
-  float* d_out = reinterpret_cast<float*>(take(64));
-  float* d_rew = reinterpret_cast<float*>(take((size_t)T * 4));
-  float* d_advseq = reinterpret_cast<float*>(take((size_t)T * 4));
-  int32_t* d_off = reinterpret_cast<int32_t*>(take((size_t)(T + 1) * 4));
-  cudaStream_t st = c->stream;
-  if (T > 0) {
-    cudaMemcpyAsync(dH_in, H_host, (size_t)T * d * 2, cudaMemcpyHostToDevice, st);
-    cudaMemcpyAsync(d_tok, tokens_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
-    cudaMemcpyAsync(d_old, old_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
-    if (ref_host) cudaMemcpyAsync(d_ref, ref_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
-    if (adv_host) {
-      cudaMemcpyAsync(d_adv, adv_host, (size_t)T * 4, cudaMemcpyHostToDevice, st);
-    } else {
-      cudaMemcpyAsync(d_rew, rewards_host, (size_t)n_seq * 4, cudaMemcpyHostToDevice, st);
-      cudaMemcpyAsync(d_off, seq_offsets_host, (size_t)(n_seq + 1) * 4, cudaMemcpyHostToDevice, st);
-      rl_status sa = rl_grpo_advantages_ex(c, d_rew, n_seq, group_size, 1, 1e-6f, d_off, T, d_advseq, d_adv);
-      if (sa != RL_OK) return sa;
-    }
-    if (mask_host) cudaMemcpyAsync(d_mask, mask_host, (size_t)T, cudaMemcpyHostToDevice, st);
-  }
-  rl_loss_opts opts;
-  memset(&opts, 0, sizeof(opts));
-  opts.struct_size = sizeof(opts);
-  opts.ent_coef = ent_coef;
-  opts.metrics_out = d_out + 8;
-  s = rl_policy_loss_fwd_bwd_ex(c, dH_in, d, W, ldW, d_tok, d_old, ref_host ? d_ref : nullptr, d_adv,
-                                mask_host ? d_mask : nullptr, T, d, V, eps_low, eps_high, beta, d_out, dH, dW,
-                                &opts);
-  if (s != RL_OK) return s;
+  const WsLayout L = ws_layout(c, T, d, V, 1);
+  if ((s = check_ws(c, L)) != RL_OK) return s;
+  HostStage hs;
+  carve_stage(static_cast<char*>(c->ws) + L.staging, T, d, &hs);
+  if ((s = host_step_enqueue(c, hs, c->stream, nullptr, a)) != RL_OK) return s;
   float h_out[16];
-  if (cudaMemcpyAsync(h_out, d_out, sizeof(h_out), cudaMemcpyDeviceToHost, st) != cudaSuccess) return RL_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return RL_ERR_CUDA;
+  if (cudaMemcpyAsync(h_out, hs.out, sizeof(h_out), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess) return RL_ERR_CUDA;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return RL_ERR_CUDA;
   loss_host[0] = h_out[0];
   if (metrics_host) memcpy(metrics_host, h_out + 8, 32);
+  return RL_OK;
+}
+
+rl_status rl_workspace_bytes_host_pipelined(rl_ctx* c, int64_t T, int64_t d, int64_t V, size_t* bytes) {
+  if (!c || !bytes || T < 0 || d <= 0 || V <= 0) return RL_ERR_INVALID_ARG;
+  *bytes = ws_layout(c, T, d, V, 2).total;
+  return RL_OK;
+}
+
+rl_status rl_policy_loss_fwd_bwd_host_submit(rl_ctx* c, int slot, const void* H_host, int64_t ldH, const void* W,
+                                             int64_t ldW, const int32_t* tokens_host, const float* old_host,
+                                             const float* ref_host, const float* adv_host,
+                                             const float* rewards_host, int64_t n_seq, int group_size,
+                                             const int32_t* seq_offsets_host, const uint8_t* mask_host, int64_t T,
+                                             int64_t d, int64_t V, float eps_low, float eps_high, float beta,
+                                             float ent_coef, void* dH, float* dW) {
+  const HostStepArgs a = {H_host, ldH, W, ldW, tokens_host, old_host, ref_host, adv_host, rewards_host, n_seq, group_size,
+                          seq_offsets_host, mask_host, T, d, V, eps_low, eps_high, beta, ent_coef, dH, dW};
+  rl_status s = host_step_check(c, a);
+  if (s != RL_OK) return s;
+  if (slot < 0 || slot > 1 || c->slot_busy[slot]) return RL_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(c, T, d, V, 2);
+  if ((s = check_ws(c, L)) != RL_OK) return s;
+  if (!c->copy_stream) {
+    // first pipelined call on this context: the copy stream, two events and 64 pinned bytes per slot
+    bool ok = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaEventCreateWithFlags(&c->copy_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->step_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaHostAlloc(reinterpret_cast<void**>(&c->pinned_out[i]), 64, cudaHostAllocDefault) == cudaSuccess;
+    if (!ok) return RL_ERR_CUDA;
+  }
+  HostStage hs;
+  const size_t stage = carve_stage(nullptr, T, d, nullptr);
+  carve_stage(static_cast<char*>(c->ws) + L.staging + (size_t)slot * stage, T, d, &hs);
+  // the stage of this slot is free: its previous step was waited for (slot_busy is clear)
+  if ((s = host_step_enqueue(c, hs, c->copy_stream, c->copy_done[slot], a)) != RL_OK) return s;
+  if (cudaMemcpyAsync(c->pinned_out[slot], hs.out, 64, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+      cudaEventRecord(c->step_done[slot], c->stream) != cudaSuccess)
+    return RL_ERR_CUDA;
+  c->slot_busy[slot] = 1;
+  return RL_OK;
+}
+
+rl_status rl_policy_loss_fwd_bwd_host_wait(rl_ctx* c, int slot, float* loss_host, float* metrics_host) {
+  if (!c || slot < 0 || slot > 1 || !loss_host || !c->slot_busy[slot]) return RL_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(c->step_done[slot]) != cudaSuccess) return RL_ERR_CUDA;
+  c->slot_busy[slot] = 0;
+  loss_host[0] = c->pinned_out[slot][0];
+  if (metrics_host) memcpy(metrics_host, c->pinned_out[slot] + 8, 32);
   return RL_OK;
 }
 

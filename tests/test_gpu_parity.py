@@ -664,6 +664,61 @@ def test_host_buffer_step_matches_device_call(ctx):
         assert loss2 == ref["loss"].item() and torch.equal(dW, ref["dW"])
 
 
+def test_pipelined_host_steps_match_the_blocking_call():
+    # steps submitted two deep (the copies of step i+1 overlap the kernels of step i) must give exactly
+    # what the blocking host call gives for each step's own inputs, with two workloads of the same shape
+    # alternating so that a stale stage or result word would show; slot protocol errors are reported
+    from paper_2512_21450_b200 import Context, RLHeadError
+    from paper_2512_21450_b200.workloads import make_workload
+    c = Context(0)
+    try:
+        ws = [make_workload(4, prompts=2, L_max=16, seed=95 + i, d=256, V=5000) for i in range(2)]
+        pin = lambda x: None if x is None else x.cpu().pin_memory()  # noqa: E731
+        hosts, expect = [], []
+        for w in ws:
+            h = dict(H=pin(w.H), tok=pin(w.tokens), old=pin(w.old_logp), ref=pin(w.ref_logp), mask=pin(w.mask),
+                     rew=pin(w.rewards), off=pin(w.seq_offsets))
+            hosts.append(h)
+            dH = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+            dW = torch.empty(w.V, w.d, dtype=torch.float32, device="cuda")
+            loss, metrics = c.rl_policy_loss_fwd_bwd_host(h["H"], w.W, h["tok"], h["old"], h["ref"], None, h["mask"], w.eps_low,
+                                                          w.eps_high, w.beta, w.ent_coef, dH, dW, rewards_host=h["rew"],
+                                                          group_size=w.G, seq_offsets_host=h["off"])
+            expect.append((loss, metrics, dH.clone(), dW.clone()))
+        assert expect[0][0] != expect[1][0]
+        outs = [(torch.empty_like(expect[0][2]), torch.empty_like(expect[0][3])) for _ in range(2)]   # one dH / dW pair per slot
+
+        def submit(step):
+            k = step % 2
+            w, h = ws[k], hosts[k]
+            c.rl_policy_loss_fwd_bwd_host_submit(k, h["H"], w.W, h["tok"], h["old"], h["ref"], None, h["mask"], w.eps_low,
+                                                 w.eps_high, w.beta, w.ent_coef, outs[k][0], outs[k][1],
+                                                 rewards_host=h["rew"], group_size=w.G, seq_offsets_host=h["off"])
+
+        n_steps = 7
+        submit(0)
+        for step in range(1, n_steps + 1):
+            if step < n_steps:
+                submit(step)
+            k = (step - 1) % 2
+            loss, metrics = c.rl_policy_loss_fwd_bwd_host_wait(k)
+            assert loss == expect[k][0] and metrics == expect[k][1], step
+            assert torch.equal(outs[k][0], expect[k][2]) and torch.equal(outs[k][1], expect[k][3]), step
+        status, detail = c.last_device_status()
+        assert status == 0, (status, detail)
+        # protocol: waiting on an idle slot, submitting to a busy one, a slot that does not exist
+        with pytest.raises(RLHeadError):
+            c.rl_policy_loss_fwd_bwd_host_wait(0)
+        submit(0)
+        with pytest.raises(RLHeadError):
+            submit(0)
+        with pytest.raises(RLHeadError):
+            c.rl_policy_loss_fwd_bwd_host_wait(2)
+        c.rl_policy_loss_fwd_bwd_host_wait(0)
+    finally:
+        c.close()
+
+
 def test_autograd_front_end(ctx):
     from paper_2512_21450_b200.autograd import fused_grpo_head_loss
     from paper_2512_21450_b200.workloads import make_workload
