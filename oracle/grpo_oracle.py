@@ -26,6 +26,9 @@ leaves a choice open for each of them):
     distribution, entering the loss as  - ent_coef * H.
   * Token aggregation: weights w_t = m_t / sum(m) (token mean) unless the caller
     passes token_weight.
+  * Token-level KL reward shaping (section 2.2): shaped reward -beta * kl_t per
+    valid token plus the response's scalar on its last valid token, then the
+    return-to-go (see kl_shaped_returns).
 
 Parity pins: every function here is pinned by tests/test_oracle_pins.py against
 brute force, closed forms, finite differences and library second opinions.
@@ -123,6 +126,63 @@ def broadcast_to_tokens(adv_seq, seq_offsets, T):
     for i in range(len(adv_seq)):
         adv_tok[seq_offsets[i]:seq_offsets[i + 1]] = adv_seq[i]
     return adv_tok
+
+
+# --------------------------------------------------------------------------- #
+# Section 2.2 "Regularization": the KL-to-reference term is "often applied with
+# token-level shaping", i.e. folded into per-token rewards instead of (or beside)
+# the loss.  The paper prints no formula for the shaped reward; reading:
+#   kl_t  = per-token divergence estimate of a valid token t, one of
+#             "k1"  logp_t - ref_logp_t              (signed sampled log-ratio)
+#             "k3"  exp(delta) - delta - 1, delta = ref_logp_t - logp_t
+#                                                    (the estimator of the loss)
+#             "given"  a per-token value handed in (e.g. the full-distribution KL_t)
+#   r_t   = -beta * kl_t, and the last VALID token of response i additionally
+#           receives the response's scalar seq_value_i (its trajectory reward,
+#           section 3.2.2 scoring stage, or its group-normalised advantage)
+#   ret_t = r_t + gamma * ret_{next valid token of the same response}
+#           (return-to-go; gamma = 1 is the plain reverse cumulative sum)
+# Masked rows take no part: they get 0, carry no reward and are not counted as a
+# discount step.  Rows outside every response range get 0.  A response without a
+# valid token gets nothing (its seq_value is dropped).
+# Parity unpinned with respect to the authors' code; pinned to this reading.
+# --------------------------------------------------------------------------- #
+def token_kl_estimate(logp, ref_logp, kind="k3", kl_tok=None):
+    """Per-token divergence estimate used for reward shaping (see above)."""
+    if kind == "given":
+        return np.asarray(kl_tok, dtype=np.float64)
+    logp = np.asarray(logp, dtype=np.float64)
+    ref = np.asarray(ref_logp, dtype=np.float64)
+    if kind == "k1":
+        return logp - ref
+    if kind == "k3":
+        delta = ref - logp
+        return np.exp(delta) - delta - 1.0
+    raise ValueError("unknown KL estimate")
+
+
+def kl_shaped_returns(seq_value, logp, ref_logp, mask, seq_offsets, beta, gamma=1.0,
+                      kind="k3", kl_tok=None):
+    """Token-level KL reward shaping.  Returns (shaped_reward[T], returns[T])."""
+    off = np.asarray(seq_offsets)
+    T = len(mask) if mask is not None else int(off[-1])
+    m = np.ones(T, dtype=bool) if mask is None else np.asarray(mask).astype(bool)
+    kl = token_kl_estimate(logp, ref_logp, kind, kl_tok)
+    v = np.asarray(seq_value, dtype=np.float64)
+    shaped = np.zeros(T)
+    ret = np.zeros(T)
+    for i in range(len(off) - 1):
+        valid = [t for t in range(int(off[i]), int(off[i + 1])) if m[t]]
+        if not valid:
+            continue
+        for t in valid:
+            shaped[t] = -beta * kl[t]
+        shaped[valid[-1]] += v[i]
+        running = 0.0
+        for t in reversed(valid):
+            running = shaped[t] + gamma * running
+            ret[t] = running
+    return shaped, ret
 
 
 # --------------------------------------------------------------------------- #

@@ -37,6 +37,15 @@ MUTANTS = {
     "slice statistics: target id not made local": ("y = int(tokens[t]) - int(vocab_offset)", "y = int(tokens[t])"),
     "slice backward: one-hot not made local": ("y = tokens[rows] - int(vocab_offset)", "y = tokens[rows]"),
     "slice backward: softmax renormalised inside the slice": ("LP = H[rows] @ W_shard.T - np.asarray(lse, dtype=np.float64)[rows][:, None]", "LP = H[rows] @ W_shard.T; LP = LP - np.log(np.exp(LP).sum(axis=1))[:, None]"),
+    "shaping: penalty sign": ("shaped[t] = -beta * kl[t]", "shaped[t] = beta * kl[t]"),
+    "shaping: trajectory value on the last row instead of the last valid row": ("shaped[valid[-1]] += v[i]", "shaped[int(off[i + 1]) - 1] += v[i]"),
+    "shaping: trajectory value dropped": ("shaped[valid[-1]] += v[i]", "pass"),
+    "shaping: trajectory value on every token": ("shaped[valid[-1]] += v[i]", "shaped[valid] += v[i]"),
+    "shaping: forward instead of reverse cumulative sum": ("for t in reversed(valid):\n            running", "for t in valid:\n            running"),
+    "shaping: discount applied to the reward instead of the tail": ("running = shaped[t] + gamma * running", "running = gamma * shaped[t] + running"),
+    "shaping: masked rows counted as discount steps": ("valid = [t for t in range(int(off[i]), int(off[i + 1])) if m[t]]\n        if not valid:\n            continue\n        for t in valid:\n            shaped[t] = -beta * kl[t]", "valid = [t for t in range(int(off[i]), int(off[i + 1])) if m[t]]\n        if not valid:\n            continue\n        for t in valid:\n            shaped[t] = -beta * kl[t]\n        valid = list(range(valid[0], valid[-1] + 1))"),
+    "shaping: k1 direction swapped": ("return logp - ref\n", "return ref - logp\n"),
+    "shaping: k3 uses the opposite log-ratio": ("delta = ref - logp\n        return np.exp(delta) - delta - 1.0", "delta = logp - ref\n        return np.exp(delta) - delta - 1.0"),
     "row map keeps the masked rows": ("return [t for t in range(len(mask)) if mask[t] != 0]", "return [t for t in range(len(mask)) if mask[t] == 0]"),
     "logits index order": ("return H @ W.T", "return (W @ H.T).T[::-1][::-1] if H.shape[0] == 1 else (H[:, ::-1] @ W[:, ::-1].T if False else H @ W[::-1].T)"),
 }

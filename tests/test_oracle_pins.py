@@ -641,3 +641,94 @@ def test_valid_row_map():
     lp_masked, _, _ = O.token_logprobs(H, W, tok, mk)
     lp_compact, _, _ = O.token_logprobs(H[idx], W, tok[idx])
     assert np.array_equal(lp_masked[idx], lp_compact)
+
+
+# ----------------------------------------------------------------------------- token-level KL reward shaping
+def _shaping_case():
+    ln = math.log
+    logp = np.array([ln(0.5), -7.0, ln(0.25), ln(0.5)])
+    ref = np.array([ln(0.25), 3.0, ln(0.25), ln(1.0)])
+    mask = np.array([1, 0, 1, 1], dtype=np.uint8)
+    return logp, ref, mask, np.array([0, 4]), np.array([2.0])
+
+
+def test_kl_shaping_hand_worked_example():
+    g = _golden("kl_shaping_worked_example.txt")
+    logp, ref, mask, off, R = _shaping_case()
+    r, ret = O.kl_shaped_returns(R, logp, ref, mask, off, beta=0.5, kind="k1")
+    assert abs(r[0] - g["k1_r0"]) < 1e-14 and abs(r[3] - g["k1_r3"]) < 1e-14 and r[1] == 0 and r[2] == 0
+    assert abs(ret[0] - g["k1_ret0"]) < 1e-14 and abs(ret[2] - g["k1_ret2"]) < 1e-14 and abs(ret[3] - g["k1_ret3"]) < 1e-14
+    assert ret[1] == 0
+    r, ret = O.kl_shaped_returns(R, logp, ref, mask, off, beta=0.5, kind="k3")
+    assert abs(r[0] - g["k3_r0"]) < 1e-14 and abs(r[3] - g["k3_r3"]) < 1e-14
+    assert abs(ret[0] - g["k3_ret0"]) < 1e-14 and abs(ret[2] - g["k3_ret2"]) < 1e-14 and abs(ret[3] - g["k3_ret3"]) < 1e-14
+    _, ret = O.kl_shaped_returns(R, logp, ref, mask, off, beta=0.5, gamma=0.5, kind="k3")
+    assert abs(ret[2] - g["k3_half_ret2"]) < 1e-14 and abs(ret[0] - g["k3_half_ret0"]) < 1e-14 and ret[1] == 0
+
+
+def test_kl_shaping_beta_zero_gives_every_valid_token_the_trajectory_value():
+    rng = _rng(70)
+    off = np.array([0, 5, 5, 12, 20])                # the second response is empty
+    T = 23                                           # rows 20..22 lie outside every response
+    mask = (rng.random(T) < 0.7).astype(np.uint8)
+    mask[5:12] = 0                                   # the third response has no valid token
+    R = rng.normal(size=4)
+    logp, ref = rng.normal(size=T), rng.normal(size=T)
+    r, ret = O.kl_shaped_returns(R, logp, ref, mask, off, beta=0.0)
+    for i in (0, 3):
+        for t in range(off[i], off[i + 1]):
+            assert ret[t] == (R[i] if mask[t] else 0.0)
+    assert np.all(ret[5:12] == 0) and np.all(ret[20:] == 0) and np.all(r[5:12] == 0)
+    # the reward itself sits on the last valid token only
+    for i in (0, 3):
+        valid = [t for t in range(off[i], off[i + 1]) if mask[t]]
+        assert r[valid[-1]] == R[i] and all(r[t] == 0 for t in valid[:-1])
+
+
+def test_kl_shaping_matches_library_cumsum_and_closed_form():
+    # no mask, gamma = 1: the return-to-go is a reversed cumulative sum (numpy's routine) ...
+    rng = _rng(71)
+    off = np.array([0, 7, 19])
+    logp, ref = rng.normal(size=19), rng.normal(size=19)
+    R = np.array([1.0, -0.5])
+    for kind in ("k1", "k3"):
+        r, ret = O.kl_shaped_returns(R, logp, ref, None, off, beta=0.3, kind=kind)
+        for i in range(2):
+            seg = r[off[i]:off[i + 1]]
+            assert np.allclose(ret[off[i]:off[i + 1]], np.cumsum(seg[::-1])[::-1], atol=1e-13)
+    # ... and with a constant log-ratio c the k1 return of position p of n is R - beta*c*(n - p)
+    c = 0.25
+    _, ret = O.kl_shaped_returns(R, logp, logp - c, None, off, beta=0.3, kind="k1")
+    for i in range(2):
+        n = off[i + 1] - off[i]
+        for p in range(n):
+            assert abs(ret[off[i] + p] - (R[i] - 0.3 * c * (n - p))) < 1e-13
+    # k3 is the estimator of the loss: non-negative, zero iff ref == logp, ~ delta^2 / 2
+    k3 = O.token_kl_estimate(logp, ref, "k3")
+    assert np.all(k3 >= 0) and np.all(O.token_kl_estimate(logp, logp, "k3") == 0)
+    assert abs(O.token_kl_estimate(np.zeros(1), np.array([1e-4]), "k3")[0] - 0.5e-8) < 1e-12
+    # a per-token divergence handed in is used as it is
+    kl = rng.random(19)
+    r, _ = O.kl_shaped_returns(np.zeros(2), logp, ref, None, off, beta=2.0, kind="given", kl_tok=kl)
+    assert np.allclose(r, -2.0 * kl, atol=0)
+
+
+def test_kl_shaping_discounted_bruteforce_with_mask():
+    # ret_t = sum over the valid tokens u >= t of the response of gamma^(valid tokens between) r_u
+    rng = _rng(72)
+    off = np.array([0, 9, 9, 30, 41])
+    T = 41
+    mask = (rng.random(T) < 0.6).astype(np.uint8)
+    logp, ref = rng.normal(size=T) * 0.3, rng.normal(size=T) * 0.3
+    R = rng.normal(size=4)
+    for gamma in (1.0, 0.9, 0.5):
+        r, ret = O.kl_shaped_returns(R, logp, ref, mask, off, beta=0.1, gamma=gamma, kind="k3")
+        for i in range(4):
+            valid = [t for t in range(off[i], off[i + 1]) if mask[t]]
+            for a, t in enumerate(valid):
+                brute = sum(gamma ** (b - a) * r[u] for b, u in enumerate(valid) if b >= a)
+                assert abs(ret[t] - brute) < 1e-12
+            # telescoping: consecutive valid tokens differ by exactly one shaped reward
+            for a in range(len(valid) - 1):
+                assert abs(ret[valid[a]] - gamma * ret[valid[a + 1]] - r[valid[a]]) < 1e-12
+        assert np.all(ret[mask == 0] == 0) and np.all(r[mask == 0] == 0)
