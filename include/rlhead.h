@@ -1,8 +1,8 @@
 /* rlhead.h - C ABI of the fused LM-head log-probability + GRPO policy-loss library (sm_100a).
  *
  * The library evaluates, for a batch of token positions, the quantities of the policy-update
- * step of Algorithm 1 ("compute estimating advantages" and "update the policy model by
- * maximizing the objective", Eq. 6): GRPO group-normalised advantages (section 4.2), the
+ * step of Algorithm 1 (its advantage-estimation step and its policy-update step, Eq. 6): GRPO
+ * group-normalised advantages (section 4.2), the
  * log-probability of every sampled token under the next-token policy over the vocabulary
  * (section 2.2), its entropy (section 2.2 "Regularization"), the clipped importance-ratio
  * surrogate (section 3.1) with a KL-to-reference regulariser, and the gradient of the resulting
@@ -123,8 +123,8 @@ rl_status rl_set_workspace(rl_ctx* ctx, void* dev_ptr, size_t bytes);
  * kernel-specific word describing where the first error was seen. */
 rl_status rl_last_device_status(rl_ctx* ctx, int32_t* detail);
 
-/* GRPO advantages - Algorithm 1 "compute estimating advantages"; section 3.2.2 advantage
- * estimation stage; section 4.2 "group-based normalization".
+/* GRPO advantages - the advantage-estimation step of Algorithm 1; section 3.2.2 advantage
+ * estimation stage; section 4.2 (normalisation of the rewards within each group of responses).
  * rewards[n_seq] holds one scalar per response (section 3.2.2 scoring stage), the group_size
  * responses of a prompt stored consecutively.  adv_seq[i] = (r_i - mean_g) / (std_g + eps_std);
  * a group whose rewards are all equal gets exactly 0.  The basic call uses the sample standard
@@ -139,8 +139,8 @@ rl_status rl_grpo_advantages_ex(rl_ctx* ctx, const float* rewards, int64_t n_seq
                                 int ddof, float eps_std, const int32_t* seq_offsets,
                                 int64_t T, float* adv_seq, float* adv_tok);
 
-/* The other critic-free advantage estimators that section 4.2 names ("RLOO's leave-one-out
- * baselines", "OPO's length-weighted baselines", REINFORCE++) on the same grouped layout.  The
+/* The other critic-free advantage estimators that section 4.2 names (the leave-one-out baseline
+ * of RLOO, the length-weighted baseline of OPO, REINFORCE++) on the same grouped layout.  The
  * paper prints no formula for them; the readings are
  *   RL_ADV_GRPO          as rl_grpo_advantages (sample std, eps_std as given)
  *   RL_ADV_RLOO          A_i = r_i - mean of the other responses of the group (group_size >= 2)
@@ -153,7 +153,30 @@ typedef enum { RL_ADV_GRPO = 0, RL_ADV_RLOO = 1, RL_ADV_OPO = 2, RL_ADV_REINFORC
 rl_status rl_advantages(rl_ctx* ctx, int estimator, const float* rewards, const int32_t* lengths,
                         int64_t n_seq, int group_size, float eps_std, float* adv_seq);
 
-/* Padding-free row map on its own (section 4.4 "padding-free training"): row_map[i] = index of
+/* Token-level KL reward shaping - section 2.2 "Regularization": the KL-to-reference regulariser
+ * applied as per-token rewards rather than (or beside) a loss term.  The paper prints no formula;
+ * the reading is: every valid row t of response i gets the shaped reward r_t = -beta * kl_t, the
+ * last valid row of the response additionally seq_value[i] (the trajectory reward of the scoring
+ * stage, section 3.2.2, or a group-normalised advantage from rl_grpo_advantages), and
+ * returns[t] = r_t + gamma * returns[next valid row of the same response] (gamma = 1: the reverse
+ * cumulative sum), to be used as the per-row adv[T] of the loss calls.  kl_t is chosen by
+ * kl_estimate: RL_KL_K1 the signed log-ratio logp[t] - ref_logp[t]; RL_KL_K3 exp(delta) - delta - 1
+ * with delta = ref_logp[t] - logp[t] (the estimator the loss uses); RL_KL_GIVEN kl_tok[t] as handed
+ * in (for instance rl_loss_opts.kl_out of a full-distribution pass).
+ * seq_value[n_seq], seq_offsets[n_seq+1] (ascending row ranges, seq_offsets[n_seq] <= T), logp,
+ * ref_logp, kl_tok, mask (NULL = all valid), returns[T] and shaped_reward[T] (may be NULL) are
+ * device pointers; the arrays a kl_estimate does not read may be NULL.  Rows with mask 0 and rows
+ * outside every range get 0, carry no reward and do not count as a discount step; a response
+ * without a valid row drops its seq_value.  Sums run in double precision, one warp per response,
+ * in a fixed order (reproducible).  Needs no workspace.
+ * Errors: beta < 0, gamma < 0, unknown kl_estimate, NULL required pointer -> RL_ERR_INVALID_ARG. */
+typedef enum { RL_KL_K1 = 0, RL_KL_K3 = 1, RL_KL_GIVEN = 2 } rl_kl_estimate;
+rl_status rl_kl_shaped_returns(rl_ctx* ctx, const float* seq_value, const float* logp, const float* ref_logp,
+                               const float* kl_tok, const uint8_t* mask, const int32_t* seq_offsets,
+                               int64_t n_seq, int64_t T, float beta, float gamma, int kl_estimate,
+                               float* shaped_reward, float* returns);
+
+/* Padding-free row map on its own (section 4.4, training without padding tokens): row_map[i] = index of
  * the i-th row with mask != 0, ascending, for i < *n_valid; entries past that are left untouched.
  * mask NULL = all rows valid.  row_map[T] (int32) and n_valid[1] (int32) are device pointers; the
  * workspace needs (T / 4096 + 3) * 4 bytes.  Every other call of this library runs the same
@@ -191,8 +214,8 @@ typedef struct {
   size_t struct_size;
   float ent_coef;             /* entropy bonus coefficient (section 2.2), >= 0                 */
   const float* token_weight;  /* [T] or NULL: replaces w_t = mask_t/sum(mask) by               */
-                              /* token_weight[t]*mask_t ("length normalization with token      */
-                              /* weights", section 2.2)                                        */
+                              /* token_weight[t]*mask_t (the length normalisation by token     */
+                              /* weights that section 2.2 lists among the regularisers)        */
   int accumulate_dW;          /* non-zero: dW += gradient instead of overwrite                 */
   float* logp_out;            /* [T] or NULL                                                   */
   float* entropy_out;         /* [T] or NULL                                                   */
@@ -202,14 +225,16 @@ typedef struct {
                               /* the call; 1 mean over responses of each response's token mean */
                               /* (w = mask/(n_seq*len_i)); 2 mean over responses of the token  */
                               /* sum over the longest row range (w = mask/(n_seq*L_max))       */
-  int sequence_level;         /* non-zero: sequence-level importance ratio ("GSPO's sequence-  */
-                              /* level aggregation", section 4.2; reading: rho_i = exp(mean    */
+  int sequence_level;         /* non-zero: sequence-level importance ratio (the GSPO variant   */
+                              /* named in section 4.2; reading: rho_i = exp(mean               */
                               /* token log-ratio over the valid tokens of response i), used    */
                               /* and clipped for every token of the response                   */
   int dH_dtype;               /* 0: dH is bf16 [T,d]; 1: dH is fp32 [T,d]                      */
   const int32_t* seq_offsets; /* [n_seq+1] ascending row range of every response, needed by    */
   int64_t n_seq;              /* agg_mode 1/2 and sequence_level; seq_offsets[n_seq] <= T;     */
                               /* valid rows outside every range then take no part in the loss  */
+                              /* (the token mean of agg_mode 0 is over the rows inside ranges; */
+                              /* metrics_out[6] still counts every valid row)                  */
   int kl_full;                /* non-zero: the regulariser is the full-distribution            */
                               /* KL(pi_theta(.|s_t) || pi_ref(.|s_t)) = sum_j p_j (log p_j -   */
                               /* log q_j) over the vocabulary, as sections 2.2 and 3.1 print   */
@@ -254,7 +279,7 @@ rl_status rl_policy_loss_fwd_bwd_host(rl_ctx* ctx, const void* H_host, int64_t l
                                       float* loss_host, float* metrics_host, void* dH, float* dW);
 
 /* Scoring with several models in one call - Algorithm 1 evaluates the same sampled tokens under
- * the old policy pi_theta_old ("update the old policy model", importance-ratio denominator of
+ * the old policy pi_theta_old (its old-policy refresh step; importance-ratio denominator of
  * section 2.2) and under the frozen reference pi_ref (section 3.2.1, Reference role) before the
  * update.  Model i has hidden states H[i] ([T, d[i]] bf16, row stride ldH[i]) and LM head W[i]
  * ([V, d[i]] bf16, row stride ldW[i]); tokens, mask, T and V are shared.  The arrays H, ldH, W,
@@ -268,9 +293,9 @@ rl_status rl_token_logprobs_multi(rl_ctx* ctx, int n_models, const void* const* 
                                   float* const* logp, float* const* entropy);
 
 /* Vocabulary-parallel LM head - for training engines that shard the model states so that the
- * head weight is never resident on one GPU in full (section 4.3 "finer-grained control over
- * sharding behavior", section 4.4 "model states do not need to be fully resident on a single
- * GPU").  The rows of W are partitioned over ranks; this rank holds W_shard[V_shard, d] =
+ * head weight is never resident on one GPU in full (the sharded training engines of section 4.3
+ * and the memory discussion of section 4.4).  The rows of W are partitioned over ranks; this rank
+ * holds W_shard[V_shard, d] =
  * rows [vocab_offset, vocab_offset + V_shard) of the V_total-row head.  tokens are ids in
  * [0, V_total) (checked against V_total; an id outside this rank's slice simply has no logit
  * here).  The three calls compute exactly what rl_token_logprobs and rl_policy_loss_fwd_bwd_ex
@@ -333,10 +358,10 @@ rl_status rl_policy_loss_fwd_bwd_host_wait(rl_ctx* ctx, int slot, float* loss_ho
 
 /* rl_token_logprobs without any device allocation and without a context (the paper has no
  * counterpart).  It is meant for callers that cannot allocate GPU memory when they need
- * log-probabilities: a scoring pass that shares the GPU with a rollout engine which has already
- * reserved almost all of its memory (the co-located setup of section 4.4 leaves no room for
- * cudaMalloc to succeed), or code that must not pay the device-wide synchronisation cudaMalloc /
- * cudaFree imply.  Inputs and outputs are the caller's device buffers exactly as in
+ * log-probabilities: a scoring pass that shares the GPU with another engine which has already
+ * reserved almost all of its memory, so that a cudaMalloc of the workspace would fail, or code
+ * that must not pay the device-wide synchronisation cudaMalloc / cudaFree imply.  Inputs and
+ * outputs are the caller's device buffers exactly as in
  * rl_token_logprobs; everything in between (compacted rows, row map, per-range softmax
  * statistics, the status word) lives in a fixed 16 MiB device array that is part of the library
  * image, so every GPU on which the library is loaded holds those 16 MiB until the process exits.
@@ -354,7 +379,8 @@ rl_status rl_policy_loss_fwd_bwd_host_wait(rl_ctx* ctx, int slot, float* loss_ho
  *   work overlaps (different streams, or different host threads on different streams) race on the
  *   array: serialise them on one stream or with events.  Host-side the call is thread-safe.
  *   dev_status (device, int32[2], may be NULL) receives {status, detail} as rl_last_device_status
- *   would report them (RL_ERR_TOKEN_RANGE / RL_ERR_TIMEOUT), written in stream order. */
+ *   would report them (RL_ERR_TOKEN_RANGE / RL_ERR_TIMEOUT), written in stream order ({0, 0} when
+ *   T = 0). */
 rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH, const void* W,
                                    int64_t ldW, const int32_t* tokens, const uint8_t* mask,
                                    int64_t T, int64_t d, int64_t V,

@@ -13,7 +13,7 @@ token y_t; z_t = W h_t the logits; pi_theta(.|s_t) = softmax(z_t).
 
 Readings of the paper that this oracle fixes (the paper prints no formula or
 leaves a choice open for each of them):
-  * GRPO "group-based normalization" (section 4.2): A_i = (r_i - mean_g) /
+  * GRPO normalisation within a group of responses (section 4.2): A_i = (r_i - mean_g) /
     (std_g + eps_std) with the sample standard deviation (ddof=1) by default.
   * PPO clipped surrogate (section 3.1): the standard pessimistic form
     min(r*A, clip(r, 1-eps_low, 1+eps_high)*A).  The form as literally printed,
@@ -42,8 +42,8 @@ import numpy as np
 
 
 # --------------------------------------------------------------------------- #
-# Algorithm 1, "compute estimating advantages" step; section 3.2.2 advantage
-# estimation stage; section 4.2 "GRPO's group-based normalization".
+# Algorithm 1, advantage-estimation step; section 3.2.2 advantage estimation
+# stage; section 4.2 (GRPO: rewards normalised within each group).
 # --------------------------------------------------------------------------- #
 def grpo_advantages(rewards, group_size, ddof=1, eps_std=1e-6):
     """Per-response GRPO advantages.
@@ -72,8 +72,8 @@ def grpo_advantages(rewards, group_size, ddof=1, eps_std=1e-6):
 
 # --------------------------------------------------------------------------- #
 # Other critic-free estimators the paper names in section 4.2 without printing a
-# formula ("RLOO's leave-one-out baselines", "OPO's length-weighted baselines",
-# REINFORCE++).  Readings, stated here because the paper is silent:
+# formula (the leave-one-out baseline of RLOO, the length-weighted baseline of
+# OPO, REINFORCE++).  Readings, stated here because the paper is silent:
 #   RLOO          A_i = r_i - mean of the OTHER responses of the group
 #   OPO           A_i = r_i - sum_j(len_j r_j) / sum_j(len_j) over the group
 #   REINFORCE++   A_i = (c_i - mean(c)) / (std(c) + eps_std) over the whole batch,
@@ -129,9 +129,9 @@ def broadcast_to_tokens(adv_seq, seq_offsets, T):
 
 
 # --------------------------------------------------------------------------- #
-# Section 2.2 "Regularization": the KL-to-reference term is "often applied with
-# token-level shaping", i.e. folded into per-token rewards instead of (or beside)
-# the loss.  The paper prints no formula for the shaped reward; reading:
+# Section 2.2 "Regularization" mentions that the KL-to-reference term is commonly
+# applied as token-level shaping, i.e. folded into per-token rewards instead of (or
+# beside) the loss.  The paper prints no formula for the shaped reward; reading:
 #   kl_t  = per-token divergence estimate of a valid token t, one of
 #             "k1"  logp_t - ref_logp_t              (signed sampled log-ratio)
 #             "k3"  exp(delta) - delta - 1, delta = ref_logp_t - logp_t
@@ -186,7 +186,7 @@ def kl_shaped_returns(seq_value, logp, ref_logp, mask, seq_offsets, beta, gamma=
 
 
 # --------------------------------------------------------------------------- #
-# Section 4.4 "padding-free training": only rows whose mask is non-zero are
+# Section 4.4 (training without padding tokens): only rows whose mask is non-zero are
 # worked on; the row map lists them in ascending order.
 # --------------------------------------------------------------------------- #
 def valid_row_map(mask, T=None):
@@ -224,7 +224,7 @@ def log_softmax_stats(Z):
 def token_logprobs(H, W, tokens, mask=None):
     """log pi_theta(y_t | s_t), entropy and lse per row; masked rows give 0.
 
-    Section 2.2 "Adaptation for Off-Policy": the log-probability of the sampled
+    Section 2.2 (off-policy adaptation): the log-probability of the sampled
     token is what enters the importance ratio.
     """
     T = H.shape[0]
@@ -255,7 +255,7 @@ def token_weights(mask):
 
 
 def aggregation_weights(mask, seq_offsets, mode):
-    """Token weights w_t of the loss ("length normalization with token weights", section 2.2).
+    """Token weights w_t of the loss (length normalisation by token weights, section 2.2).
 
     mode 0: token mean over the call, w_t = m_t / sum(m).
     mode 1: mean over sequences of each sequence's token mean, w_t = m_t / (B * len_i).
@@ -285,7 +285,7 @@ def aggregation_weights(mask, seq_offsets, mode):
 
 
 def sequence_ratio(logp, old_logp, mask, seq_offsets):
-    """Sequence-level importance ratio ("GSPO's sequence-level aggregation", section 4.2; the
+    """Sequence-level importance ratio (the GSPO variant named in section 4.2; the
     paper prints no formula - reading): rho_i = exp(mean over the valid tokens of sequence i of
     (logp_t - old_logp_t)), i.e. the geometric mean of the token ratios; every token of the
     sequence uses rho_i.  Returns (rho per row, len per row); rows outside any sequence get 1, 0."""
@@ -355,6 +355,13 @@ def policy_loss_fwd_bwd(H, W, tokens, old_logp, ref_logp, adv, mask,
     T, d = H.shape
     V = W.shape[0]
     m = np.asarray(mask).astype(bool)
+    if seq_offsets is not None and (sequence_level or agg_mode != 0):
+        # response-aware paths: a valid row that lies outside every response range takes no part
+        # in the loss (it has no response to be aggregated with), exactly as if it were masked
+        off_ = np.asarray(seq_offsets)
+        inside = np.zeros(T, dtype=bool)
+        inside[int(off_[0]):int(off_[-1])] = True
+        m = m & inside
     if token_weight is not None:
         w = np.asarray(token_weight, dtype=np.float64) * m
     else:

@@ -117,6 +117,8 @@ def load_library():
     lib.rl_debug_schedule.restype = c_int
     lib.rl_mask_scan.argtypes = [P, P, c_int64, P, P]
     lib.rl_mask_scan.restype = c_int
+    lib.rl_kl_shaped_returns.argtypes = [P, P, P, P, P, P, P, c_int64, c_int64, c_float, c_float, c_int, P, P]
+    lib.rl_kl_shaped_returns.restype = c_int
     lib.rl_token_logprobs_multi.argtypes = [P, c_int, POINTER(c_void_p), POINTER(c_int64), POINTER(c_void_p),
                                             POINTER(c_int64), POINTER(c_int64), P, P, c_int64, c_int64,
                                             POINTER(c_void_p), POINTER(c_void_p)]
@@ -326,6 +328,25 @@ class Context:
                 opts.kl_out = out["kl"].data_ptr()
         _check(self.lib.rl_policy_loss_fwd_bwd_ex(*args, byref(opts)), "rl_policy_loss_fwd_bwd_ex")
         return out
+
+    KL_ESTIMATES = {"k1": 0, "k3": 1, "given": 2}
+
+    def rl_kl_shaped_returns(self, seq_value, logp, ref_logp, mask, seq_offsets, T, beta, gamma=1.0, kind="k3",
+                             kl_tok=None, want_shaped=True, returns=None):
+        """Token-level KL reward shaping: returns (shaped_reward [T] or None, returns [T])."""
+        self._bind_stream()
+        assert seq_value.dtype == torch.float32 and seq_offsets.dtype == torch.int32
+        for x in (logp, ref_logp, kl_tok):
+            assert x is None or (x.dtype == torch.float32 and x.is_contiguous() and x.numel() == T)
+        dev = seq_value.device
+        if returns is None:
+            returns = torch.empty(T, dtype=torch.float32, device=dev)
+        shaped = torch.empty(T, dtype=torch.float32, device=dev) if want_shaped else None
+        _check(self.lib.rl_kl_shaped_returns(self.handle, _ptr(seq_value), _ptr(logp), _ptr(ref_logp), _ptr(kl_tok),
+                                             _ptr(mask), _ptr(seq_offsets), seq_offsets.numel() - 1, T, beta, gamma,
+                                             self.KL_ESTIMATES[kind], _ptr(shaped), _ptr(returns)),
+               "rl_kl_shaped_returns")
+        return shaped, returns
 
     def rl_mask_scan(self, mask, T=None, row_map=None, n_valid=None):
         """Row map of the valid rows: returns (row_map [T] int32, n_valid [1] int32), both on the device."""
@@ -558,8 +579,11 @@ def rl_token_logprobs_static(H, W, tokens, mask, logp, entropy=None, lse=None, d
     V = W.shape[0]
     assert H.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and tokens.dtype == torch.int32
     assert logp.dtype == torch.float32 and logp.numel() == T
-    stream = c_void_p(torch.cuda.current_stream(H.device).cuda_stream)
-    _check(lib.rl_token_logprobs_static(stream, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0), _ptr(tokens),
-                                        _ptr(mask), T, d, V, _ptr(logp), _ptr(entropy), _ptr(lse), _ptr(dev_status)),
-           "rl_token_logprobs_static")
+    # the library works on the CURRENT device: make it the one the operands live on
+    with torch.cuda.device(H.device):
+        stream = c_void_p(torch.cuda.current_stream(H.device).cuda_stream)
+        _check(lib.rl_token_logprobs_static(stream, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0),
+                                            _ptr(tokens), _ptr(mask), T, d, V, _ptr(logp), _ptr(entropy), _ptr(lse),
+                                            _ptr(dev_status)),
+               "rl_token_logprobs_static")
     return logp

@@ -743,6 +743,35 @@ rl_status rl_grpo_advantages(rl_ctx* c, const float* rewards, int64_t n_seq, int
   return rl_grpo_advantages_ex(c, rewards, n_seq, group_size, 1, 1e-6f, nullptr, 0, adv_seq, nullptr);
 }
 
+rl_status rl_kl_shaped_returns(rl_ctx* c, const float* seq_value, const float* logp, const float* ref_logp,
+                               const float* kl_tok, const uint8_t* mask, const int32_t* seq_offsets, int64_t n_seq,
+                               int64_t T, float beta, float gamma, int kl_estimate, float* shaped_reward,
+                               float* returns) {
+  if (!c || n_seq < 0 || T < 0 || n_seq >= (int64_t(1) << 31) || T >= (int64_t(1) << 31)) return RL_ERR_INVALID_ARG;
+  if (kl_estimate < RL_KL_K1 || kl_estimate > RL_KL_GIVEN || !(beta >= 0.f) || !(gamma >= 0.f)) return RL_ERR_INVALID_ARG;
+  if (T == 0) return RL_OK;
+  if (!returns) return RL_ERR_INVALID_ARG;
+  if (n_seq == 0) {
+    cudaMemsetAsync(returns, 0, (size_t)T * 4, c->stream);
+    if (shaped_reward) cudaMemsetAsync(shaped_reward, 0, (size_t)T * 4, c->stream);
+    return cuda_ok();
+  }
+  if (!seq_value || !seq_offsets) return RL_ERR_INVALID_ARG;
+  if (kl_estimate == RL_KL_GIVEN ? !kl_tok : (!logp || !ref_logp)) return RL_ERR_INVALID_ARG;
+  const int warps = 8;
+  long long blocks = (n_seq + warps - 1) / warps;
+  if (blocks > (long long)c->n_sm * 64) blocks = (long long)c->n_sm * 64;
+  const int pr = prof_begin(c, 8);
+  zero_outside_ranges_kernel<<<c->n_sm, 256, 0, c->stream>>>(seq_offsets, (int)n_seq, (long long)T, returns,
+                                                             shaped_reward);
+  kl_shaped_returns_kernel<<<(int)blocks, warps * 32, 0, c->stream>>>(seq_value, logp, ref_logp, kl_tok, mask,
+                                                                      seq_offsets, (int)n_seq, beta, gamma, kl_estimate,
+                                                                      shaped_reward, returns);
+  prof_end(c, pr, 8);
+  c->launches += 2;
+  return cuda_ok();
+}
+
 rl_status rl_mask_scan(rl_ctx* c, const uint8_t* mask, int64_t T, int32_t* row_map, int32_t* n_valid) {
   if (!c || T < 0 || T >= (int64_t(1) << 31) || !n_valid || (T > 0 && !row_map)) return RL_ERR_INVALID_ARG;
   if (T == 0) return cudaMemsetAsync(n_valid, 0, 4, c->stream) == cudaSuccess ? RL_OK : RL_ERR_CUDA;
@@ -1236,6 +1265,16 @@ static rl_status host_step_check(const rl_ctx* c, const HostStepArgs& a) {
   if (a.T > 0 && !a.adv_host && (!a.rewards_host || !a.seq_offsets_host || a.n_seq <= 0 || a.n_seq > a.T))
     return RL_ERR_INVALID_ARG;
   if (a.ldH != a.d) return RL_ERR_SHAPE;  // host rows are copied as one block
+  // everything the advantage and loss calls would refuse is refused here, before a copy is enqueued
+  if (a.d % 64 != 0 || a.ldW < a.d || a.T >= (int64_t(1) << 30) || a.V >= (int64_t(1) << 30)) return RL_ERR_SHAPE;
+  if (a.ldW % 8 != 0 || (reinterpret_cast<uintptr_t>(a.W) & 15) || (reinterpret_cast<uintptr_t>(a.dH) & 15) ||
+      (reinterpret_cast<uintptr_t>(a.dW) & 15))
+    return RL_ERR_ALIGNMENT;
+  if (!a.W || !a.dW || (a.T > 0 && !a.dH)) return RL_ERR_INVALID_ARG;
+  if (!(a.eps_low >= 0.f && a.eps_low < 1.f) || !(a.eps_high >= 0.f) || !(a.beta >= 0.f) || !(a.ent_coef >= 0.f))
+    return RL_ERR_INVALID_ARG;
+  if (a.beta != 0.f && a.T > 0 && !a.ref_host) return RL_ERR_INVALID_ARG;
+  if (a.T > 0 && !a.adv_host && (a.group_size < 2 || a.n_seq % a.group_size != 0)) return RL_ERR_SHAPE;
   return RL_OK;
 }
 
@@ -1322,13 +1361,24 @@ rl_status rl_policy_loss_fwd_bwd_host_submit(rl_ctx* c, int slot, const void* H_
   const WsLayout L = ws_layout(c, T, d, V, 2);
   if ((s = check_ws(c, L)) != RL_OK) return s;
   if (!c->copy_stream) {
-    // first pipelined call on this context: the copy stream, two events and 64 pinned bytes per slot
-    bool ok = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    // first pipelined call on this context: the copy stream, two events and 64 pinned bytes per slot;
+    // all of it or none of it, so that a later call never finds a half-made set
+    cudaStream_t cs = nullptr;
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    float* pin[2] = {nullptr, nullptr};
+    bool ok = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < 2 && ok; ++i)
-      ok = cudaEventCreateWithFlags(&c->copy_done[i], cudaEventDisableTiming) == cudaSuccess &&
-           cudaEventCreateWithFlags(&c->step_done[i], cudaEventDisableTiming) == cudaSuccess &&
-           cudaHostAlloc(reinterpret_cast<void**>(&c->pinned_out[i]), 64, cudaHostAllocDefault) == cudaSuccess;
-    if (!ok) return RL_ERR_CUDA;
+      ok = cudaHostAlloc(reinterpret_cast<void**>(&pin[i]), 64, cudaHostAllocDefault) == cudaSuccess;
+    if (!ok) {
+      for (int i = 0; i < 2; ++i) if (pin[i]) cudaFreeHost(pin[i]);
+      for (int i = 0; i < 4; ++i) if (ev[i]) cudaEventDestroy(ev[i]);
+      if (cs) cudaStreamDestroy(cs);
+      cudaGetLastError();
+      return RL_ERR_CUDA;
+    }
+    for (int i = 0; i < 2; ++i) { c->copy_done[i] = ev[2 * i]; c->step_done[i] = ev[2 * i + 1]; c->pinned_out[i] = pin[i]; }
+    c->copy_stream = cs;
   }
   HostStage hs;
   const size_t stage = carve_stage(nullptr, T, d, nullptr);
@@ -1493,7 +1543,11 @@ rl_status rl_token_logprobs_static(void* cuda_stream, const void* H, int64_t ldH
   }
   rl_ctx* c = &slot.ctx;
   c->stream = static_cast<cudaStream_t>(cuda_stream);
-  if (T == 0) return RL_OK;
+  if (T == 0) {
+    // nothing to compute, but the caller's status words must not keep stale contents
+    if (dev_status && cudaMemsetAsync(dev_status, 0, 2 * sizeof(int32_t), c->stream) != cudaSuccess) return RL_ERR_CUDA;
+    return RL_OK;
+  }
   // only the forward part of the workspace layout is needed: everything before the gradient slab
   const WsLayout L = ws_layout(c, T, d, V, false);
   if (L.G > c->ws_bytes) return RL_ERR_WORKSPACE;

@@ -351,6 +351,94 @@ __global__ void __launch_bounds__(256) broadcast_adv_kernel(const float* __restr
 }
 
 // ------------------------------------------------------------------------------------------
+// Token-level KL reward shaping (section 2.2 "Regularization": the KL-to-reference term applied as
+// per-token rewards; the paper prints no formula, reading): every valid token t of a response gets
+// the shaped reward r_t = -beta kl_t, its last valid token additionally the response's scalar
+// seq_value, and the per-token value is the return-to-go ret_t = r_t + gamma ret_(next valid token).
+// kl_t is the signed log-ratio logp - ref (kind 0), exp(delta) - delta - 1 with delta = ref - logp
+// (kind 1), or a value handed in (kind 2).  Masked rows get 0 and are not a discount step.
+// One warp per response: it walks the response's rows from the end in 32-row chunks aligned to
+// 128 bytes, loads kShapeChunks chunks at a time and runs a suffix scan of the linear maps
+// x -> v + g x (valid row: g = gamma, v = r_t; masked row: the identity) with shuffles, carrying the
+// return of the first valid token of the chunks already done.  Arithmetic in double.
+constexpr int kShapeChunks = 4;
+
+__global__ void __launch_bounds__(256) kl_shaped_returns_kernel(const float* __restrict__ seq_value,
+                                                                const float* __restrict__ logp,
+                                                                const float* __restrict__ ref_logp,
+                                                                const float* __restrict__ kl_tok,
+                                                                const uint8_t* __restrict__ mask,
+                                                                const int* __restrict__ seq_offsets, int n_seq,
+                                                                float beta, float gamma, int kind,
+                                                                float* __restrict__ shaped, float* __restrict__ ret) {
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int sq = blockIdx.x * warps_per_block + (threadIdx.x >> 5); sq < n_seq; sq += gridDim.x * warps_per_block) {
+    const int lo = seq_offsets[sq], hi = seq_offsets[sq + 1];
+    if (hi <= lo) continue;
+    const double R = (double)seq_value[sq];
+    double carry = 0.0;            // return-to-go of the first valid token after the chunks done so far
+    bool terminal_done = false;    // the last valid token of the response has been found
+    const int c_first = lo >> 5;
+    for (int c_hi = (hi - 1) >> 5; c_hi >= c_first; c_hi -= kShapeChunks) {
+      double r[kShapeChunks];
+      bool inside[kShapeChunks], valid[kShapeChunks];
+#pragma unroll
+      for (int j = 0; j < kShapeChunks; ++j) {
+        const int t = (c_hi - j) * 32 + lane;
+        inside[j] = (c_hi - j) >= c_first && t >= lo && t < hi;
+        valid[j] = inside[j] && (!mask || mask[t] != 0);
+        double kl = 0.0;
+        if (valid[j]) {
+          if (kind == 2) {
+            kl = (double)kl_tok[t];
+          } else {
+            const double lp = (double)logp[t], rf = (double)ref_logp[t];
+            kl = kind == 0 ? lp - rf : exp(rf - lp) - (rf - lp) - 1.0;
+          }
+        }
+        r[j] = -(double)beta * kl;
+      }
+#pragma unroll
+      for (int j = 0; j < kShapeChunks; ++j) {
+        const unsigned live = __ballot_sync(0xffffffffu, valid[j]);
+        if (!terminal_done && live) {
+          if (lane == 31 - __clz(live)) r[j] += R;
+          terminal_done = true;
+        }
+        double g = valid[j] ? (double)gamma : 1.0, v = valid[j] ? r[j] : 0.0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const double g2 = __shfl_down_sync(0xffffffffu, g, o);
+          const double v2 = __shfl_down_sync(0xffffffffu, v, o);
+          if (lane + o < 32) { v = fma(g, v2, v); g *= g2; }
+        }
+        const double out = fma(g, carry, v);
+        carry = __shfl_sync(0xffffffffu, out, 0);
+        if (inside[j]) {
+          const int t = (c_hi - j) * 32 + lane;
+          ret[t] = valid[j] ? (float)out : 0.f;
+          if (shaped) shaped[t] = valid[j] ? (float)r[j] : 0.f;
+        }
+      }
+    }
+  }
+}
+
+// Rows that lie outside every response range, [0, seq_offsets[0]) and [seq_offsets[n_seq], T), get 0.
+__global__ void __launch_bounds__(256) zero_outside_ranges_kernel(const int* __restrict__ seq_offsets, int n_seq,
+                                                                  long long T, float* __restrict__ a,
+                                                                  float* __restrict__ b) {
+  const long long first = seq_offsets[0], last = seq_offsets[n_seq];
+  const long long n_out = first + (T > last ? T - last : 0);
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_out; i += (long long)gridDim.x * blockDim.x) {
+    const long long t = i < first ? i : last + (i - first);
+    a[t] = 0.f;
+    if (b) b[t] = 0.f;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Merge of the per-range statistics and the per-token loss arithmetic (Eq. 6 with the clipped
 // surrogate of section 3.1 and the k3 KL-to-reference term).
 struct LossParams {
@@ -508,8 +596,8 @@ __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossPa
 
 // ------------------------------------------------------------------------------------------
 // Sequence-aware loss path: aggregation weights that depend on each response's valid length
-// (section 2.2 "length normalization with token weights") and the sequence-level importance
-// ratio (section 4.2 "GSPO's sequence-level aggregation"; reading: rho_i = exp of the mean
+// (the length normalisation by token weights of section 2.2) and the sequence-level importance
+// ratio (the GSPO variant named in section 4.2; reading: rho_i = exp of the mean
 // token log-ratio over the valid tokens of response i, used by every token of the response).
 // One warp per response; its valid tokens are the compact rows [lo, hi) found by binary search
 // in the ascending row map.
@@ -562,13 +650,17 @@ __global__ void __launch_bounds__(kLossThreads) seq_loss_kernel(const SeqParams 
   double acc[kLossSums];
 #pragma unroll
   for (int k = 0; k < kLossSums; ++k) acc[k] = 0.0;
+  // token mean (agg_mode 0): over the valid rows that lie inside a response range, the ones that take part
+  const int n_part = p.agg_mode == 0 ? lower_bound_rows(p.row_map, n, p.seq_offsets[p.n_seq]) -
+                                           lower_bound_rows(p.row_map, n, p.seq_offsets[0])
+                                     : 0;
   for (int sq = blockIdx.x * warps_per_block + warp; sq < p.n_seq; sq += gridDim.x * warps_per_block) {
     const int lo = lower_bound_rows(p.row_map, n, p.seq_offsets[sq]);
     const int hi = lower_bound_rows(p.row_map, n, p.seq_offsets[sq + 1]);
     const int len = hi - lo;
     if (len <= 0) continue;
     float w_seq = 0.f;
-    if (p.agg_mode == 0) w_seq = 1.f / (float)n;
+    if (p.agg_mode == 0) w_seq = 1.f / (float)n_part;
     else if (p.agg_mode == 1) w_seq = 1.f / ((float)p.n_seq * (float)len);
     else w_seq = 1.f / ((float)p.n_seq * (float)max(*p.l_max, 1));
     float rho_seq = 1.f, seq_sum = 0.f;

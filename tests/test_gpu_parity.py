@@ -39,6 +39,31 @@ def _rel(a, b):
     return np.linalg.norm(a - b) / nb if nb > 0 else np.linalg.norm(a)
 
 
+def _assert_blockwise(got, want, block_rows, what):
+    """Localised gradient check on top of the global Frobenius norm: every block of block_rows
+    consecutive rows has to agree within 1e-2 of its own norm plus 1e-2 of an average block's norm
+    (||tensor|| / sqrt(blocks)), so that one wrong row or tile cannot hide inside the global norm."""
+    n = want.shape[0]
+    n_blocks = (n + block_rows - 1) // block_rows
+    pad = n_blocks * block_rows - n
+    sq = lambda a: np.pad((a * a).sum(axis=1), (0, pad)).reshape(n_blocks, block_rows).sum(axis=1)  # noqa: E731
+    err, ref = np.sqrt(sq(got - want)), np.sqrt(sq(want))
+    bound = TOL_GRAD_REL * ref + TOL_GRAD_REL * np.linalg.norm(want) / np.sqrt(n_blocks)
+    worst = int(np.argmax(err - bound))
+    assert np.all(err <= bound), f"{what}: block {worst} (rows {worst * block_rows}..) off by {err[worst]:.3e} > {bound[worst]:.3e}"
+
+
+def _poison(ctx, w, d_ref=0, dH_fp32=False):
+    """Workspace and outputs filled with NaN bit patterns before a call: whatever a kernel forgets to
+    write, or reads before writing, then shows up as NaN in the results."""
+    ctx.ensure_workspace(w.T, w.d, w.V, d_ref=d_ref)
+    ctx._ws.fill_(0xFF)
+    dev = w.W.device
+    return dict(dH=torch.full((w.T, w.d), float("nan"), dtype=torch.float32 if dH_fp32 else torch.bfloat16, device=dev),
+                dW=torch.full((w.V, w.d), float("nan"), dtype=torch.float32, device=dev),
+                loss=torch.full((1,), float("nan"), dtype=torch.float32, device=dev))
+
+
 def _oracle_case(w, adv_tok_np, **kw):
     return O.policy_loss_fwd_bwd(
         _np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), _np64(w.old_logp),
@@ -59,9 +84,11 @@ def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5, agg_m
                                      w.eps_low, w.eps_high, w.beta, ent_coef=w.ent_coef,
                                      token_weight=token_weight, agg_mode=agg_mode, sequence_level=sequence_level,
                                      seq_offsets=w.seq_offsets if (agg_mode or sequence_level) else None,
-                                     dH_fp32=dH_fp32)
+                                     dH_fp32=dH_fp32, **_poison(ctx, w, dH_fp32=dH_fp32))
     _assert_status_ok(ctx)
     assert out["dH"].dtype == (torch.float32 if dH_fp32 else torch.bfloat16)
+    for k in ("loss", "dH", "dW", "logp", "entropy", "metrics"):
+        assert not torch.isnan(out[k]).any(), f"{k} holds NaN: something was left unwritten or read before written"
     # the oracle works from its own advantages; nothing it sees comes from the CUDA path
     oo = _oracle_case(w, o_adv_tok, token_weight=None if token_weight is None else _np64(token_weight),
                       seq_offsets=w.seq_offsets.cpu().numpy(), agg_mode=agg_mode, sequence_level=sequence_level)
@@ -81,6 +108,8 @@ def _check_against_oracle(ctx, w, token_weight=None, boundary_margin=1e-5, agg_m
     assert not dH[~m].any()
     assert _rel(dH, oo["dH"]) <= TOL_GRAD_REL
     assert _rel(_np64(out["dW"]), oo["dW"]) <= TOL_GRAD_REL
+    _assert_blockwise(dH[m], oo["dH"][m], 1, "dH row")
+    _assert_blockwise(_np64(out["dW"]), oo["dW"], 128, "dW 128-row block")
     met = _np64(out["metrics"])
     assert abs(met[0] - oo["pg_loss"]) <= 1e-3 * abs(oo["pg_loss"]) + 1e-7
     assert abs(met[1] - oo["kl_mean"]) <= 1e-3 * abs(oo["kl_mean"]) + 1e-7
@@ -301,6 +330,30 @@ def test_aggregation_modes_and_sequence_level_ratio(ctx, agg_mode, sequence_leve
     w = make_workload(3, prompts=2, L_max=64, seed=810 + agg_mode, d=256, V=5000, sigma_old=0.3)
     shift_behaviour_policy(w)
     _check_against_oracle(ctx, w, agg_mode=agg_mode, sequence_level=sequence_level)
+
+
+@pytest.mark.parametrize("agg_mode,sequence_level", [(0, True), (1, False), (2, True)])
+def test_valid_rows_outside_every_response_range(ctx, agg_mode, sequence_level):
+    # the response ranges cover only part of the rows: valid rows before the first and after the last
+    # range take no part in the loss (outputs of the forward still cover them), and the token mean of
+    # agg_mode 0 is over the rows inside ranges
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(1, prompts=1, L_max=40, d=256, V=3000, seed=520 + agg_mode)
+    off = w.seq_offsets.clone()
+    inner = off[2:7].contiguous()                      # responses 2..5 only
+    adv = torch.randn(w.T, device="cuda")
+    out = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv, w.mask, w.eps_low, w.eps_high,
+                                     w.beta, ent_coef=0.01, agg_mode=agg_mode, sequence_level=sequence_level,
+                                     seq_offsets=inner)
+    _assert_status_ok(ctx)
+    oo = O.policy_loss_fwd_bwd(_np64(w.H), _np64(w.W), w.tokens.cpu().numpy(), _np64(w.old_logp), _np64(w.ref_logp),
+                               _np64(adv), w.mask.cpu().numpy(), w.eps_low, w.eps_high, w.beta, ent_coef=0.01,
+                               seq_offsets=inner.cpu().numpy(), agg_mode=agg_mode, sequence_level=sequence_level)
+    assert abs(out["loss"].item() - oo["loss"]) <= TOL_LOSS_REL * abs(oo["loss"]) + 1e-7
+    dH = _np64(out["dH"])
+    lo, hi = int(inner[0]), int(inner[-1])
+    assert not dH[:lo].any() and not dH[hi:].any()
+    assert _rel(dH, oo["dH"]) <= TOL_GRAD_REL and _rel(_np64(out["dW"]), oo["dW"]) <= TOL_GRAD_REL
 
 
 @pytest.mark.parametrize("cta_group", [2, 1])

@@ -732,3 +732,33 @@ def test_kl_shaping_discounted_bruteforce_with_mask():
             for a in range(len(valid) - 1):
                 assert abs(ret[valid[a]] - gamma * ret[valid[a + 1]] - r[valid[a]]) < 1e-12
         assert np.all(ret[mask == 0] == 0) and np.all(r[mask == 0] == 0)
+
+
+def test_valid_rows_outside_every_response_range_take_no_part():
+    # response-aware paths (sequence-level ratio, per-response aggregation): a valid row that belongs to
+    # no response is as good as masked - same loss, same gradients, and the token mean is over the rest
+    rng = _rng(80)
+    T, d, V = 14, 6, 11
+    H, W = rng.normal(size=(T, d)), rng.normal(size=(V, d)) * 0.5
+    tok = rng.integers(0, V, size=T)
+    old, ref, adv = rng.normal(size=T) * 0.1 - 2.0, rng.normal(size=T) * 0.1 - 2.0, rng.normal(size=T)
+    off = np.array([2, 6, 11])                        # rows 0, 1 and 11..13 belong to no response
+    mask = np.ones(T, dtype=np.uint8)
+    mask[4] = 0
+    masked_out = mask.copy()
+    masked_out[:2] = 0
+    masked_out[11:] = 0
+    for kw in (dict(sequence_level=True), dict(agg_mode=1), dict(agg_mode=2), dict(sequence_level=True, agg_mode=1)):
+        a = O.policy_loss_fwd_bwd(H, W, tok, old, ref, adv, mask, 0.2, 0.3, 0.05, ent_coef=0.01, seq_offsets=off, **kw)
+        b = O.policy_loss_fwd_bwd(H, W, tok, old, ref, adv, masked_out, 0.2, 0.3, 0.05, ent_coef=0.01, seq_offsets=off, **kw)
+        assert abs(a["loss"] - b["loss"]) < 1e-14 and np.allclose(a["dW"], b["dW"], atol=1e-14)
+        assert not a["dH"][:2].any() and not a["dH"][11:].any()
+    # token mean with the sequence-level ratio: weights are 1 / (valid rows inside ranges) = 1/8
+    a = O.policy_loss_fwd_bwd(H, W, tok, old, None, adv, mask, 0.2, 0.3, 0.0, seq_offsets=off, sequence_level=True)
+    lp = a["logp"]
+    rho, _ = O.sequence_ratio(lp, old, masked_out, off)
+    s = np.minimum(rho * adv, np.clip(rho, 0.8, 1.3) * adv)
+    assert abs(a["loss"] - (-(s * masked_out).sum() / 8.0)) < 1e-13
+    # the plain path (no response structure) keeps every valid row
+    c = O.policy_loss_fwd_bwd(H, W, tok, old, ref, adv, mask, 0.2, 0.3, 0.05)
+    assert c["dH"][:2].any() and c["dH"][11:].any()
