@@ -115,6 +115,25 @@ rl_status rl_set_row_group_bytes(rl_ctx* ctx, int64_t bytes);
  * whole step on a board that sits at its power limit does not (the other passes slow down by as
  * much), which is why it is opt-in. */
 rl_status rl_set_dh_stream_k(rl_ctx* ctx, int on);
+/* Upper bound on the CTAs of the persistent tensor-core grids (default: one per SM).  A caller that
+ * overlaps a collective with the backward pass (sections 4.3 / 4.4: sharded training engines) can
+ * leave a few SMs to the collective's kernels this way; an odd bound is rounded down to whole CTA
+ * pairs.  0 restores the default.  Results do not depend on it except where the forward pass
+ * chooses its vocabulary split from the number of workers (summation order of the merge).
+ * Errors: max_ctas < 0 or, after rounding, fewer than 2 -> RL_ERR_INVALID_ARG. */
+rl_status rl_set_max_ctas(rl_ctx* ctx, int max_ctas);
+/* Gradient hand-over for data-parallel training (the paper has no kernel-level counterpart; its
+ * training engines all-reduce gradients after the backward pass).  The backward pass finishes dW
+ * one slab of vocabulary rows at a time.  When a hook is set, rl_policy_loss_fwd_bwd[_ex] calls
+ * hook(user, slab, row_begin, row_end) on the calling host thread right after it has ENQUEUED the
+ * launch that completes rows [row_begin, row_end) of dW: work the hook enqueues behind an event
+ * recorded on the context's stream at that moment (for instance an all-reduce of those rows on
+ * another stream) runs while the remaining slabs are still being computed.  Slabs are reported in
+ * ascending order and cover [0, V) exactly once per call; nothing is reported for T = 0 (dW is then
+ * zero, or untouched when accumulating).  hook = NULL removes it.  The hook must not call into
+ * this context. */
+typedef void (*rl_dw_slab_hook)(void* user, int slab, int64_t row_begin, int64_t row_end);
+rl_status rl_set_dw_slab_hook(rl_ctx* ctx, rl_dw_slab_hook hook, void* user);
 /* Caller-owned device scratch, 256-byte aligned; must outlive the calls that use it. */
 rl_status rl_set_workspace(rl_ctx* ctx, void* dev_ptr, size_t bytes);
 
@@ -250,6 +269,13 @@ typedef struct {
                               /* of 8, bases 16-byte aligned; the reference model is a         */
                               /* constant: no gradient flows to H_ref / W_ref                  */
   float* kl_out;              /* [T] or NULL: per-token KL_t of the kl_full mode (masked rows 0) */
+  const int64_t* token_count; /* device scalar or NULL: the token mean (agg_mode 0 without          */
+                              /* token_weight) divides by *token_count instead of this call's own  */
+                              /* number of valid rows.  Data-parallel ranks pass the count summed   */
+                              /* over ranks, so that the per-rank losses and gradients add up to    */
+                              /* those of the global batch; it is read on the device in stream      */
+                              /* order, the host never sees it.  Not used by the response-aware     */
+                              /* paths (sequence_level, agg_mode 1 / 2).                            */
 } rl_loss_opts;
 
 rl_status rl_policy_loss_fwd_bwd_ex(rl_ctx* ctx, const void* H, int64_t ldH, const void* W,
@@ -406,6 +432,20 @@ rl_status rl_profile_read(rl_ctx* ctx, double* ms, int64_t* launches);
 rl_status rl_selftest_gemm(rl_ctx* ctx, const void* A, const void* B, float* C,
                            int64_t M, int64_t N, int64_t K, int a_mn_major, int b_mn_major,
                            int accumulate);
+
+/* Measurement of data movement between the CTAs of a thread-block cluster through distributed shared
+ * memory (the paper has no counterpart; it prices designs that would keep the gradient with respect
+ * to the logits on chip).  mode 0: per round every CTA of a cluster of cluster_size (2, 4 or 8) sums
+ * its 128 / cluster_size rows of the 128 x 128 fp32 tiles all CTAs hold (remote loads), rounds to
+ * bf16 and writes the result into every CTA's 128 x 128 bf16 tile (remote stores), with two cluster
+ * barriers: per CTA (cluster_size - 1) * (128 / cluster_size) * 128 * 4 bytes come in and half as
+ * many go out.  mode 1: per round every CTA sends `bytes` (multiple of 16, at most 48 KiB) to the CTA
+ * whose rank is its own XOR partner_xor with one bulk shared-to-shared copy that completes on the
+ * receiver's barrier, one cluster barrier per round.  The kernel runs `iters` rounds on as many
+ * clusters as fit the device (n_clusters_host, may be NULL); ms_host (host) receives the device time
+ * of one launch after a warm-up launch.  Synchronises the context's stream. */
+rl_status rl_selftest_cluster_exchange(rl_ctx* ctx, int mode, int cluster_size, int iters, int bytes,
+                                       int partner_xor, float* ms_host, int* n_clusters_host);
 
 /* Host-only view of how a tensor-core pass distributes its work (no GPU is touched; the paper has
  * no counterpart).  For a pass over n_valid rows (at most rows_cap), K extent k_len, n_tiles column

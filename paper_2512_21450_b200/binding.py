@@ -49,7 +49,10 @@ class rl_loss_opts(ctypes.Structure):
         ("ldW_ref", c_int64),
         ("d_ref", c_int64),
         ("kl_out", c_void_p),
+        ("token_count", c_void_p),
     ]
+
+DW_SLAB_HOOK = ctypes.CFUNCTYPE(None, c_void_p, c_int, c_int64, c_int64)
 
 
 _lib = None
@@ -82,6 +85,10 @@ def load_library():
     lib.rl_set_wide_tiles.restype = c_int
     lib.rl_set_dh_stream_k.argtypes = [P, c_int]
     lib.rl_set_dh_stream_k.restype = c_int
+    lib.rl_set_max_ctas.argtypes = [P, c_int]
+    lib.rl_set_max_ctas.restype = c_int
+    lib.rl_set_dw_slab_hook.argtypes = [P, DW_SLAB_HOOK, P]
+    lib.rl_set_dw_slab_hook.restype = c_int
     lib.rl_set_cta_group.argtypes = [P, c_int]
     lib.rl_set_cta_group.restype = c_int
     lib.rl_last_device_status.argtypes = [P, POINTER(c_int32)]
@@ -115,6 +122,8 @@ def load_library():
     lib.rl_debug_schedule.argtypes = [c_int64, c_int64, c_int64, c_int64, c_int, c_int, c_int, c_int, c_int, c_int, c_int,
                                       P, c_int64, POINTER(c_int64)]
     lib.rl_debug_schedule.restype = c_int
+    lib.rl_selftest_cluster_exchange.argtypes = [P, c_int, c_int, c_int, c_int, c_int, POINTER(c_float), POINTER(c_int)]
+    lib.rl_selftest_cluster_exchange.restype = c_int
     lib.rl_mask_scan.argtypes = [P, P, c_int64, P, P]
     lib.rl_mask_scan.restype = c_int
     lib.rl_kl_shaped_returns.argtypes = [P, P, P, P, P, P, P, c_int64, c_int64, c_float, c_float, c_int, P, P]
@@ -211,6 +220,18 @@ class Context:
     def set_dh_stream_k(self, on):
         _check(self.lib.rl_set_dh_stream_k(self.handle, int(on)), "rl_set_dh_stream_k")
 
+    def set_max_ctas(self, max_ctas):
+        _check(self.lib.rl_set_max_ctas(self.handle, int(max_ctas)), "rl_set_max_ctas")
+
+    def set_dw_slab_hook(self, fn):
+        """fn(slab, row_begin, row_end) is called on the host right after the launch that completes those
+        rows of dW has been enqueued; None removes the hook."""
+        if fn is None:
+            self._hook = DW_SLAB_HOOK(0)
+        else:
+            self._hook = DW_SLAB_HOOK(lambda user, slab, r0, r1: fn(slab, r0, r1))
+        _check(self.lib.rl_set_dw_slab_hook(self.handle, self._hook, None), "rl_set_dw_slab_hook")
+
     def set_cta_group(self, cta_group):
         _check(self.lib.rl_set_cta_group(self.handle, cta_group), "rl_set_cta_group")
 
@@ -268,7 +289,7 @@ class Context:
     def rl_policy_loss_fwd_bwd(self, H, W, tokens, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta,
                                ent_coef=0.0, token_weight=None, accumulate_dW=False, dW=None, want_aux=True,
                                dH=None, loss=None, agg_mode=0, sequence_level=False, seq_offsets=None,
-                               dH_fp32=False, H_ref=None, W_ref=None):
+                               dH_fp32=False, H_ref=None, W_ref=None, token_count=None):
         """H_ref [T, d_ref] and W_ref [V, d_ref] (bf16) switch the regulariser to the full-distribution
         KL(pi_theta || pi_ref) against softmax(W_ref h_ref); ref_logp is then unused."""
         self._bind_stream()
@@ -290,7 +311,7 @@ class Context:
             dW = torch.empty(V, d, dtype=torch.float32, device=dev)
         out = dict(loss=loss, dH=dH, dW=dW)
         plain = (ent_coef == 0.0 and token_weight is None and not accumulate_dW and not want_aux and agg_mode == 0
-                 and not sequence_level and not dH_fp32 and not kl_full)
+                 and not sequence_level and not dH_fp32 and not kl_full and token_count is None)
         args = [self.handle, _ptr(H), H.stride(0) if T else d, _ptr(W), W.stride(0), _ptr(tokens), _ptr(old_logp),
                 _ptr(ref_logp), _ptr(adv), _ptr(mask), T, d, V, eps_low, eps_high, beta, _ptr(loss), _ptr(dH),
                 _ptr(dW)]
@@ -305,6 +326,9 @@ class Context:
         opts.agg_mode = agg_mode
         opts.sequence_level = int(sequence_level)
         opts.dH_dtype = int(dH_fp32)
+        if token_count is not None:
+            assert token_count.dtype == torch.int64 and token_count.is_cuda and token_count.numel() == 1
+            opts.token_count = token_count.data_ptr()
         if kl_full:
             opts.kl_full = 1
             opts.H_ref = H_ref.data_ptr() if T else None
@@ -456,6 +480,14 @@ class Context:
     def selftest_wait_timeout(self, limit_ms=20):
         self._bind_stream()
         _check(self.lib.rl_selftest_wait_timeout(self.handle, limit_ms), "rl_selftest_wait_timeout")
+
+    def selftest_cluster_exchange(self, mode, cluster_size, iters, nbytes=0, partner_xor=1):
+        """Device time (ms) of `iters` rounds of the cluster exchange and the number of clusters that ran."""
+        self._bind_stream()
+        ms, ncl = c_float(), c_int()
+        _check(self.lib.rl_selftest_cluster_exchange(self.handle, mode, cluster_size, iters, nbytes, partner_xor,
+                                                     byref(ms), byref(ncl)), "rl_selftest_cluster_exchange")
+        return ms.value, ncl.value
 
     def launch_count(self):
         n = c_int64()

@@ -1,31 +1,47 @@
-// Persistent, warp-specialised bf16 GEMM main loop for sm_100a with pluggable epilogues.
+// Persistent, warp-specialised bf16 GEMM main loop for sm_100a with pluggable epilogues.  One
+// kernel template serves every tensor-core pass of the library; a tile mode picks how the two
+// 256-column fp32 accumulators of tensor memory are used.
 //
 //   warp 0      : TMA producer (one lane) - streams A and B k-slices (64 elements of K) into a
 //                 shared-memory ring, 128-byte swizzled.
-//   warp 1      : allocates tensor memory; one lane issues tcgen05.mma into one of two
-//                 256-column fp32 accumulators.
+//   warp 1      : allocates tensor memory; one lane issues tcgen05.mma.
 //   warps 2..5  : epilogue - each warp owns the 32 tensor-memory lanes (tile rows) that its
 //                 rank modulo 4 may read, pulls the accumulator out in 32-column chunks and
-//                 hands them to the epilogue functor.  While they drain accumulator a, the MMA
-//                 warp already fills accumulator a^1.
+//                 hands them to the epilogue functor.
 //
-// CG = 1: one CTA per 128x256 output tile (4 stages of 16 KB A + 32 KB B).
-// CG = 2: a cluster of two CTAs (one SM pair) per 256x256 output tile.  Each CTA stages its own
-//         128 rows of A and 128 of the 256 columns of B (7 stages of 16 KB + 16 KB), the even
-//         CTA issues tcgen05.mma.cta_group::2 (M = 256) which reads both halves of B and writes
-//         128 accumulator rows into each CTA's tensor memory; both CTAs run their own epilogue.
-//         All TMA completions of a stage are counted on the even CTA's barrier; stage-free and
-//         accumulator-ready signals reach both CTAs through one tcgen05.commit; the odd CTA's
-//         epilogue reports "accumulator drained" to the even CTA with a remote mbarrier arrive.
-//         Every TMA load is addressed to the shared memory of the CTA that issues it.
+// Tile modes (per CTA 128 accumulator rows):
+//   kTileSquare : a tile is 256 columns wide and lives in ONE accumulator; tile t uses accumulator
+//                 t & 1, so the MMAs of tile t + 1 overlap the epilogue of tile t.  Used where K is
+//                 short and the epilogue heavy (forward statistics, gradient of the logits).
+//   kTileWide   : a tile is 512 columns wide and fills BOTH accumulators; a stage holds A and two B
+//                 boxes, every k-slice of A feeds two UMMAs, so a CTA pulls a quarter fewer operand
+//                 bytes from L2 per flop; the epilogue of a tile no longer overlaps the next main
+//                 loop (about 1 % of a tile at K of 17-19 thousand).  CTA pairs only.  Used for the
+//                 two long-K gradient products dH = G W and dW = G^T H.
+//   kTileDual   : a tile is 256 columns wide and BOTH accumulators hold it, one per product:
+//                 Z = A B^T (K = k_len) and Z2 = A2 B2^T (K = k2_len) of the same rows and columns,
+//                 whose 32-column chunks reach the epilogue side by side.  Used for the
+//                 full-distribution KL (policy and reference logits).  All operands K-major.
+//
+// CG = 1: one CTA per 128-row tile (4 stages of 16 KB A + 32 KB B).
+// CG = 2: a cluster of two CTAs (one SM pair) per 256-row tile.  Each CTA stages its own 128 rows
+//         of A and 128 of every 256 columns of B, the even CTA issues tcgen05.mma.cta_group::2
+//         (M = 256) which reads both halves of B and writes 128 accumulator rows into each CTA's
+//         tensor memory; both CTAs run their own epilogue.  All TMA completions of a stage are
+//         counted on the even CTA's barrier; stage-free and accumulator-ready signals reach both
+//         CTAs through one tcgen05.commit; the odd CTA's epilogue reports its accumulator drained
+//         to the even CTA with a remote mbarrier arrive.  Every TMA load is addressed to the
+//         shared memory of the CTA that issues it.
 //
 // Either operand may be K-major (its global tensor is [rows, K], K contiguous) or MN-major
 // (its global tensor is [K, rows], rows contiguous).  A K-major tile is one 2-D TMA box
 // {64 k, rows}; an MN-major tile is one 3-D box {64 rows, 64 k, rows/64}, which lands in shared
 // memory as rows/64 panels of 8 KB, each panel 64 k-lines of 128 bytes.
 //
-// Every wait is bounded: when one runs out the block raises a shared abort flag, every role
-// leaves its loop, the status word is latched and the block still frees its tensor memory.
+// All three roles walk the same list of work units (UnitWalk), so K slices, stream-K balancing and
+// row groups exist for every tile mode.  Every wait is bounded: when one runs out the block raises
+// a shared abort flag, every role leaves its loop, the status word is latched and the block still
+// frees its tensor memory.
 #pragma once
 #include <cuda.h>
 
@@ -45,14 +61,17 @@ constexpr int kTmemCols = 512;
 constexpr int kMaxSplit = 16;   // most column ranges per row tile when the split is chosen to fill the machine
 constexpr int kFwdRange = 8;    // column tiles per work unit when there is plenty of work
 
+enum TileMode { kTileSquare = 0, kTileWide = 1, kTileDual = 2 };
+
 // kStaging: bytes of shared memory the epilogue keeps for itself behind the ring.
-template <int CG, int kStaging>
+template <int CG, int MODE, int kStaging>
 struct StageCfg {
-  static constexpr int kBRows = BN / CG;                    // B rows (output columns) staged per CTA
+  static constexpr int kBRows = BN / CG;                    // B rows (output columns) of one box staged per CTA
   static constexpr int kBBytes = kBRows * BK * 2;
-  static constexpr int kStageBytes = kAStageBytes + kBBytes;
-  static constexpr int kRingBytes = (kTileSmemBytes - kStaging) / kStageBytes * kStageBytes;
-  static constexpr int kStages = kRingBytes / kStageBytes;  // 4 (CG = 1); 7 or 6 (CG = 2)
+  static constexpr int kBBoxes = MODE == kTileWide ? 2 : 1; // B boxes per stage
+  static constexpr int kStageBytes = kAStageBytes + kBBoxes * kBBytes;
+  static constexpr int kStages = (kTileSmemBytes - kStaging) / kStageBytes;   // 4 (CG = 1); 7 or 6 (pairs); 4 (wide)
+  static constexpr int kRingBytes = kStages * kStageBytes;
   static constexpr uint32_t kTxBytes = uint32_t(kStageBytes) * CG;  // bytes counted on the issuing CTA's barrier
 };
 constexpr int kMaxStages = 7;
@@ -261,19 +280,25 @@ struct UnitWalk {
 // Epilogue functor contract (all methods run in the 128 epilogue threads, one tile row each):
 //   struct Epi { struct Params; struct State;
 //     static void begin_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows, int slab_off, int k_slice);
-//     static void chunk(const Params&, State&, int m_tile, int n_tile, int chunk, int row_in_tile, int m_rows, const float (&v)[32]);
+//     static void chunk(const Params&, State&, int m_tile, int n_tile, int chunk, int row_in_tile, int m_rows, const float (&v)[32],
+//                       const CUtensorMap* out_map, uint32_t staging);
 //     static void end_unit(const Params&, State&, int m_tile, int n_range_idx, int row_in_tile, int m_rows);
 //     static void init(State&); static void finish(State&);     // once per kernel, per thread
 //     static constexpr int kStagingBytes;                      // shared memory behind the ring (0 or 32 KB) };
-//   chunk additionally receives the output tensor map and the warp's staging address.
-// m_tile counts 128-row tiles.
-template <class Epi, int A_MN, int B_MN, int CG>
+//   kTileDual: chunk receives the chunk of the second product as well (..., v, v2, out_map, staging).
+// m_tile counts 128-row tiles, n_tile 256-column tiles (a wide tile n covers column tiles 2n and 2n + 1;
+// sh.n_tiles then counts 512-wide tiles).  tmA2 / tmB2 / k2_len are read by kTileDual only.
+template <class Epi, int A_MN, int B_MN, int CG, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const __grid_constant__ CUtensorMap tmC, const GemmShape sh, const typename Epi::Params ep,
-            DevStatus* status) {
-  using Cfg = StageCfg<CG, Epi::kStagingBytes>;
+            const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
+            const __grid_constant__ CUtensorMap tmC, const GemmShape sh, const int k2_len,
+            const typename Epi::Params ep, DevStatus* status) {
+  static_assert(MODE != kTileWide || CG == 2, "wide tiles run on CTA pairs");
+  static_assert(MODE != kTileDual || (A_MN == 0 && B_MN == 0), "the two-product mode takes K-major operands");
+  using Cfg = StageCfg<CG, MODE, Epi::kStagingBytes>;
   constexpr int kStages = Cfg::kStages;
+  constexpr int kProducts = MODE == kTileDual ? 2 : 1;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
@@ -298,6 +323,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
+    if (MODE == kTileDual) { prefetch_tmap(&tmA2); prefetch_tmap(&tmB2); }
   }
   if (warp == 1) {
     if (CG == 2) { tmem_alloc_pair(smem_u32(&tmem_base_smem), kTmemCols); tmem_relinquish_pair(); }
@@ -311,10 +337,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_p = &abort_flag;
 
   const GemmExtents ex = gemm_extents(sh, sh.n_valid ? *sh.n_valid : 0, CG, n_workers);
+  const int k2_blocks = MODE == kTileDual ? (k2_len + BK - 1) / BK : 0;
+  // the two-product mode has nothing to do unless both products have a K range
+  const bool run = MODE != kTileDual || (ex.k_blocks > 0 && k2_blocks > 0);
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer (both CTAs)
-    if (lane == 0) {
+    if (lane == 0 && run) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -323,35 +352,47 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       while (ok && walk.next(mu, nr, ks, kb0, kb1)) {
         const int m = mu * CG + (int)rank;
         const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
+        const int a_row = sh.a_mn_off + (sh.a_mn_slab ? ex.slab_off : 0) + m * BM;
         for (int n = n0; n < n1 && ok; ++n) {
-          for (int kb = kb0; kb < kb1; ++kb) {
-            if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p)) {
-              latch_status(status, kStatusTimeout, (1 << 28) | (blockIdx.x << 8) | stage);
-              ok = false;
-              break;
-            }
-            const uint32_t full_local = smem_u32(&bar_full[stage]);
-            const uint32_t a_dst = tiles_base + stage * Cfg::kStageBytes;
-            const uint32_t b_dst = a_dst + kAStageBytes;
-            const int a_row = sh.a_mn_off + (sh.a_mn_slab ? ex.slab_off : 0) + m * BM;
-            const int b_row = sh.b_mn_off + n * BN + (int)rank * Cfg::kBRows;
-            const int b_k = sh.b_k_off + (sh.b_k_slab ? ex.slab_off : 0) + kb * BK;
-            if (CG == 1) {
-              mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
-              if (A_MN) tma_load_3d(a_dst, &tmA, full_local, 0, sh.a_k_off + kb * BK, a_row / 64);
-              else      tma_load_2d(a_dst, &tmA, full_local, sh.a_k_off + kb * BK, a_row);
-              if (B_MN) tma_load_3d(b_dst, &tmB, full_local, 0, b_k, b_row / 64);
-              else      tma_load_2d(b_dst, &tmB, full_local, b_k, b_row);
-            } else {
+          for (int prod = 0; prod < kProducts && ok; ++prod) {
+            const CUtensorMap* ta = prod ? &tmA2 : &tmA;
+            const CUtensorMap* tb = prod ? &tmB2 : &tmB;
+            const int lo = prod ? 0 : kb0, hi = prod ? k2_blocks : kb1;
+            for (int kb = lo; kb < hi; ++kb) {
+              if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p)) {
+                latch_status(status, kStatusTimeout, (1 << 28) | (blockIdx.x << 8) | stage);
+                ok = false;
+                break;
+              }
+              const uint32_t full_local = smem_u32(&bar_full[stage]);
+              const uint32_t a_dst = tiles_base + stage * Cfg::kStageBytes;
+              const uint32_t b_dst = a_dst + kAStageBytes;
+              const int a_k = (prod ? 0 : sh.a_k_off) + kb * BK;
+              const int b_k = (prod ? 0 : sh.b_k_off + (sh.b_k_slab ? ex.slab_off : 0)) + kb * BK;
               // the even CTA's barrier counts the bytes of both CTAs' copies
-              if (rank == 0) mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
-              const uint32_t full = mapa_cluster(full_local, 0);
-              if (A_MN) tma_load_3d_pair(a_dst, &tmA, full, 0, sh.a_k_off + kb * BK, a_row / 64);
-              else      tma_load_2d_pair(a_dst, &tmA, full, sh.a_k_off + kb * BK, a_row);
-              if (B_MN) tma_load_3d_pair(b_dst, &tmB, full, 0, b_k, b_row / 64);
-              else      tma_load_2d_pair(b_dst, &tmB, full, b_k, b_row);
+              if (CG == 1 || rank == 0) mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
+              const uint32_t full = CG == 2 ? mapa_cluster(full_local, 0) : full_local;
+              if (CG == 1) {
+                if (A_MN) tma_load_3d(a_dst, ta, full, 0, a_k, a_row / 64);
+                else      tma_load_2d(a_dst, ta, full, a_k, a_row);
+              } else {
+                if (A_MN) tma_load_3d_pair(a_dst, ta, full, 0, a_k, a_row / 64);
+                else      tma_load_2d_pair(a_dst, ta, full, a_k, a_row);
+              }
+#pragma unroll
+              for (int s = 0; s < Cfg::kBBoxes; ++s) {
+                const int b_row = sh.b_mn_off + (n * Cfg::kBBoxes + s) * BN + (int)rank * Cfg::kBRows;
+                const uint32_t dst = b_dst + s * Cfg::kBBytes;
+                if (CG == 1) {
+                  if (B_MN) tma_load_3d(dst, tb, full, 0, b_k, b_row / 64);
+                  else      tma_load_2d(dst, tb, full, b_k, b_row);
+                } else {
+                  if (B_MN) tma_load_3d_pair(dst, tb, full, 0, b_k, b_row / 64);
+                  else      tma_load_2d_pair(dst, tb, full, b_k, b_row);
+                }
+              }
+              if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
       }
@@ -375,41 +416,53 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       constexpr uint32_t b_kstep = B_MN ? 2048 : 32;
       int stage = 0;
       uint32_t phase = 0;
-      uint32_t t = 0;
+      uint32_t t = 0;   // tiles issued so far
       bool ok = true;
-      if (ex.k_blocks > 0) {
+      if (run && ex.k_blocks > 0) {
         UnitWalk walk(sh, ex, worker, n_workers);
         int mu, nr, ks, kb0, kb1;
         while (ok && walk.next(mu, nr, ks, kb0, kb1)) {
           if (kb1 <= kb0) continue;   // empty K slice: the epilogue handles it without an accumulator
           const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
           for (int n = n0; n < n1 && ok; ++n, ++t) {
-            const uint32_t a = t & 1u, round = t >> 1;
-            if (!mbar_wait_bounded_cluster(smem_u32(&bar_acc_empty[a]), (round & 1u) ^ 1u, abort_p)) {
-              latch_status(status, kStatusTimeout, (2 << 28) | (blockIdx.x << 8) | a);
-              ok = false;
-              break;
-            }
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + a * BN;
-            for (int kb = kb0; kb < kb1; ++kb) {
-              if (!mbar_wait_bounded_cluster(smem_u32(&bar_full[stage]), phase, abort_p)) {
-                latch_status(status, kStatusTimeout, (3 << 28) | (blockIdx.x << 8) | stage);
+            // square tiles alternate between the accumulators; the other modes need both drained
+            const uint32_t a = MODE == kTileSquare ? (t & 1u) : 0u;
+            const uint32_t par = MODE == kTileSquare ? (((t >> 1) & 1u) ^ 1u) : ((t & 1u) ^ 1u);
+            for (uint32_t w = a; w < (MODE == kTileWide ? 2u : a + 1u) && ok; ++w) {
+              if (!mbar_wait_bounded_cluster(smem_u32(&bar_acc_empty[w]), par, abort_p)) {
+                latch_status(status, kStatusTimeout, (2 << 28) | (blockIdx.x << 8) | w);
                 ok = false;
-                break;
               }
-              tc_fence_after();
-              const uint32_t a_src = tiles_base + stage * Cfg::kStageBytes;
-              const uint32_t b_src = a_src + kAStageBytes;
+            }
+            if (!ok) break;
+            tc_fence_after();
+            for (int prod = 0; prod < kProducts && ok; ++prod) {
+              const uint32_t d_tmem = tmem_base + (MODE == kTileDual ? prod : a) * BN;
+              const int lo = prod ? 0 : kb0, hi = prod ? k2_blocks : kb1;
+              for (int kb = lo; kb < hi; ++kb) {
+                if (!mbar_wait_bounded_cluster(smem_u32(&bar_full[stage]), phase, abort_p)) {
+                  latch_status(status, kStatusTimeout, (3 << 28) | (blockIdx.x << 8) | stage);
+                  ok = false;
+                  break;
+                }
+                tc_fence_after();
+                const uint32_t a_src = tiles_base + stage * Cfg::kStageBytes;
+                const uint32_t b_src = a_src + kAStageBytes;
 #pragma unroll
-              for (int k = 0; k < BK / 16; ++k) {
-                const uint64_t da = smem_desc(a_hi, a_src + k * a_kstep), db = smem_desc(b_hi, b_src + k * b_kstep);
-                if (CG == 2) umma_bf16_pair(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-                else         umma_bf16(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                for (int k = 0; k < BK / 16; ++k) {
+                  const uint64_t da = smem_desc(a_hi, a_src + k * a_kstep);
+                  const uint32_t acc = (kb > lo || k > 0) ? 1u : 0u;
+#pragma unroll
+                  for (int s = 0; s < Cfg::kBBoxes; ++s) {
+                    const uint64_t db = smem_desc(b_hi, b_src + s * Cfg::kBBytes + k * b_kstep);
+                    if (CG == 2) umma_bf16_pair(d_tmem + s * BN, da, db, idesc, acc);
+                    else         umma_bf16(d_tmem + s * BN, da, db, idesc, acc);
+                  }
+                }
+                if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_empty[stage]), 3);
+                else         umma_commit(smem_u32(&bar_empty[stage]));
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
               }
-              if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_empty[stage]), 3);
-              else         umma_commit(smem_u32(&bar_empty[stage]));
-              if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
             if (ok) {
               if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_acc_full[a]), 3);
@@ -436,15 +489,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     bool ok = true;
     UnitWalk walk(sh, ex, worker, n_workers);
     int mu, nr, ks, kb0, kb1;
-    while (ok && walk.next(mu, nr, ks, kb0, kb1)) {
+    while (ok && run && walk.next(mu, nr, ks, kb0, kb1)) {
       const bool has_k = kb1 > kb0;   // an empty K slice contributes zeros
       const int m = mu * CG + (int)rank;
       const int n0 = nr * ex.n_range, n1 = min(n0 + ex.n_range, sh.n_tiles);
       Epi::begin_unit(ep, st, m, nr, row_in_tile, ex.m_rows, ex.slab_off, ks);
       for (int n = n0; n < n1 && ok; ++n, t += has_k ? 1u : 0u) {
-        const uint32_t a = t & 1u, round = t >> 1;
+        const uint32_t a = MODE == kTileSquare ? (t & 1u) : 0u;
         if (has_k) {
-          if (!mbar_wait_bounded_cluster(smem_u32(&bar_acc_full[a]), round & 1u, abort_p)) {
+          const uint32_t par = MODE == kTileSquare ? ((t >> 1) & 1u) : (t & 1u);
+          if (!mbar_wait_bounded_cluster(smem_u32(&bar_acc_full[a]), par, abort_p)) {
             latch_status(status, kStatusTimeout, (5 << 28) | (blockIdx.x << 8) | a);
             ok = false;
           }
@@ -452,28 +506,43 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (!ok) break;
           tc_fence_after();
         }
-        const uint32_t taddr = tmem_base + a * BN + (uint32_t(q * 32) << 16);
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          float v[32];
-          if (has_k) {
-            uint32_t r[32];
-            tmem_ld_32x32(taddr + c * 32, r);
-            tmem_ld_wait();
+        for (int s = 0; s < Cfg::kBBoxes; ++s) {
+          const uint32_t acc_i = a + (uint32_t)s;   // accumulator this half of the tile sits in
+          const uint32_t taddr = tmem_base + acc_i * BN + (uint32_t(q * 32) << 16);
+#pragma unroll 1
+          for (int c = 0; c < BN / 32; ++c) {
+            float v[32];
+            if constexpr (MODE == kTileDual) {
+              uint32_t r[32], r2[32];
+              tmem_ld_32x32(taddr + c * 32, r);
+              tmem_ld_32x32(taddr + BN + c * 32, r2);
+              tmem_ld_wait();
+              float v2[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-          } else {
+              for (int i = 0; i < 32; ++i) { v[i] = __uint_as_float(r[i]); v2[i] = __uint_as_float(r2[i]); }
+              Epi::chunk(ep, st, m, n, c, row_in_tile, ex.m_rows, v, v2, &tmC, staging);
+            } else {
+              if (has_k) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + c * 32, r);
+                tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = 0.f;
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = 0.f;
+              }
+              Epi::chunk(ep, st, m, n * Cfg::kBBoxes + s, c, row_in_tile, ex.m_rows, v, &tmC, staging);
+            }
           }
-          Epi::chunk(ep, st, m, n, c, row_in_tile, ex.m_rows, v, &tmC, staging);
-        }
-        if (has_k) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            if (CG == 2 && rank != 0) mbar_arrive_cluster(mapa_cluster(smem_u32(&bar_acc_empty[a]), 0));
-            else                      mbar_arrive(smem_u32(&bar_acc_empty[a]));
+          if (has_k) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+              if (CG == 2 && rank != 0) mbar_arrive_cluster(mapa_cluster(smem_u32(&bar_acc_empty[acc_i]), 0));
+              else                      mbar_arrive(smem_u32(&bar_acc_empty[acc_i]));
+            }
           }
         }
       }

@@ -1,7 +1,6 @@
-// Epilogues of the two-product engine: full-distribution KL(pi_theta || pi_ref) per token
+// Epilogues of the two-product tile mode of the GEMM engine: full-distribution KL(pi_theta || pi_ref) per token
 // (section 2.2 "KL-to-reference", section 3.1 Omega) and its gradient with respect to the logits.
 #pragma once
-#include "dual_engine.cuh"
 #include "epilogues.cuh"
 
 namespace rlh {

@@ -11,7 +11,7 @@
 
 #include "rlhead.h"
 #include "small_kernels.cuh"
-#include "wide_engine.cuh"
+#include "cluster_probe.cuh"
 
 using namespace rlh;
 
@@ -39,6 +39,9 @@ struct rl_ctx {
   int wide_tiles;   // 1: dH and dW run on 256 x 512 tiles (both accumulators hold one tile)
   int dh_stream_k;  // 1: the dH pass balances its tiles over the SMs by stream-K (needs a second accumulator buffer)
   int grid[3];    // persistent grid for cta_group 1 and 2 (index = cta_group)
+  int grid_full[3];   // the same before rl_set_max_ctas() capped it
+  rl_dw_slab_hook dw_hook;   // called after the launch that completes a slab of dW rows was enqueued
+  void* dw_hook_user;
   long long launches;  // kernels launched by this context so far
   // optional per-kernel timing: event pairs around every tensor-core launch, by kernel kind
   int prof_on;
@@ -198,21 +201,21 @@ bool map_out_bf16(rl_ctx* c, CUtensorMap* m, const void* base, uint64_t rows, ui
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <class Epi, int A_MN, int B_MN>
-cudaError_t set_smem_attr() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kGemmSmemBytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <class Epi, int A_MN, int B_MN, int CG, int MODE>
+cudaError_t set_smem_attr_one() {
+  return cudaFuncSetAttribute(gemm_kernel<Epi, A_MN, B_MN, CG, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               kGemmSmemBytes);
 }
-
+// square tiles, single CTAs and CTA pairs
+template <class Epi, int A_MN, int B_MN>
+cudaError_t set_smem_attr() {
+  cudaError_t e = set_smem_attr_one<Epi, A_MN, B_MN, 1, kTileSquare>();
+  return e != cudaSuccess ? e : set_smem_attr_one<Epi, A_MN, B_MN, 2, kTileSquare>();
+}
 template <class Epi>
 cudaError_t set_smem_attr_dual() {
-  cudaError_t e = cudaFuncSetAttribute(dual_gemm_kernel<Epi, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kGemmSmemBytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(dual_gemm_kernel<Epi, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+  cudaError_t e = set_smem_attr_one<Epi, 0, 0, 1, kTileDual>();
+  return e != cudaSuccess ? e : set_smem_attr_one<Epi, 0, 0, 2, kTileDual>();
 }
 
 // Rows of B that one CTA stages per k-slice (box height of a K-major B map) and the number of
@@ -236,9 +239,12 @@ void prof_end(rl_ctx* c, int i, int kind) {
   c->prof_used = i + 1;
 }
 
-template <class Epi, int A_MN, int B_MN>
-void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& out,
-                 const GemmShape& sh, const typename Epi::Params& ep) {
+// One launch of the tensor-core engine in tile mode MODE on the context's persistent grid (CTA pairs
+// when cta_group is 2; wide tiles exist for pairs only).  a2 / b2 / k2_len: second product (kTileDual).
+template <class Epi, int A_MN, int B_MN, int MODE>
+void launch_tiles(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
+                  const CUtensorMap& b2, const CUtensorMap& out, const GemmShape& sh, int k2_len,
+                  const typename Epi::Params& ep) {
   const int prof = prof_begin(c, kind);
   if (c->cta_group == 2) {
     cudaLaunchConfig_t cfg;
@@ -254,68 +260,35 @@ void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, gemm_kernel<Epi, A_MN, B_MN, 2>, a, b, out, sh, ep, c->dstatus);
-  } else {
-    gemm_kernel<Epi, A_MN, B_MN, 1><<<c->grid[1], kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, out, sh, ep,
-                                                                                            c->dstatus);
+    cudaLaunchKernelEx(&cfg, gemm_kernel<Epi, A_MN, B_MN, 2, MODE>, a, b, a2, b2, out, sh, k2_len, ep, c->dstatus);
+  } else if constexpr (MODE != kTileWide) {
+    gemm_kernel<Epi, A_MN, B_MN, 1, MODE><<<c->grid[1], kGemmThreads, kGemmSmemBytes, c->stream>>>(
+        a, b, a2, b2, out, sh, k2_len, ep, c->dstatus);
   }
   c->launches++;
   prof_end(c, prof, kind);
 }
 
-// 256 x 512 tiles on CTA pairs; sh.n_tiles counts 512-wide column tiles.
-inline bool use_wide(const rl_ctx* c) {
-  return c->wide_tiles && c->cta_group == 2 && c->dh_k_slices == 1 && !c->dh_stream_k;
+template <class Epi, int A_MN, int B_MN>
+void launch_gemm(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& out,
+                 const GemmShape& sh, const typename Epi::Params& ep) {
+  launch_tiles<Epi, A_MN, B_MN, kTileSquare>(c, kind, a, b, a, b, out, sh, 0, ep);
 }
+
+// 256 x 512 tiles on CTA pairs; sh.n_tiles counts 512-wide column tiles.
+inline bool use_wide(const rl_ctx* c) { return c->wide_tiles && c->cta_group == 2; }
 
 template <class Epi, int A_MN, int B_MN>
 void launch_wide(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& out,
                  const GemmShape& sh, const typename Epi::Params& ep) {
-  const int prof = prof_begin(c, kind);
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(c->grid[2]);
-  cfg.blockDim = dim3(kGemmThreads);
-  cfg.dynamicSmemBytes = kGemmSmemBytes;
-  cfg.stream = c->stream;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = 2;
-  attr.val.clusterDim.y = 1;
-  attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, gemm_wide_kernel<Epi, A_MN, B_MN>, a, b, out, sh, ep, c->dstatus);
-  c->launches++;
-  prof_end(c, prof, kind);
+  launch_tiles<Epi, A_MN, B_MN, kTileWide>(c, kind, a, b, a, b, out, sh, 0, ep);
 }
 
 template <class Epi>
 void launch_dual(rl_ctx* c, int kind, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
                  const CUtensorMap& b2, const CUtensorMap& out, const GemmShape& sh, int k2_len,
                  const typename Epi::Params& ep) {
-  const int prof = prof_begin(c, kind);
-  if (c->cta_group == 2) {
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3(c->grid[2]);
-    cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = kGemmSmemBytes;
-    cfg.stream = c->stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, dual_gemm_kernel<Epi, 2>, a, b, a2, b2, out, sh, k2_len, ep, c->dstatus);
-  } else {
-    dual_gemm_kernel<Epi, 1><<<c->grid[1], kGemmThreads, kGemmSmemBytes, c->stream>>>(a, b, a2, b2, out, sh, k2_len,
-                                                                                     ep, c->dstatus);
-  }
-  c->launches++;
-  prof_end(c, prof, kind);
+  launch_tiles<Epi, 0, 0, kTileDual>(c, kind, a, b, a2, b2, out, sh, k2_len, ep);
 }
 
 rl_status check_hw(const void* H, int64_t ldH, const void* W, int64_t ldW, int64_t T, int64_t d, int64_t V) {
@@ -496,10 +469,10 @@ rl_status rl_create(rl_ctx** out, int device) {
             set_smem_attr<EpiAcc, 0, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 0, 1>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess &&
             set_smem_attr_dual<EpiStatsKL>() == cudaSuccess && set_smem_attr_dual<EpiGradKL>() == cudaSuccess &&
-            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess &&
-            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess &&
-            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess &&
-            cudaFuncSetAttribute(gemm_wide_kernel<EpiAcc, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) == cudaSuccess;
+            set_smem_attr_one<EpiAcc, 0, 0, 2, kTileWide>() == cudaSuccess &&
+            set_smem_attr_one<EpiAcc, 0, 1, 2, kTileWide>() == cudaSuccess &&
+            set_smem_attr_one<EpiAcc, 1, 0, 2, kTileWide>() == cudaSuccess &&
+            set_smem_attr_one<EpiAcc, 1, 1, 2, kTileWide>() == cudaSuccess;
   if (!ok) { cudaFree(c->dstatus); delete c; return RL_ERR_CUDA; }
   {
     // how many CTA pairs can be resident at once (pairs must share a TPC): the persistent grid
@@ -517,7 +490,7 @@ rl_status rl_create(rl_ctx** out, int device) {
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&n_clusters, gemm_kernel<EpiAcc, 0, 0, 2>, &cfg) == cudaSuccess &&
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, gemm_kernel<EpiAcc, 0, 0, 2, kTileSquare>, &cfg) == cudaSuccess &&
         n_clusters > 0) {
       if (2 * n_clusters < c->grid[2]) c->grid[2] = 2 * n_clusters;
     } else {
@@ -526,6 +499,9 @@ rl_status rl_create(rl_ctx** out, int device) {
     }
     if (c->grid[2] >= 2) c->cta_group = 2;   // default: CTA pairs
   }
+  for (int i = 0; i < 3; ++i) c->grid_full[i] = c->grid[i];
+  c->dw_hook = nullptr;
+  c->dw_hook_user = nullptr;
   *out = c;
   return RL_OK;
 }
@@ -582,6 +558,26 @@ rl_status rl_set_cta_group(rl_ctx* c, int cta_group) {
   if (cta_group != 1 && cta_group != 2) return RL_ERR_INVALID_ARG;
   if (cta_group == 2 && c->grid[2] < 2) return RL_ERR_UNSUPPORTED_ARCH;
   c->cta_group = cta_group;
+  return RL_OK;
+}
+
+rl_status rl_set_max_ctas(rl_ctx* c, int max_ctas) {
+  if (!c || max_ctas < 0) return RL_ERR_INVALID_ARG;
+  if (max_ctas == 0) {
+    for (int i = 0; i < 3; ++i) c->grid[i] = c->grid_full[i];
+    return RL_OK;
+  }
+  if (max_ctas < 2) return RL_ERR_INVALID_ARG;
+  c->grid[1] = max_ctas < c->grid_full[1] ? max_ctas : c->grid_full[1];
+  const int pairs = max_ctas / 2 * 2;
+  c->grid[2] = pairs < c->grid_full[2] ? pairs : c->grid_full[2];
+  return RL_OK;
+}
+
+rl_status rl_set_dw_slab_hook(rl_ctx* c, rl_dw_slab_hook hook, void* user) {
+  if (!c) return RL_ERR_INVALID_ARG;
+  c->dw_hook = hook;
+  c->dw_hook_user = hook ? user : nullptr;
   return RL_OK;
 }
 
@@ -917,6 +913,7 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
   p.eps_high = eps_high;
   p.beta = beta;
   p.ent_coef = o.ent_coef;
+  p.token_count = reinterpret_cast<const long long*>(o.token_count);
   p.with_loss = 1;
   p.lse_c = reinterpret_cast<float*>(ws + L.lse_c);
   p.ent_c = reinterpret_cast<float*>(ws + L.ent_c);
@@ -1089,6 +1086,8 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
         } else {
           launch_gemm<EpiAcc, 1, 1>(c, 3, tmG_mn, tmHc_mn, tm_dW, sh, ep);
         }
+        // rows [vocab_base, vocab_base + cols) of dW are complete once the last row slab has added to them
+        if (c->dw_hook && r == n_row_slabs - 1) c->dw_hook(c->dw_hook_user, cs, vocab_base, (int64_t)vocab_base + cols);
       }
     }
     const int pr_sc = prof_begin(c, 7);
@@ -1444,6 +1443,61 @@ rl_status rl_selftest_wait_timeout(rl_ctx* c, int limit_ms) {
   wait_timeout_probe_kernel<<<1, 32, 0, c->stream>>>((unsigned long long)limit_ms * 1000000ull, c->dstatus);
   c->launches++;
   return cuda_ok();
+}
+
+rl_status rl_selftest_cluster_exchange(rl_ctx* c, int mode, int cluster_size, int iters, int bytes, int partner_xor,
+                                       float* ms_host, int* n_clusters_host) {
+  if (!c || !ms_host || (mode != 0 && mode != 1) || iters < 1 || iters > (1 << 20)) return RL_ERR_INVALID_ARG;
+  if (cluster_size != 2 && cluster_size != 4 && cluster_size != 8) return RL_ERR_INVALID_ARG;
+  size_t smem = 1024;
+  if (mode == 0) {
+    smem += (size_t)kProbeTile * kProbeTile * 6;
+  } else {
+    if (bytes < 16 || bytes % 16 != 0 || bytes > 48 * 1024 || partner_xor < 1 || partner_xor >= cluster_size)
+      return RL_ERR_INVALID_ARG;
+    smem += 4 * (size_t)bytes;
+  }
+  if (cudaFuncSetAttribute(cluster_exchange_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return RL_ERR_CUDA;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(c->n_sm / cluster_size * cluster_size);
+  cfg.blockDim = dim3(kProbeThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = cluster_size;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int n_clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&n_clusters, cluster_exchange_kernel, &cfg) != cudaSuccess || n_clusters < 1) {
+    cudaGetLastError();
+    return RL_ERR_UNSUPPORTED_ARCH;
+  }
+  if (n_clusters * cluster_size < (int)cfg.gridDim.x) cfg.gridDim = dim3(n_clusters * cluster_size);
+  if (n_clusters_host) *n_clusters_host = (int)cfg.gridDim.x / cluster_size;
+  float* sink = reinterpret_cast<float*>(reinterpret_cast<char*>(c->dstatus) + 128);   // never written in practice
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+    if (e0) cudaEventDestroy(e0);
+    return RL_ERR_CUDA;
+  }
+  rl_status rs = RL_OK;
+  for (int pass = 0; pass < 2 && rs == RL_OK; ++pass) {   // one warm-up launch, one timed
+    if (pass == 1) cudaEventRecord(e0, c->stream);
+    if (cudaLaunchKernelEx(&cfg, cluster_exchange_kernel, mode, iters, bytes, partner_xor, sink, c->dstatus) != cudaSuccess)
+      rs = RL_ERR_CUDA;
+    c->launches++;
+  }
+  cudaEventRecord(e1, c->stream);
+  if (rs == RL_OK && cudaEventSynchronize(e1) != cudaSuccess) rs = RL_ERR_CUDA;
+  if (rs == RL_OK && cudaEventElapsedTime(ms_host, e0, e1) != cudaSuccess) rs = RL_ERR_CUDA;
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  return rs;
 }
 
 rl_status rl_selftest_gemm(rl_ctx* c, const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,

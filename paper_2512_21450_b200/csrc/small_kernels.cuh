@@ -453,6 +453,7 @@ struct LossParams {
   const float* ref_logp;   // [T] or NULL
   const float* adv;        // [T]
   const float* token_weight;  // [T] or NULL
+  const long long* token_count;   // device scalar or NULL: divisor of the token mean (data-parallel global count)
   float eps_low, eps_high, beta, ent_coef;
   int with_loss;
   // full-distribution KL to the reference policy (two-product forward): second partial per
@@ -492,7 +493,8 @@ __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossPa
   double acc[kLossSums];
 #pragma unroll
   for (int k = 0; k < kLossSums; ++k) acc[k] = 0.0;
-  const float w_mean = n > 0 ? 1.f / (float)n : 0.f;
+  const long long n_mean = p.token_count ? *p.token_count : (long long)n;
+  const float w_mean = n_mean > 0 ? (float)(1.0 / (double)n_mean) : 0.f;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
     float lse, logp, ent;
     float M = -CUDART_INF_F, S = 0.f, A = 0.f;

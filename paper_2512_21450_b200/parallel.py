@@ -28,12 +28,12 @@ def global_valid_count(mask: torch.Tensor, group=None) -> torch.Tensor:
 
 
 def global_token_weight(mask: torch.Tensor, group=None) -> torch.Tensor:
-    """Per-row weight 1 / (global number of valid tokens); the loss call multiplies it by the mask."""
+    """Per-row weight 1 / (global number of valid tokens); the loss call multiplies it by the mask.
+    Everything stays on the mask's device: the host never reads the count, so the step stays
+    asynchronous.  (The loss call can also take the count itself: rl_loss_opts.token_count.)"""
     n = global_valid_count(mask, group)
-    w = torch.zeros(mask.shape[0], dtype=torch.float32, device=mask.device)
-    if int(n.item()) > 0:
-        w.fill_(1.0 / float(n.item()))
-    return w
+    inv = torch.where(n > 0, 1.0 / n.clamp_min(1).to(torch.float64), torch.zeros_like(n, dtype=torch.float64))
+    return inv.to(torch.float32).expand(mask.shape[0]).contiguous()
 
 
 def allreduce_gradients(dW: torch.Tensor, loss: torch.Tensor, group=None):
@@ -42,6 +42,61 @@ def allreduce_gradients(dW: torch.Tensor, loss: torch.Tensor, group=None):
         dist.all_reduce(dW, op=dist.ReduceOp.SUM, group=group)
         dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=group)
     return dW, loss
+
+
+class SlabGradientReducer:
+    """All-reduce of dW slab by slab while the backward pass is still running.
+
+    The backward pass completes dW one slab of vocabulary rows at a time and reports each slab
+    through the context's dW slab hook as soon as the launch that completes it has been enqueued.
+    `on_slab` then records an event on the compute stream, makes a side stream wait for it and
+    starts the all-reduce (sum) of exactly those rows there; the next slabs keep computing
+    meanwhile.  `finish` makes the compute stream wait for the side stream (and reduces the scalar
+    loss), after which dW holds the sum over ranks.  Slabs are reduced in the order they are
+    reported, the same on every rank, so the collectives match up.  On CPU tensors (gloo) there
+    are no streams and each slab is reduced at once; the result is the same.
+    """
+
+    def __init__(self, dW: torch.Tensor, group=None):
+        self.dW = dW
+        self.group = group
+        self.cuda = dW.is_cuda
+        self.slabs = []
+        self.world = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
+        if self.cuda:
+            self.side = torch.cuda.Stream(device=dW.device)
+            self.events = []
+
+    def begin(self):
+        """Call before the loss call of a step: the side stream must be done with the previous dW."""
+        self.slabs = []
+        if self.cuda:
+            self.side.wait_stream(torch.cuda.current_stream(self.dW.device))
+
+    def on_slab(self, slab: int, row_begin: int, row_end: int):
+        self.slabs.append((slab, row_begin, row_end))
+        if self.world <= 1:
+            return
+        rows = self.dW[row_begin:row_end]
+        if not self.cuda:
+            dist.all_reduce(rows, op=dist.ReduceOp.SUM, group=self.group)
+            return
+        k = len(self.slabs) - 1
+        if k >= len(self.events):
+            self.events.append(torch.cuda.Event())
+        ev = self.events[k]
+        ev.record(torch.cuda.current_stream(self.dW.device))
+        self.side.wait_event(ev)
+        with torch.cuda.stream(self.side):
+            dist.all_reduce(rows, op=dist.ReduceOp.SUM, group=self.group)
+
+    def finish(self, loss: torch.Tensor = None):
+        """dW (and loss, if given) hold the sums over ranks for everything enqueued after this returns."""
+        if self.cuda:
+            torch.cuda.current_stream(self.dW.device).wait_stream(self.side)
+        if loss is not None and self.world > 1:
+            dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=self.group)
+        return self.dW
 
 
 # ---------------------------------------------------------------------------------------------

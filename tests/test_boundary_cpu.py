@@ -132,6 +132,20 @@ def test_tile_schedules_cover_every_tile_once():
     for worker, mu, c0, c1, ks, kb0, kb1, kpt in u:
         work[worker] += kb1 - kb0
     assert work.max() - work.min() <= 1 and work.sum() == 66 * 8 * 296
+    # the same pass on 256 x 512 tiles (the tile counter then counts 512-wide tiles: d = 2048 -> 4, 2560 -> 5,
+    # 3584 -> 7): 264 tiles on 74 pairs are 3.57 waves; stream-K evens them out, K slices cover every k-block
+    for d_tiles, n_valid in ((4, 16896), (5, 32768), (7, 32768), (4, 300), (7, 20001)):
+        m_units = -(-n_valid // 256)
+        u = _check_schedule(n_valid, 32768, 18944, d_tiles, 2, 74, n_fastest=1, stream_k=1)
+        work = np.zeros(74, dtype=np.int64)
+        for worker, mu, c0, c1, ks, kb0, kb1, kpt in u:
+            work[worker] += kb1 - kb0
+        assert work.sum() == m_units * d_tiles * 296
+        if m_units * d_tiles >= 74 and (m_units * d_tiles) % 74:
+            assert work.max() - work.min() <= 296      # full waves of whole tiles plus one balanced share each
+            tail = work - (m_units * d_tiles // 74 - 1) * 296
+            assert tail.max() - tail.min() <= 1
+        _check_schedule(n_valid, 32768, 18944, d_tiles, 2, 74, n_fastest=1, k_split_max=4)
     # row groups: 66 row tiles with a budget of 36 tiles become two groups of 33; within a group all
     # column ranges are walked before the next group starts
     u = _check_schedule(16896, 32768, 2048, 74, 2, 74, m_group=36)

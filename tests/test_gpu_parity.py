@@ -539,19 +539,21 @@ def test_dh_k_slices(slices):
         c2.close()
 
 
-@pytest.mark.parametrize("cta_group", [2, 1])
-def test_dh_stream_k(cta_group):
+@pytest.mark.parametrize("cta_group,wide", [(2, False), (2, True), (1, False)])
+def test_dh_stream_k(cta_group, wide):
     # dH tiles balanced over the SMs by stream-K: a case with more tiles than workers and a ragged last
     # wave (10 row tiles of 256 x 8 column tiles = 80 tiles on 74 pairs; 160 on 148 single CTAs), several
     # vocabulary slabs (parts are added to what earlier slabs left) - against the oracle, against the
     # plain tile loop, and bitwise reproducible
     from paper_2512_21450_b200 import Context
     from paper_2512_21450_b200.workloads import make_workload
-    w = make_workload(1, prompts=1, L_max=640, V=1200, seed=83)
-    assert 2304 < w.n_valid <= 2560
+    # on 256 x 512 tiles the same ragged wave needs twice the rows: 20 row tiles x 4 wide tiles = 80 on 74 pairs
+    w = make_workload(1, prompts=2 if wide else 1, L_max=640, V=1200, seed=83)
+    assert (4864 < w.n_valid <= 5120) if wide else (2304 < w.n_valid <= 2560)
     c2 = Context(0)
     try:
         c2.set_cta_group(cta_group)
+        c2.set_wide_tiles(wide)
         c2.set_slab_limits(32768, 512)
         c2.set_dh_stream_k(True)
         out, _ = _check_against_oracle(c2, w)
@@ -865,3 +867,59 @@ def test_run_to_run_determinism(ctx):
     b = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, 0.2, 0.2, 0.04)
     for k in ("loss", "dH", "dW", "logp", "entropy"):
         assert torch.equal(a[k], b[k]), k
+
+
+def test_global_token_count_and_gradient_hand_over(ctx):
+    # data-parallel hooks on one GPU: (1) the token mean divided by a count handed in on the device equals
+    # the same loss with explicit per-row weights 1 / count; (2) the dW slab hook reports every row of dW
+    # exactly once, in ascending order, also with several row slabs; (3) a capped grid gives the same result
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    w = make_workload(1, prompts=1, L_max=64, d=256, V=3000, seed=905)
+    adv_seq, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+    n_global = 3 * w.n_valid + 17                      # as if two more ranks held tokens
+    cnt = torch.tensor([n_global], dtype=torch.int64, device="cuda")
+    a = ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, w.eps_low, w.eps_high,
+                                   w.beta, token_count=cnt)
+    o_adv = O.broadcast_to_tokens(O.grpo_advantages(w.rewards.cpu().numpy(), w.G), w.seq_offsets.cpu().numpy(), w.T)
+    oo = _oracle_case(w, o_adv, token_weight=np.full(w.T, 1.0 / n_global))
+    assert abs(a["loss"].item() - oo["loss"]) <= TOL_LOSS_REL * abs(oo["loss"]) + 1e-7
+    assert _rel(_np64(a["dH"]), oo["dH"]) <= TOL_GRAD_REL and _rel(_np64(a["dW"]), oo["dW"]) <= TOL_GRAD_REL
+    _assert_status_ok(ctx)
+
+    c2 = Context(0)
+    try:
+        seen = []
+        c2.set_dw_slab_hook(lambda slab, r0, r1: seen.append((slab, r0, r1)))
+        for limits in ((0, 0), (128, 512)):           # default slabs: one; small slabs: 6 column x several row slabs
+            c2.set_slab_limits(*limits)
+            seen.clear()
+            b = c2.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, w.eps_low,
+                                          w.eps_high, w.beta, token_count=cnt)
+            _assert_status_ok(c2)
+            assert [s[0] for s in seen] == list(range(len(seen))) and seen[0][1] == 0 and seen[-1][2] == w.V
+            assert all(seen[i][2] == seen[i + 1][1] for i in range(len(seen) - 1))
+            assert len(seen) == (1 if limits == (0, 0) else -(-w.V // 512))
+            assert _rel(_np64(b["dW"]), oo["dW"]) <= TOL_GRAD_REL
+        c2.set_dw_slab_hook(None)
+        c2.set_slab_limits(0, 0)
+        seen.clear()
+        c2.set_max_ctas(140)
+        b = c2.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, w.eps_low, w.eps_high,
+                                      w.beta, token_count=cnt)
+        _assert_status_ok(c2)
+        assert not seen
+        assert abs(b["loss"].item() - oo["loss"]) <= TOL_LOSS_REL * abs(oo["loss"]) + 1e-7
+        assert _rel(_np64(b["dH"]), oo["dH"]) <= TOL_GRAD_REL and _rel(_np64(b["dW"]), oo["dW"]) <= TOL_GRAD_REL
+        c2.set_max_ctas(0)
+    finally:
+        c2.close()
+
+
+@pytest.mark.parametrize("mode,cluster,nbytes,px", [(0, 2, 0, 1), (0, 8, 0, 1), (1, 4, 8192, 2), (1, 8, 16384, 4)])
+def test_cluster_exchange_probe_runs_and_returns(ctx, mode, cluster, nbytes, px):
+    # the measurement kernels for cluster data movement: a short run must come back with a time, a cluster
+    # count and a clean status word (their one mbarrier wait is bounded)
+    ms, n_clusters = ctx.selftest_cluster_exchange(mode, cluster, 50, nbytes, px)
+    _assert_status_ok(ctx)
+    assert ms > 0 and 1 <= n_clusters <= 148 // cluster

@@ -53,7 +53,19 @@ def _worker(rank, world, port, q):
                                 P["mask"][rows], 0.2, 0.28, 0.04, ent_coef=0.01, token_weight=tw.double().numpy())
     dW = torch.from_numpy(out["dW"].copy())
     loss = torch.tensor([out["loss"]], dtype=torch.float64)
+    # the same gradient handed over slab by slab, as the backward pass reports it (7 vocabulary rows per
+    # slab here, ragged last slab): must give the same sum as one all-reduce of the whole matrix
+    dW_slabs = torch.from_numpy(out["dW"].copy())
+    loss_slabs = loss.clone()
+    red = par.SlabGradientReducer(dW_slabs)
+    red.begin()
+    V = dW.shape[0]
+    for k, r0 in enumerate(range(0, V, 7)):
+        red.on_slab(k, r0, min(V, r0 + 7))
+    red.finish(loss_slabs)
+    assert [s[1] for s in red.slabs] == list(range(0, V, 7)) and red.slabs[-1][2] == V
     par.allreduce_gradients(dW, loss)
+    assert torch.equal(dW, dW_slabs) and torch.equal(loss, loss_slabs)
     if rank == 0:
         q.put((dW.numpy(), float(loss.item()), int(par.global_valid_count(mask).item())))
     else:
