@@ -22,8 +22,8 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "fused LM-head logprob+GRPO loss fwd+bwd tokens/s; % of bf16 tensor peak"
-KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad> (dlogits slab)",
-              "gemm_wide_kernel<EpiAcc,K,MN> (dH)", "gemm_wide_kernel<EpiAcc,MN,MN> (dW)"]
+KIND_NAMES = ["gemm_kernel<EpiStats,square> (forward statistics)", "gemm_kernel<EpiGrad,square> (dlogits slab)",
+              "gemm_kernel<EpiAcc,K,MN,wide> (dH)", "gemm_kernel<EpiAcc,MN,MN,wide> (dW)"]
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core kernels from one ncu
 # capture of config 1 (profiles/gemm_kernels_config1_ncu_full.md), valid only for the sources of those
@@ -31,7 +31,7 @@ KIND_NAMES = ["gemm_kernel<EpiStats> (forward statistics)", "gemm_kernel<EpiGrad
 # launch (whole vocabulary); kinds 1-3 were captured on a full slab of 18944 vocabulary columns and their
 # traffic grows with the slab's columns, so an average launch of a step (the last slab is short) carries
 # bytes x (V / 18944) / launches-per-step.
-KERNEL_SOURCES = ("epilogues.cuh", "gemm_engine.cuh", "wide_engine.cuh", "ptx.cuh")
+KERNEL_SOURCES = ("epilogues.cuh", "gemm_engine.cuh", "ptx.cuh")
 NCU_TRAFFIC = {"sources_sha256": "342babed9f7a58b43c9f7e96dcecc1767751cf83fcb8e9e8c6016b8d9b38ac31", "config": 1,
                "slab_cols": 18944,
                "bytes": {0: 1620276000 + 24176896, 1: 336381000 + 611500032, 2: 969988000 + 120208896,
@@ -300,6 +300,16 @@ def run_small_kernel_stress(args):
     ms = timed(lambda: ctx.rl_merge_logit_stats(stats, mask))
     report("merge of softmax statistics -> logp, entropy, lse", ms, 16 * T + T + 12 * T,
            "16 B of statistics + 1 B of mask read, three fp32 outputs written per row (the binding allocates the outputs)")
+    # token-level KL reward shaping: responses of 512 rows, k3 estimate, both outputs
+    n_resp = T // 512
+    off512 = torch.arange(0, T + 1, 512, dtype=torch.int32, device="cuda")
+    value = torch.rand(n_resp, generator=g, device="cuda")
+    lp = -torch.rand(T, generator=g, device="cuda")
+    rf = lp + 0.1 * torch.randn(T, generator=g, device="cuda")
+    ret = torch.empty(T, device="cuda")
+    ms = timed(lambda: ctx.rl_kl_shaped_returns(value, lp, rf, mask, off512, T, 0.04, returns=ret, want_shaped=False))
+    report("KL-shaped returns (k3, responses of 512 rows)", ms, 9 * T + 4 * T + 8 * n_resp,
+           "two fp32 inputs + 1 B of mask read, returns written per row; offsets and per-response value read")
     status, _ = ctx.last_device_status()
     assert status == 0
     print(json.dumps({"small_kernel_stress": {"rows": T, "valid_rows": N, "groups": n_groups, "group_size": G,
@@ -307,6 +317,29 @@ def run_small_kernel_stress(args):
 
 
 SEED_STRESS = 251221450 + 99
+
+
+def run_reduced_case(args):
+    """A reduced copy of the bench workload for profiler captures: same d and distributions, 37888 vocabulary
+    rows (W = 155 MB, larger than L2), two prompts (about 4.6 K valid rows), a few steps, nothing timed.
+    One step launches the forward pass and, per 18944-column slab, the dlogits, dH and dW passes."""
+    import torch
+    from paper_2512_21450_b200 import Context
+    from paper_2512_21450_b200.workloads import make_workload
+    ctx = Context(0)
+    w = make_workload(args.config, V=37888, prompts=2)
+    dH = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty(w.V, w.d, dtype=torch.float32, device="cuda")
+    loss = torch.empty(1, dtype=torch.float32, device="cuda")
+    for _ in range(args.steps):
+        _, adv_tok = ctx.rl_grpo_advantages(w.rewards, w.G, seq_offsets=w.seq_offsets, T=w.T)
+        ctx.rl_policy_loss_fwd_bwd(w.H, w.W, w.tokens, w.old_logp, w.ref_logp, adv_tok, w.mask, w.eps_low, w.eps_high,
+                                   w.beta, ent_coef=w.ent_coef, dW=dW, dH=dH, loss=loss, want_aux=False)
+    torch.cuda.synchronize()
+    status, detail = ctx.last_device_status()
+    assert status == 0, (status, detail)
+    print(json.dumps({"reduced_case": workload_label(args.config, w), "steps": args.steps, "loss": loss.item(),
+                      "launches": ctx.launch_count()}))
 
 
 def run_cluster_probe(args):
@@ -436,6 +469,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cluster-probe", action="store_true",
                     help="instead of the benchmark line, time data movement between the CTAs of a cluster")
+    ap.add_argument("--reduced-case", action="store_true",
+                    help="instead of the benchmark line, run --steps steps of a reduced workload (for profiler captures)")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short runs of the other large workloads (configs 1-4 besides --config)")
     ap.add_argument("--other-steps", type=int, default=8)
@@ -459,6 +494,9 @@ def main():
         return
     if args.cluster_probe:
         run_cluster_probe(args)
+        return
+    if args.reduced_case:
+        run_reduced_case(args)
         return
 
 
