@@ -25,17 +25,14 @@ METRIC = "fused LM-head logprob+GRPO loss fwd+bwd tokens/s; % of bf16 tensor pea
 KIND_NAMES = ["gemm_kernel<EpiStats,square> (forward statistics)", "gemm_kernel<EpiGrad,square> (dlogits slab)",
               "gemm_kernel<EpiAcc,K,MN,wide> (dH)", "gemm_kernel<EpiAcc,MN,MN,wide> (dW)"]
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core kernels from one ncu
-# capture of config 1 (profiles/gemm_kernels_config1_ncu_full.md), valid only for the sources of those
-# kernels (main loop, epilogues, PTX wrappers) whose hash is recorded with it.  Kind 0 is the forward
-# launch (whole vocabulary); kinds 1-3 were captured on a full slab of 18944 vocabulary columns and their
-# traffic grows with the slab's columns, so an average launch of a step (the last slab is short) carries
-# bytes x (V / 18944) / launches-per-step.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core kernels from one ncu capture
+# of a whole config-1 step (profiles/gemm_kernel_dram_config1.md; these three metrics take one pass), valid only
+# for the sources of those kernels (main loop, epilogues, PTX wrappers) whose hash is recorded with it.  Bytes
+# per AVERAGE launch of a step: kind 0 is the one forward launch, kinds 1-3 the mean over the nine vocabulary
+# slabs (eight of 18944 columns and a last one of 384).
 KERNEL_SOURCES = ("epilogues.cuh", "gemm_engine.cuh", "ptx.cuh")
-NCU_TRAFFIC = {"sources_sha256": "342babed9f7a58b43c9f7e96dcecc1767751cf83fcb8e9e8c6016b8d9b38ac31", "config": 1,
-               "slab_cols": 18944,
-               "bytes": {0: 1620276000 + 24176896, 1: 336381000 + 611500032, 2: 969988000 + 120208896,
-                         3: 934376000 + 120284928}}
+NCU_TRAFFIC = {"sources_sha256": "1b2a79199ac50c98db470e8abd69b8f5c99f0d92fcbd0feb2bf7b9d49bd41a65", "config": 1,
+               "bytes_per_avg_launch": {0: 2221588440, 1: 861360776, 2: 1107407029, 3: 973881151}}
 
 
 def sources_hash():
@@ -628,9 +625,7 @@ def main():
     achieved = flops_launch / (avg_launch_ms / 1e3) / 1e12
     traffic = None
     if NCU_TRAFFIC["sources_sha256"] == sources_hash() and NCU_TRAFFIC["config"] == args.config:
-        traffic = float(NCU_TRAFFIC["bytes"][dom])
-        if dom != 0:
-            traffic *= (w.V / NCU_TRAFFIC["slab_cols"]) / launches_dom
+        traffic = float(NCU_TRAFFIC["bytes_per_avg_launch"][dom])
     # which measured peak the kernel is held to: the burst figure when the timed region is short (the board
     # has not settled at its power limit yet), the sustained one for a region of seconds; both are printed
     timed_s = ms / 1e3
