@@ -360,7 +360,7 @@ __global__ void __launch_bounds__(256) broadcast_adv_kernel(const float* __restr
 // One warp per response: it walks the response's rows from the end in 32-row chunks aligned to
 // 128 bytes, loads kShapeChunks chunks at a time and runs a suffix scan of the linear maps
 // x -> v + g x (valid row: g = gamma, v = r_t; masked row: the identity) with shuffles, carrying the
-// return of the first valid token of the chunks already done.  Arithmetic in double.
+// return of the first valid token of the chunks already done.  Per-token terms in fp32, sums in double.
 constexpr int kShapeChunks = 4;
 
 __global__ void __launch_bounds__(256) kl_shaped_returns_kernel(const float* __restrict__ seq_value,
@@ -393,8 +393,11 @@ __global__ void __launch_bounds__(256) kl_shaped_returns_kernel(const float* __r
           if (kind == 2) {
             kl = (double)kl_tok[t];
           } else {
-            const double lp = (double)logp[t], rf = (double)ref_logp[t];
-            kl = kind == 0 ? lp - rf : exp(rf - lp) - (rf - lp) - 1.0;
+            // the difference of two fp32 values is exact in double; the exponential itself is taken in fp32
+            // (expm1f keeps small log-ratios accurate to an ulp), the sums below run in double
+            const double delta = (double)ref_logp[t] - (double)logp[t];
+            const float df = (float)delta;
+            kl = kind == 0 ? -delta : (double)expm1f(df) - delta;
           }
         }
         r[j] = -(double)beta * kl;
@@ -407,11 +410,20 @@ __global__ void __launch_bounds__(256) kl_shaped_returns_kernel(const float* __r
           terminal_done = true;
         }
         double g = valid[j] ? (double)gamma : 1.0, v = valid[j] ? r[j] : 0.0;
+        if (gamma == 1.f) {
+          // no discount: a plain suffix sum
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const double g2 = __shfl_down_sync(0xffffffffu, g, o);
-          const double v2 = __shfl_down_sync(0xffffffffu, v, o);
-          if (lane + o < 32) { v = fma(g, v2, v); g *= g2; }
+          for (int o = 1; o < 32; o <<= 1) {
+            const double v2 = __shfl_down_sync(0xffffffffu, v, o);
+            if (lane + o < 32) v += v2;
+          }
+        } else {
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const double g2 = __shfl_down_sync(0xffffffffu, g, o);
+            const double v2 = __shfl_down_sync(0xffffffffu, v, o);
+            if (lane + o < 32) { v = fma(g, v2, v); g *= g2; }
+          }
         }
         const double out = fma(g, carry, v);
         carry = __shfl_sync(0xffffffffu, out, 0);
