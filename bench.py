@@ -471,6 +471,9 @@ def main():
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short runs of the other large workloads (configs 1-4 besides --config)")
     ap.add_argument("--other-steps", type=int, default=8)
+    ap.add_argument("--dp-path-on-one-gpu", action="store_true",
+                    help="run the data-parallel code path (global count, slab-wise all-reduce on a side stream, capped "
+                         "grid) in a process group of one rank, to exercise it where only one GPU is at hand")
     ap.add_argument("--dp-free-sms", type=int, default=4,
                     help="with more than one GPU: SMs the persistent grids leave to the all-reduce kernels")
     ap.add_argument("--compare-library", action="store_true",
@@ -511,7 +514,13 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    if world > 1:
+    dp_path = world > 1 or args.dp_path_on_one_gpu
+    if dp_path:
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29533")
+            os.environ.setdefault("RANK", "0")
+            os.environ.setdefault("WORLD_SIZE", "1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
     peaks = measured_peaks()
@@ -520,12 +529,12 @@ def main():
     w = make_workload(args.config, device=dev, seed=SEED_BASE + args.config + 1000 * rank)
     ctx = Context(local)
     reducer, token_count = None, None
-    if world > 1:
+    if dp_path:
         # data parallel: the token mean is over all ranks' valid tokens (count summed on the device, never
         # read by the host) and dW is all-reduced slab by slab on a side stream while the backward pass of
         # the remaining slabs runs; a few SMs are left to the collective's kernels
         token_count = par.global_valid_count(w.mask)
-        reducer = par.SlabGradientReducer(torch.empty(0, device=dev))
+        reducer = par.SlabGradientReducer(torch.empty(0, device=dev), single_rank_too=True)
         ctx.set_dw_slab_hook(reducer.on_slab)
         if args.dp_free_sms > 0:
             ctx.set_max_ctas(torch.cuda.get_device_properties(dev).multi_processor_count - args.dp_free_sms)
@@ -599,7 +608,7 @@ def main():
 
     # ---- the other large workloads, a few steps each (one GPU only): the record carries all four
     other = []
-    if world == 1 and not args.no_other_configs:
+    if world == 1 and not dp_path and not args.no_other_configs:
         del outs, hH
         for cfg_id in (1, 2, 3, 4):
             if cfg_id == args.config:
@@ -669,7 +678,7 @@ def main():
         "config": {"workload": workload_label(args.config, w),
                    "l2": "inputs larger than L2 (W alone is %.0f MB; L2 126 MB)" % (w.V * w.d * 2 / 1e6),
                    "parallelism": (f"dp{world}: prompts sharded, dW all-reduced slab by slab under the backward pass"
-                                   if world > 1 else "single GPU"),
+                                   if dp_path else "single GPU"),
                    "masked_rows": "skipped (row compaction)",
                    "row_tiles": "%d valid rows = %d tiles of 256 rows%s" % (
                        N, (N + 255) // 256, " exactly (no ragged row tile at this seed)" if N % 256 == 0 else
@@ -698,7 +707,7 @@ def main():
                                "kind": "oracle", "sample": f"first {n} valid rows of the same workload, full d and V, "
                                                            f"float64 numpy, one pass ({dt:.1f} s)"}
     print(json.dumps(out))
-    if world > 1:
+    if dp_path:
         dist.destroy_process_group()
 
 

@@ -57,9 +57,10 @@ class SlabGradientReducer:
     are no streams and each slab is reduced at once; the result is the same.
     """
 
-    def __init__(self, dW: torch.Tensor, group=None):
+    def __init__(self, dW: torch.Tensor, group=None, single_rank_too: bool = False):
         self.dW = dW
         self.group = group
+        self.min_world = 1 if single_rank_too else 2   # single_rank_too: run the collectives even in a group of one
         self.cuda = dW.is_cuda
         self.slabs = []
         self.world = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
@@ -75,7 +76,7 @@ class SlabGradientReducer:
 
     def on_slab(self, slab: int, row_begin: int, row_end: int):
         self.slabs.append((slab, row_begin, row_end))
-        if self.world <= 1:
+        if self.world < self.min_world:
             return
         rows = self.dW[row_begin:row_end]
         if not self.cuda:
@@ -94,7 +95,7 @@ class SlabGradientReducer:
         """dW (and loss, if given) hold the sums over ranks for everything enqueued after this returns."""
         if self.cuda:
             torch.cuda.current_stream(self.dW.device).wait_stream(self.side)
-        if loss is not None and self.world > 1:
+        if loss is not None and self.world >= self.min_world:
             dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=self.group)
         return self.dW
 
