@@ -414,8 +414,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       constexpr uint64_t b_hi = B_MN ? make_smem_desc_hi(8192, 1024) : make_smem_desc_hi(16, 1024);
       constexpr uint32_t a_kstep = A_MN ? 2048 : 32;
       constexpr uint32_t b_kstep = B_MN ? 2048 : 32;
+      // The issuing thread is a serial chain - wait for a stage, fence, four (or eight) UMMAs, commit - that has
+      // to stay shorter than the tensor work it hands out (512 clocks per k-slice for square tiles).  Two things
+      // keep it short: the barrier of the NEXT stage is polled before the UMMAs of this one are issued, so the
+      // latency of that poll hides behind them (`ready` carries its answer into the next round, also across tiles);
+      // and descriptors, barrier addresses and stage offsets are kept as running 32-bit words instead of being
+      // rebuilt from the stage index.
+      constexpr uint32_t a_hi32 = uint32_t(a_hi >> 32), b_hi32 = uint32_t(b_hi >> 32);
+      constexpr uint32_t a_lo_const = uint32_t(a_hi), b_lo_const = uint32_t(b_hi);   // bits [16, 30): leading offset
+      const uint32_t ring_lo = (tiles_base & 0x3FFFFu) >> 4;
       int stage = 0;
       uint32_t phase = 0;
+      uint32_t ready = 0;   // 1: the full barrier of `stage` is already known to have completed at `phase`
       uint32_t t = 0;   // tiles issued so far
       bool ok = true;
       if (run && ex.k_blocks > 0) {
@@ -440,28 +450,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               const uint32_t d_tmem = tmem_base + (MODE == kTileDual ? prod : a) * BN;
               const int lo = prod ? 0 : kb0, hi = prod ? k2_blocks : kb1;
               for (int kb = lo; kb < hi; ++kb) {
-                if (!mbar_wait_bounded_cluster(smem_u32(&bar_full[stage]), phase, abort_p)) {
+                if (!ready && !mbar_wait_bounded_cluster(smem_u32(&bar_full[stage]), phase, abort_p)) {
                   latch_status(status, kStatusTimeout, (3 << 28) | (blockIdx.x << 8) | stage);
                   ok = false;
                   break;
                 }
+                // poll the next ring position now; the answer is looked at after this stage's UMMAs are out
+                const int nstage = stage + 1 == kStages ? 0 : stage + 1;
+                const uint32_t nphase = stage + 1 == kStages ? phase ^ 1u : phase;
+                const uint32_t peek = mbar_try_wait_cluster(smem_u32(&bar_full[nstage]), nphase);
                 tc_fence_after();
-                const uint32_t a_src = tiles_base + stage * Cfg::kStageBytes;
-                const uint32_t b_src = a_src + kAStageBytes;
+                const uint32_t a_lo = a_lo_const | (ring_lo + uint32_t(stage) * (Cfg::kStageBytes >> 4));
+                const uint32_t b_lo = b_lo_const | (ring_lo + uint32_t(stage) * (Cfg::kStageBytes >> 4) + (kAStageBytes >> 4));
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k) {
-                  const uint64_t da = smem_desc(a_hi, a_src + k * a_kstep);
                   const uint32_t acc = (kb > lo || k > 0) ? 1u : 0u;
 #pragma unroll
-                  for (int s = 0; s < Cfg::kBBoxes; ++s) {
-                    const uint64_t db = smem_desc(b_hi, b_src + s * Cfg::kBBytes + k * b_kstep);
-                    if (CG == 2) umma_bf16_pair(d_tmem + s * BN, da, db, idesc, acc);
-                    else         umma_bf16(d_tmem + s * BN, da, db, idesc, acc);
-                  }
+                  for (int s = 0; s < Cfg::kBBoxes; ++s)
+                    umma_bf16_words<CG>(d_tmem + s * BN, a_lo + k * (a_kstep >> 4), a_hi32,
+                                        b_lo + (s * Cfg::kBBytes + k * b_kstep) / 16, b_hi32, idesc, acc);
                 }
                 if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_empty[stage]), 3);
                 else         umma_commit(smem_u32(&bar_empty[stage]));
-                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                stage = nstage;
+                phase = nphase;
+                ready = peek;
               }
             }
             if (ok) {
