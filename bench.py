@@ -28,11 +28,11 @@ KIND_NAMES = ["gemm_kernel<EpiStats,square> (forward statistics)", "gemm_kernel<
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core kernels from one ncu capture
 # of a whole config-1 step (profiles/gemm_kernel_dram_config1.md; these three metrics take one pass), valid only
 # for the sources of those kernels (main loop, epilogues, PTX wrappers) whose hash is recorded with it.  Bytes
-# per AVERAGE launch of a step: kind 0 is the one forward launch, kinds 1-3 the mean over the nine vocabulary
-# slabs (eight of 18944 columns and a last one of 384).
+# per AVERAGE launch of a step: kind 0 is the one forward launch, kinds 1-3 the mean over the five vocabulary
+# slabs (four of 37888 columns and a last one of 384).
 KERNEL_SOURCES = ("epilogues.cuh", "gemm_engine.cuh", "ptx.cuh")
 NCU_TRAFFIC = {"sources_sha256": "e3dfbdc11587c0b38a925f3bcbdef8d61f6a8d4ea1fabf947f80527283617a60", "config": 1,
-               "bytes_per_avg_launch": {0: 2261708624, 1: 840471042, 2: 1102467203, 3: 960852862}}
+               "bytes_per_avg_launch": {0: 2094349000, 1: 1566771400, 2: 2241300600, 3: 2323983400}}
 
 
 def sources_hash():
@@ -319,7 +319,7 @@ SEED_STRESS = 251221450 + 99
 def run_reduced_case(args):
     """A reduced copy of the bench workload for profiler captures: same d and distributions, 37888 vocabulary
     rows (W = 155 MB, larger than L2), two prompts (about 4.6 K valid rows), a few steps, nothing timed.
-    One step launches the forward pass and, per 18944-column slab, the dlogits, dH and dW passes."""
+    One step launches the forward pass and, per 37888-column slab, the dlogits, dH and dW passes."""
     import torch
     from paper_2512_21450_b200 import Context
     from paper_2512_21450_b200.workloads import make_workload
@@ -540,7 +540,7 @@ def main():
             ctx.set_max_ctas(torch.cuda.get_device_properties(dev).multi_processor_count - args.dp_free_sms)
 
     r = measure_config(ctx, w, args.steps, args.warmup, dev, world, reducer, token_count,
-                       profile_steps=max(1, min(args.steps, 5)))
+                       profile_steps=max(1, min(args.steps, 20)))
     ms, dH, dW, loss = r["ms"], r["dH"], r["dW"], r["loss"]
     fence = r["fence"]
     device_loss = float(loss.item())

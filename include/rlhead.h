@@ -70,9 +70,11 @@ rl_status rl_workspace_bytes(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, size_
 rl_status rl_workspace_bytes_kl(rl_ctx* ctx, int64_t T, int64_t d, int64_t V, int64_t d_ref, size_t* bytes);
 /* Size of the slab the backward pass works in: at most max_rows token rows x max_cols vocabulary
  * columns of the gradient with respect to the logits exist at a time (bf16, in the workspace).
- * max_rows a multiple of 128, max_cols a multiple of 256; 0 restores a default (32768 x 18944,
- * chosen so that the tile counts of the dlogits and dW passes are multiples of the 74 SM pairs
- * for d = 2048, 2560 and 3584).  Changes what rl_workspace_bytes() returns: call it first. */
+ * max_rows a multiple of 128, max_cols a multiple of 256, max_rows * max_cols at most 2^31; 0 restores a
+ * default (32768 x 37888: 2.5 GB of slab at most, chosen so that the tile counts of the dlogits and dW
+ * passes are multiples of the 74 SM pairs for d = 2048, 2560 and 3584; half as many columns cost 0.5-1.7 %
+ * of a step in launch ramps and accumulator traffic).  Changes what rl_workspace_bytes() returns: call it
+ * first. */
 rl_status rl_set_slab_limits(rl_ctx* ctx, int max_rows, int max_cols);
 /* Tile shape of the tensor-core passes: 1 = one CTA per 128x256 output tile, 2 = CTA pairs
  * (clusters of two SMs, tcgen05 cta_group::2) on 256x256 tiles, which halves the shared-memory

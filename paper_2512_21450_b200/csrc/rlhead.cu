@@ -60,7 +60,7 @@ namespace {
 constexpr long long kRowGroupBytes = 36ll << 20;   // A panels walked together by the rows-first passes (L2 is 126 MB)
 constexpr int kSlabRowsMax = 32768;        // rows of one gradient slab
 constexpr int kDhSplitMax = 4;             // most K slices (separate fp32 accumulators) of the dH pass
-constexpr int kSlabColsMax = 148 * 128;    // vocabulary columns of one gradient slab (74 tiles of 256)
+constexpr int kSlabColsMax = 148 * 256;    // vocabulary columns of one gradient slab (148 tiles of 256: two per SM pair)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -87,7 +87,7 @@ def test_full_size_sampled(cfg_id, n_rows, n_cols):
         tok_valid = w.tokens.cpu().numpy()[valid]
         freq = np.argsort(np.bincount(tok_valid, minlength=w.V))[-8:]
         sel = np.unique(np.concatenate([rng.choice(w.V, size=n_cols, replace=False), freq,
-                                        np.arange(w.V - 4, w.V), np.array([0, 255, 256, 18943, 18944])]))
+                                        np.arange(w.V - 4, w.V), np.array([0, 255, 256, 18943, 18944, 37887, 37888])]))
         # the loss call does not return lse; the forward-only call does
         _, _, lse_t = ctx.rl_token_logprobs(w.H, w.W, w.tokens, w.mask)
         lse = _np64(lse_t)[valid]

@@ -441,7 +441,7 @@ def test_clip_exercised_and_peaked_rows(ctx):
     _check_against_oracle(ctx, w)
 
 
-@pytest.mark.parametrize("V,L_max", [(4096, 13), (4000, 16), (4100, 16), (300, 9), (18944 + 256 + 40, 11)])
+@pytest.mark.parametrize("V,L_max", [(4096, 13), (4000, 16), (4100, 16), (300, 9), (37888 + 256 + 40, 11)])
 def test_ragged_shapes(ctx, V, L_max):
     # rows not a multiple of 128, vocabulary not a multiple of 256 / 32, more than one vocabulary slab
     from paper_2512_21450_b200.workloads import make_workload

@@ -33,7 +33,7 @@ def test_random_shapes_and_options(seed):
                           d=d, V=V, seed=int(rng.integers(1 << 30)), sigma_old=float(rng.choice([0.05, 0.3])))
         opts = dict(cta_group=int(rng.choice([1, 2])), wide=int(rng.integers(0, 2)), stream_k=int(rng.integers(0, 2)),
                     k_slices=int(rng.choice([1, 1, 2, 3])), group=int(rng.choice([0, 1 << 16, 1 << 19, 36 << 20])),
-                    slab=(int(rng.choice([128, 256, 1024, 32768])), int(rng.choice([256, 512, 2048, 18944]))),
+                    slab=(int(rng.choice([128, 256, 1024, 32768])), int(rng.choice([256, 512, 2048, 18944, 37888]))),
                     dH_fp32=bool(rng.integers(0, 2)))
         c = Context(0)
         try:
