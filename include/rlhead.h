@@ -451,7 +451,9 @@ rl_status rl_selftest_cluster_exchange(rl_ctx* ctx, int mode, int cluster_size, 
 
 /* Host-only view of how a tensor-core pass distributes its work (no GPU is touched; the paper has
  * no counterpart).  For a pass over n_valid rows (at most rows_cap), K extent k_len, n_tiles column
- * tiles walked n_range at a time (0: chosen as the forward pass does), with the ordering options
+ * tiles walked n_range at a time (0: split that fills the SMs, or 8 with plenty of work; -h with 1 <= h < 100:
+ * chosen in [1, h] as the gradient-of-the-logits pass does; -100 - h: chosen in [8, h] when there is plenty of
+ * work, else as 0), with the ordering options
  * of the library (n_fastest, row groups of m_group row tiles, stream-K, K slices) on n_workers
  * workers of cta_group CTAs each, writes one record of eight int32 per work unit, worker by worker
  * in the order the worker walks them: {worker, row tile, first column tile, end column tile,

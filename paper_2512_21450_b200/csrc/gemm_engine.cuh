@@ -3,7 +3,8 @@
 // 256-column fp32 accumulators of tensor memory are used.
 //
 //   warp 0      : TMA producer (one lane) - streams A and B k-slices (64 elements of K) into a
-//                 shared-memory ring, 128-byte swizzled.
+//                 shared-memory ring, 128-byte swizzled; a ring stage holds one k-slice, or two for
+//                 the 256-column pair tiles (see StageCfg::kKSub).
 //   warp 1      : allocates tensor memory; one lane issues tcgen05.mma.
 //   warps 2..5  : epilogue - each warp owns the 32 tensor-memory lanes (tile rows) that its
 //                 rank modulo 4 may read, pulls the accumulator out in 32-column chunks and
@@ -68,9 +69,14 @@ template <int CG, int MODE, int kStaging>
 struct StageCfg {
   static constexpr int kBRows = BN / CG;                    // B rows (output columns) of one box staged per CTA
   static constexpr int kBBytes = kBRows * BK * 2;
-  static constexpr int kBBoxes = MODE == kTileWide ? 2 : 1; // B boxes per stage
-  static constexpr int kStageBytes = kAStageBytes + kBBoxes * kBBytes;
-  static constexpr int kStages = (kTileSmemBytes - kStaging) / kStageBytes;   // 4 (CG = 1); 7 or 6 (pairs); 4 (wide)
+  static constexpr int kBBoxes = MODE == kTileWide ? 2 : 1; // B boxes per k-slice
+  static constexpr int kSliceBytes = kAStageBytes + kBBoxes * kBBytes;   // one k-slice of 64: A box, then the B boxes
+  // k-slices per ring stage.  The MMA issuer is one thread whose chain per stage - wait, fence, UMMAs, commit - has
+  // to stay shorter than the tensor work it hands out; a 256-column pair tile has only 512 tensor clocks per
+  // k-slice, so its stages hold two k-slices (eight UMMAs per barrier round trip, as a wide tile has).
+  static constexpr int kKSub = (CG == 2 && MODE != kTileWide) ? 2 : 1;
+  static constexpr int kStageBytes = kKSub * kSliceBytes;
+  static constexpr int kStages = (kTileSmemBytes - kStaging) / kStageBytes;   // 4 (CG = 1); 3 (square pairs); 4 (wide)
   static constexpr int kRingBytes = kStages * kStageBytes;
   static constexpr uint32_t kTxBytes = uint32_t(kStageBytes) * CG;  // bytes counted on the issuing CTA's barrier
 };
@@ -98,6 +104,9 @@ struct GemmShape {
   int k_cap, k_dyn, k_dyn_off;
   int n_tiles;      // number of 256-wide column tiles
   int n_range;      // consecutive column tiles per work unit; 0 = choose so that units fill the SMs
+  // With n_range == 0 and n_range_hi > 0 the range length is chosen in [n_range_lo, n_range_hi] by choose_range():
+  // always (n_range_always != 0) or only when there is plenty of work (otherwise the split that fills the SMs).
+  int n_range_lo, n_range_hi, n_range_always;
   int skip_if_k0;   // nothing to do at all when K is empty (otherwise the epilogue sees zeros)
   int n_fastest;    // 1: consecutive units walk the column ranges of one row tile first
   // Row slabs of the backward pass: when slab_cap > 0 the valid rows are cut into
@@ -139,6 +148,23 @@ __host__ __device__ inline int choose_split(int m_units, int n_tiles, int n_work
     long waves = (units + n_workers - 1) / n_workers;
     long cost = waves * ((n_tiles + s - 1) / s);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+// Column tiles per work unit, in [lo, hi], for a pass whose units all cost the same per tile: minimises the time of
+// the busiest worker, estimated as (waves of units) x (range length), with 5 % of a tile charged per unit for what
+// the roles do between units (unit coordinates on the MMA issuer's serial chain, per-row loads of the epilogue).
+// Measured on the gradient-of-the-logits pass (148 column tiles, 66 row tiles, 74 workers): ranges of 1 / 2 / 4 / 8
+// tiles take 8.02 / 7.86 / 7.80 / 7.90 ms.
+__host__ __device__ inline int choose_range(int m_units, int n_tiles, int n_workers, int lo, int hi) {
+  int best = lo;
+  long best_cost = -1;
+  for (int nr = lo; nr <= hi; ++nr) {
+    const long ranges = (n_tiles + nr - 1) / nr;
+    const long waves = ((long)m_units * ranges + n_workers - 1) / n_workers;
+    const long cost = waves * (100 * nr + 5);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = nr; }
   }
   return best;
 }
@@ -189,9 +215,12 @@ __host__ __device__ inline GemmExtents gemm_extents(const GemmShape& sh, int n_v
   const int k_len = sh.k_dyn ? k : sh.k_cap;
   e.m_units = (e.m_rows + BM * cg - 1) / (BM * cg);
   e.k_blocks = (k_len + BK - 1) / BK;
+  const bool plenty = (long)e.m_units * ((sh.n_tiles + kFwdRange - 1) / kFwdRange) >= 4L * n_workers;
   if (sh.n_range > 0) {
     e.n_range = sh.n_range;
-  } else if ((long)e.m_units * ((sh.n_tiles + kFwdRange - 1) / kFwdRange) >= 4L * n_workers) {
+  } else if (sh.n_range_hi > 0 && (sh.n_range_always || plenty)) {
+    e.n_range = choose_range(e.m_units, sh.n_tiles, n_workers, sh.n_range_lo > 0 ? sh.n_range_lo : 1, sh.n_range_hi);
+  } else if (plenty) {
     // plenty of work: short fixed ranges, walked rows-first, keep every worker within a few
     // column tiles of the others, so the B operand is fetched from DRAM about once
     e.n_range = kFwdRange;
@@ -358,37 +387,42 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const CUtensorMap* ta = prod ? &tmA2 : &tmA;
             const CUtensorMap* tb = prod ? &tmB2 : &tmB;
             const int lo = prod ? 0 : kb0, hi = prod ? k2_blocks : kb1;
-            for (int kb = lo; kb < hi; ++kb) {
+            for (int kb = lo; kb < hi; kb += Cfg::kKSub) {
               if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p)) {
                 latch_status(status, kStatusTimeout, (1 << 28) | (blockIdx.x << 8) | stage);
                 ok = false;
                 break;
               }
               const uint32_t full_local = smem_u32(&bar_full[stage]);
-              const uint32_t a_dst = tiles_base + stage * Cfg::kStageBytes;
-              const uint32_t b_dst = a_dst + kAStageBytes;
-              const int a_k = (prod ? 0 : sh.a_k_off) + kb * BK;
-              const int b_k = (prod ? 0 : sh.b_k_off + (sh.b_k_slab ? ex.slab_off : 0)) + kb * BK;
               // the even CTA's barrier counts the bytes of both CTAs' copies
               if (CG == 1 || rank == 0) mbar_arrive_expect_tx(full_local, Cfg::kTxBytes);
               const uint32_t full = CG == 2 ? mapa_cluster(full_local, 0) : full_local;
-              if (CG == 1) {
-                if (A_MN) tma_load_3d(a_dst, ta, full, 0, a_k, a_row / 64);
-                else      tma_load_2d(a_dst, ta, full, a_k, a_row);
-              } else {
-                if (A_MN) tma_load_3d_pair(a_dst, ta, full, 0, a_k, a_row / 64);
-                else      tma_load_2d_pair(a_dst, ta, full, a_k, a_row);
-              }
+              // A stage always receives all its k-slices: one that lies past the K range of the unit is loaded all
+              // the same (past the tensor it reads as zeros) and the issuer leaves it out.
 #pragma unroll
-              for (int s = 0; s < Cfg::kBBoxes; ++s) {
-                const int b_row = sh.b_mn_off + (n * Cfg::kBBoxes + s) * BN + (int)rank * Cfg::kBRows;
-                const uint32_t dst = b_dst + s * Cfg::kBBytes;
+              for (int j = 0; j < Cfg::kKSub; ++j) {
+                const uint32_t a_dst = tiles_base + stage * Cfg::kStageBytes + j * Cfg::kSliceBytes;
+                const uint32_t b_dst = a_dst + kAStageBytes;
+                const int a_k = (prod ? 0 : sh.a_k_off) + (kb + j) * BK;
+                const int b_k = (prod ? 0 : sh.b_k_off + (sh.b_k_slab ? ex.slab_off : 0)) + (kb + j) * BK;
                 if (CG == 1) {
-                  if (B_MN) tma_load_3d(dst, tb, full, 0, b_k, b_row / 64);
-                  else      tma_load_2d(dst, tb, full, b_k, b_row);
+                  if (A_MN) tma_load_3d(a_dst, ta, full, 0, a_k, a_row / 64);
+                  else      tma_load_2d(a_dst, ta, full, a_k, a_row);
                 } else {
-                  if (B_MN) tma_load_3d_pair(dst, tb, full, 0, b_k, b_row / 64);
-                  else      tma_load_2d_pair(dst, tb, full, b_k, b_row);
+                  if (A_MN) tma_load_3d_pair(a_dst, ta, full, 0, a_k, a_row / 64);
+                  else      tma_load_2d_pair(a_dst, ta, full, a_k, a_row);
+                }
+#pragma unroll
+                for (int s = 0; s < Cfg::kBBoxes; ++s) {
+                  const int b_row = sh.b_mn_off + (n * Cfg::kBBoxes + s) * BN + (int)rank * Cfg::kBRows;
+                  const uint32_t dst = b_dst + s * Cfg::kBBytes;
+                  if (CG == 1) {
+                    if (B_MN) tma_load_3d(dst, tb, full, 0, b_k, b_row / 64);
+                    else      tma_load_2d(dst, tb, full, b_k, b_row);
+                  } else {
+                    if (B_MN) tma_load_3d_pair(dst, tb, full, 0, b_k, b_row / 64);
+                    else      tma_load_2d_pair(dst, tb, full, b_k, b_row);
+                  }
                 }
               }
               if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -414,9 +448,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       constexpr uint64_t b_hi = B_MN ? make_smem_desc_hi(8192, 1024) : make_smem_desc_hi(16, 1024);
       constexpr uint32_t a_kstep = A_MN ? 2048 : 32;
       constexpr uint32_t b_kstep = B_MN ? 2048 : 32;
-      // The issuing thread is a serial chain - wait for a stage, fence, four (or eight) UMMAs, commit - that has
-      // to stay shorter than the tensor work it hands out (512 clocks per k-slice for square tiles).  Two things
-      // keep it short: the barrier of the NEXT stage is polled before the UMMAs of this one are issued, so the
+      // The issuing thread is a serial chain - wait for a stage, fence, eight UMMAs (four on single-CTA tiles), commit -
+      // that has to stay shorter than the tensor work it hands out (1024 clocks per stage of a pair tile).  Besides
+      // the two k-slices per stage of the 256-column tiles, two things keep it short: the barrier of the NEXT stage is polled before the UMMAs of this one are issued, so the
       // latency of that poll hides behind them (`ready` carries its answer into the next round, also across tiles);
       // and descriptors, barrier addresses and stage offsets are kept as running 32-bit words instead of being
       // rebuilt from the stage index.
@@ -449,7 +483,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             for (int prod = 0; prod < kProducts && ok; ++prod) {
               const uint32_t d_tmem = tmem_base + (MODE == kTileDual ? prod : a) * BN;
               const int lo = prod ? 0 : kb0, hi = prod ? k2_blocks : kb1;
-              for (int kb = lo; kb < hi; ++kb) {
+              for (int kb = lo; kb < hi; kb += Cfg::kKSub) {
                 if (!ready && !mbar_wait_bounded_cluster(smem_u32(&bar_full[stage]), phase, abort_p)) {
                   latch_status(status, kStatusTimeout, (3 << 28) | (blockIdx.x << 8) | stage);
                   ok = false;
@@ -463,12 +497,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const uint32_t a_lo = a_lo_const | (ring_lo + uint32_t(stage) * (Cfg::kStageBytes >> 4));
                 const uint32_t b_lo = b_lo_const | (ring_lo + uint32_t(stage) * (Cfg::kStageBytes >> 4) + (kAStageBytes >> 4));
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k) {
-                  const uint32_t acc = (kb > lo || k > 0) ? 1u : 0u;
+                for (int j = 0; j < Cfg::kKSub; ++j) {
+                  if (j > 0 && kb + j >= hi) break;   // a k-slice past the unit's K range was loaded but is not used
 #pragma unroll
-                  for (int s = 0; s < Cfg::kBBoxes; ++s)
-                    umma_bf16_words<CG>(d_tmem + s * BN, a_lo + k * (a_kstep >> 4), a_hi32,
-                                        b_lo + (s * Cfg::kBBytes + k * b_kstep) / 16, b_hi32, idesc, acc);
+                  for (int k = 0; k < BK / 16; ++k) {
+                    const uint32_t acc = (kb > lo || j > 0 || k > 0) ? 1u : 0u;
+#pragma unroll
+                    for (int s = 0; s < Cfg::kBBoxes; ++s)
+                      umma_bf16_words<CG>(d_tmem + s * BN, a_lo + (j * Cfg::kSliceBytes + k * a_kstep) / 16, a_hi32,
+                                          b_lo + (j * Cfg::kSliceBytes + s * Cfg::kBBytes + k * b_kstep) / 16, b_hi32,
+                                          idesc, acc);
+                  }
                 }
                 if (CG == 2) umma_commit_pair_mcast(smem_u32(&bar_empty[stage]), 3);
                 else         umma_commit(smem_u32(&bar_empty[stage]));

@@ -1022,7 +1022,7 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
         sh.m_rows_cap = rows_cap; sh.m_dyn = 1; sh.slab_cap = L.Ts; sh.slab_index = r;
         sh.k_cap = (int)d;
         sh.n_tiles = (cols + BN - 1) / BN;
-        sh.n_range = 1;
+        sh.n_range = 0; sh.n_range_lo = 1; sh.n_range_hi = kFwdRange; sh.n_range_always = 1;   // chosen on the device
         sh.a_mn_slab = 1;
         sh.b_mn_off = vocab_base;
         sh.m_group = row_group_tiles(c, d + (o.kl_full ? o.d_ref : 0));
@@ -1414,7 +1414,13 @@ rl_status rl_debug_schedule(int64_t n_valid, int64_t rows_cap, int64_t k_len, in
   sh.m_dyn = 1;
   sh.k_cap = (int)k_len;
   sh.n_tiles = (int)n_tiles;
-  sh.n_range = n_range;
+  if (n_range >= 0) {
+    sh.n_range = n_range;
+  } else if (n_range > -100) {   // as the gradient-of-the-logits pass: always chosen in [1, -n_range]
+    sh.n_range_lo = 1; sh.n_range_hi = -n_range; sh.n_range_always = 1;
+  } else {                       // as the forward pass: chosen in [8, -n_range - 100] when there is plenty of work
+    sh.n_range_lo = kFwdRange; sh.n_range_hi = -n_range - 100;
+  }
   sh.n_fastest = n_fastest;
   sh.m_group = m_group;
   sh.stream_k = stream_k;

@@ -120,6 +120,8 @@ def test_tile_schedules_cover_every_tile_once():
         _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_range=0)
         _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_range=int(rng.integers(1, 9)),
                         m_group=int(rng.integers(1, 40)))
+        _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_range=-8, m_group=int(rng.integers(0, 40)))
+        _check_schedule(n_valid, 32768, k_len, 8 * n_tiles, cg, workers, n_range=-112, m_group=int(rng.integers(0, 40)))
         _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_fastest=1, k_split_max=int(rng.integers(2, 5)))
         u = _check_schedule(n_valid, 32768, k_len, n_tiles, cg, workers, n_fastest=1, stream_k=1)
         parts = {}
@@ -132,6 +134,17 @@ def test_tile_schedules_cover_every_tile_once():
     for worker, mu, c0, c1, ks, kb0, kb1, kpt in u:
         work[worker] += kb1 - kb0
     assert work.max() - work.min() <= 1 and work.sum() == 66 * 8 * 296
+    # range lengths chosen on the device.  Gradient-of-the-logits pass of the benchmark (66 row tiles, 148 column
+    # tiles per slab, 74 pairs): ranges of 4 tiles = 33 waves of equal units; 7B-class head (88 row tiles): the same.
+    # A pass asked to choose in [8, 12] with plenty of work (594 column tiles): 9 tiles per unit (66 ranges x 66 row
+    # tiles = 58.9 waves) rather than 8.
+    for rows, tiles, nr_arg, expect in [(16896, 148, -8, 4), (22528, 148, -8, 4), (16896, 594, -112, 9),
+                                        (16896, 2, -8, 2), (300, 148, -8, 4)]:
+        u = _check_schedule(rows, 32768, 2048, tiles, 2, 74, n_range=nr_arg, m_group=36)
+        assert max(r[3] - r[2] for r in u) == expect, (rows, tiles, expect, max(r[3] - r[2] for r in u))
+    # a forward pass with few rows keeps the split that fills the machine (at most 16 ranges per row tile)
+    u = _check_schedule(300, 32768, 2048, 594, 2, 74, n_range=-112)
+    assert len({(r[2], r[3]) for r in u}) <= 16
     # the same pass on 256 x 512 tiles (the tile counter then counts 512-wide tiles: d = 2048 -> 4, 2560 -> 5,
     # 3584 -> 7): 264 tiles on 74 pairs are 3.57 waves; stream-K evens them out, K slices cover every k-block
     for d_tiles, n_valid in ((4, 16896), (5, 32768), (7, 32768), (4, 300), (7, 20001)):
