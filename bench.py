@@ -319,11 +319,13 @@ SEED_STRESS = 251221450 + 99
 def run_reduced_case(args):
     """A reduced copy of the bench workload for profiler captures: same d and distributions, 37888 vocabulary
     rows (W = 155 MB, larger than L2), two prompts (about 4.6 K valid rows), a few steps, nothing timed.
-    One step launches the forward pass and, per 37888-column slab, the dlogits, dH and dW passes."""
+    The gradient slab is limited to 18944 columns here, so that one step launches the forward pass and, for each
+    of two vocabulary slabs, the dlogits, dH and dW passes: seven tensor-core launches per step."""
     import torch
     from paper_2512_21450_b200 import Context
     from paper_2512_21450_b200.workloads import make_workload
     ctx = Context(0)
+    ctx.set_slab_limits(0, 18944)
     w = make_workload(args.config, V=37888, prompts=2)
     dH = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
     dW = torch.empty(w.V, w.d, dtype=torch.float32, device="cuda")
