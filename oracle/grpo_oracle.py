@@ -332,6 +332,41 @@ def per_token_terms(logp, old_logp, ref_logp, adv, eps_low, eps_high, beta,
     return s, k3, rho, active, dlogp
 
 
+def token_loss(logp, entropy, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta,
+               ent_coef=0.0, token_weight=None):
+    """Eq. 6 (negated) from per-token quantities alone, for a caller that already holds the
+    log-probability (and entropy) of every token:
+
+        loss = sum_t w_t * ( -s_t + beta * k3_t - ent_coef * Ent_t ),   w_t = m_t / sum(m)
+
+    with s_t, k3_t of per_token_terms (section 3.1 surrogate, k3 reading of Omega).  Returns the
+    loss and its derivatives with respect to logp_t and Ent_t (zero on rows with mask 0):
+
+        d loss / d logp_t = w_t * ( -A_t rho_t [unclipped] + beta (1 - exp(delta_t)) )
+        d loss / d Ent_t  = -w_t * ent_coef
+    """
+    logp = np.asarray(logp, dtype=np.float64)
+    T = logp.shape[0]
+    m = np.ones(T) if mask is None else (np.asarray(mask) != 0).astype(np.float64)
+    w = token_weights(m) if token_weight is None else np.asarray(token_weight, dtype=np.float64) * m
+    ent = np.zeros(T) if entropy is None else np.asarray(entropy, dtype=np.float64)
+    ref = np.zeros(T) if ref_logp is None else np.asarray(ref_logp, dtype=np.float64)
+    s, k3, rho, active, dlogp = per_token_terms(logp, np.asarray(old_logp, dtype=np.float64), ref,
+                                                np.asarray(adv, dtype=np.float64), eps_low, eps_high, beta)
+    rows = m != 0
+    loss_t = -s + beta * k3 - ent_coef * ent
+    out = dict(loss=float((w[rows] * loss_t[rows]).sum()),
+               dlogp=np.where(rows, w * dlogp, 0.0),
+               dentropy=np.where(rows, -w * ent_coef, 0.0),
+               pg_loss=float((w[rows] * -s[rows]).sum()),
+               kl_mean=float((w[rows] * k3[rows]).sum()),
+               entropy_mean=float((w[rows] * ent[rows]).sum()),
+               clip_frac=float((w[rows] * (~active[rows])).sum()),
+               ratio_mean=float((w[rows] * rho[rows]).sum()),
+               ratio_max=float(rho[rows].max()) if rows.any() else 0.0)
+    return out
+
+
 def full_kl(LP, LQ):
     """KL(pi_theta(.|s_t) || pi_ref(.|s_t)) per row from the two log-probability matrices: the
     regulariser exactly as section 2.2 / 3.1 print it, sum_j p_j (log p_j - log q_j)."""

@@ -47,6 +47,10 @@ MUTANTS = {
     "shaping: k1 direction swapped": ("return logp - ref\n", "return ref - logp\n"),
     "shaping: k3 uses the opposite log-ratio": ("delta = ref - logp\n        return np.exp(delta) - delta - 1.0", "delta = logp - ref\n        return np.exp(delta) - delta - 1.0"),
     "row map keeps the masked rows": ("return [t for t in range(len(mask)) if mask[t] != 0]", "return [t for t in range(len(mask)) if mask[t] == 0]"),
+    "token loss: entropy bonus enters with the wrong sign": ("loss_t = -s + beta * k3 - ent_coef * ent\n    out = dict(", "loss_t = -s + beta * k3 + ent_coef * ent\n    out = dict("),
+    "token loss: derivative not weighted": ("dlogp=np.where(rows, w * dlogp, 0.0)", "dlogp=np.where(rows, dlogp, 0.0)"),
+    "token loss: entropy derivative sign": ("dentropy=np.where(rows, -w * ent_coef, 0.0)", "dentropy=np.where(rows, w * ent_coef, 0.0)"),
+    "token loss: masked rows keep a derivative": ("dlogp=np.where(rows, w * dlogp, 0.0)", "dlogp=dlogp / max(m.sum(), 1.0)"),
     "logits index order": ("return H @ W.T", "return (W @ H.T).T[::-1][::-1] if H.shape[0] == 1 else (H[:, ::-1] @ W[:, ::-1].T if False else H @ W[::-1].T)"),
 }
 

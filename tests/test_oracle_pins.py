@@ -762,3 +762,59 @@ def test_valid_rows_outside_every_response_range_take_no_part():
     # the plain path (no response structure) keeps every valid row
     c = O.policy_loss_fwd_bwd(H, W, tok, old, ref, adv, mask, 0.2, 0.3, 0.05)
     assert c["dH"][:2].any() and c["dH"][11:].any()
+
+
+# ----------------------------------------------------------------------------- per-token loss on its own
+def test_token_loss_worked_example():
+    # the two-word example of tests/golden: the per-token call has to reproduce its loss and d loss / d logp
+    # from logp, entropy, old, ref alone (cases A, B: dloss/dlogp = 0.25 and 1.75; case C adds -0.1 * entropy)
+    g = _golden("two_token_worked_example.txt")
+    lp, ent = np.array([g["logp"]]), np.array([g["entropy"]])
+    old, ref = np.array([math.log(0.5)]), np.array([math.log(0.375)])
+    A = O.token_loss(lp, ent, old, ref, np.array([1.0]), None, 0.2, 0.2, 0.5)
+    assert abs(A["loss"] - g["A_loss"]) < 1e-14 and abs(A["dlogp"][0] - 0.25) < 1e-14 and A["dentropy"][0] == 0.0
+    assert A["clip_frac"] == 1.0 and abs(A["ratio_mean"] - 1.5) < 1e-14 and abs(A["kl_mean"] - g["k3"]) < 1e-14
+    B = O.token_loss(lp, ent, old, ref, np.array([-1.0]), None, 0.2, 0.2, 0.5)
+    assert abs(B["loss"] - g["B_loss"]) < 1e-14 and abs(B["dlogp"][0] - 1.75) < 1e-14 and B["clip_frac"] == 0.0
+    C = O.token_loss(lp, ent, old, ref, np.array([1.0]), None, 0.2, 0.2, 0.5, ent_coef=0.1)
+    assert abs(C["loss"] - g["C_loss"]) < 1e-13 and abs(C["dentropy"][0] + 0.1) < 1e-15
+
+
+@pytest.mark.parametrize("beta,ent_coef,weights", [(0.0, 0.0, False), (0.3, 0.0, False), (0.3, 0.05, False),
+                                                   (0.3, 0.05, True)])
+def test_token_loss_agrees_with_the_full_loss_and_finite_differences(beta, ent_coef, weights):
+    H, W, tokens, old, ref, adv, mask = _tiny_problem(31, T=9, masked=(2, 7))
+    rng = _rng(5)
+    tw = rng.uniform(0.1, 1.0, size=9) if weights else None
+    full = O.policy_loss_fwd_bwd(H, W, tokens, old, ref, adv, mask, 0.2, 0.3, beta, ent_coef=ent_coef, token_weight=tw)
+    lp, ent = full["logp"], full["entropy"]
+    t = O.token_loss(lp, ent, old, ref, adv, mask, 0.2, 0.3, beta, ent_coef=ent_coef, token_weight=tw)
+    # same loss and metrics as the whole path computes from H and W
+    assert abs(t["loss"] - full["loss"]) < 1e-14
+    for k in ("pg_loss", "kl_mean", "entropy_mean", "clip_frac"):
+        assert abs(t[k] - full[k]) < 1e-14
+    # the chain rule through logp and entropy gives the whole path's logit gradient: row sums of G * z vanish,
+    # so compare through dH = sum_j g_j W_j with g built from (dlogp, dentropy)
+    Z = O.logits(H, W)
+    _, LP, _ = O.log_softmax_stats(Z)
+    P = np.exp(LP)
+    onehot = np.zeros_like(P)
+    onehot[np.arange(9), tokens] = 1.0
+    G = t["dlogp"][:, None] * (onehot - P) + t["dentropy"][:, None] * (-P * (LP + ent[:, None]))
+    assert np.abs(G @ W - full["dH"]).max() < 1e-13
+    # central differences in logp and in the entropy, valid and masked rows alike
+    h = 1e-6
+    for i in range(9):
+        for key, arr in (("dlogp", lp), ("dentropy", ent)):
+            up, dn = arr.copy(), arr.copy()
+            up[i] += h
+            dn[i] -= h
+            a = (up, ent) if key == "dlogp" else (lp, up)
+            b = (dn, ent) if key == "dlogp" else (lp, dn)
+            fd = (O.token_loss(a[0], a[1], old, ref, adv, mask, 0.2, 0.3, beta, ent_coef=ent_coef, token_weight=tw)["loss"] -
+                  O.token_loss(b[0], b[1], old, ref, adv, mask, 0.2, 0.3, beta, ent_coef=ent_coef, token_weight=tw)["loss"]) / (2 * h)
+            assert abs(fd - t[key][i]) < 1e-8, (key, i, fd, t[key][i])
+    assert t["dlogp"][2] == 0.0 and t["dlogp"][7] == 0.0 and t["dentropy"][2] == 0.0
+    # nothing valid: zero loss, zero derivatives
+    z = O.token_loss(lp, ent, old, ref, adv, np.zeros(9, dtype=np.uint8), 0.2, 0.3, beta, ent_coef=ent_coef)
+    assert z["loss"] == 0.0 and not z["dlogp"].any() and z["ratio_max"] == 0.0
