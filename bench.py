@@ -307,6 +307,25 @@ def run_small_kernel_stress(args):
     ms = timed(lambda: ctx.rl_kl_shaped_returns(value, lp, rf, mask, off512, T, 0.04, returns=ret, want_shaped=False))
     report("KL-shaped returns (k3, responses of 512 rows)", ms, 9 * T + 4 * T + 8 * n_resp,
            "two fp32 inputs + 1 B of mask read, returns written per row; offsets and per-response value read")
+    # the same call on rollouts of a realistic length: 2^17 responses of 512 rows (2^14 groups of 8)
+    n_resp8 = n_resp // G * G
+    rewards512 = (torch.rand(n_resp8, generator=g, device="cuda") < 0.4).float()
+    ms = timed(lambda: ctx.rl_grpo_advantages(rewards512, G, seq_offsets=off512[:n_resp8 + 1], T=T))
+    report("GRPO advantages + broadcast, responses of 512 rows", ms, 12 * n_resp8 + 4 * (n_resp8 + 1) + 4 * T,
+           "as above; the per-token array is nearly all of the traffic")
+    # per-token loss on its own: ratio, clip, k3, entropy bonus, token mean; both derivatives written
+    ent = torch.rand(T, generator=g, device="cuda") * 11.0
+    adv_tok = torch.randn(T, generator=g, device="cuda")
+    old = lp + 0.05 * torch.randn(T, generator=g, device="cuda")
+    outs = dict(loss=torch.empty(1, device="cuda"), dlogp=torch.empty(T, device="cuda"),
+                dentropy=torch.empty(T, device="cuda"), metrics=torch.empty(8, device="cuda"))
+    ms = timed(lambda: ctx.rl_token_loss(lp, ent, old, rf, adv_tok, mask, 0.2, 0.28, 0.04, ent_coef=1e-3, out=outs))
+    report("per-token loss (count, ratio / clip / k3 / entropy terms, reduction)", ms, (1 + 5 * 4 + 1 + 2 * 4) * T,
+           "mask read by the count pass; five fp32 inputs + mask read and two fp32 derivatives written per row")
+    ms = timed(lambda: ctx.rl_token_loss(lp, None, old, rf, adv_tok, mask, 0.2, 0.2, 0.04, want_grads=False,
+                                         out=dict(loss=outs["loss"], metrics=outs["metrics"])))
+    report("per-token loss, loss and metrics only (no entropy term)", ms, (1 + 4 * 4 + 1) * T,
+           "mask read by the count pass; four fp32 inputs + mask read per row, nothing written per row")
     status, _ = ctx.last_device_status()
     assert status == 0
     print(json.dumps({"small_kernel_stress": {"rows": T, "valid_rows": N, "groups": n_groups, "group_size": G,

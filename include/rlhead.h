@@ -197,6 +197,27 @@ rl_status rl_kl_shaped_returns(rl_ctx* ctx, const float* seq_value, const float*
                                int64_t n_seq, int64_t T, float beta, float gamma, int kl_estimate,
                                float* shaped_reward, float* returns);
 
+/* The per-token loss arithmetic on its own: Eq. 6 (negated) with the clipped importance-ratio surrogate of
+ * section 3.1 and the k3 estimate of the KL-to-reference term of section 2.2, from per-token quantities the
+ * caller already holds (for instance the merged output of the vocabulary-parallel calls, or log-probabilities
+ * scored by another engine):
+ *     rho_t = exp(logp_t - old_logp_t),   s_t = min(rho_t A_t, clip(rho_t, 1 - eps_low, 1 + eps_high) A_t),
+ *     delta_t = ref_logp_t - logp_t,      k3_t = exp(delta_t) - delta_t - 1,
+ *     loss = sum_t w_t (-s_t + beta k3_t - ent_coef Ent_t),
+ * w_t = token_weight[t] if given, else mask_t / (number of rows with mask != 0, or *token_count if given: the
+ * data-parallel global count, a device int64).  All arrays are device pointers of T floats in the original row
+ * order; mask[T] bytes or NULL (every row valid); entropy may be NULL when ent_coef == 0 (the entropy metric
+ * is then 0); ref_logp NULL iff beta == 0.  Outputs: loss[1]; dlogp[T] = d loss / d logp_t and dentropy[T] =
+ * d loss / d Ent_t = -w_t ent_coef (either may be NULL; rows with mask 0 get 0); metrics_out[8] or NULL, laid
+ * out as rl_loss_opts.metrics_out.  A count pass over the mask, one pass of four rows per thread (16-byte
+ * loads and stores when every array is 16-byte aligned) and a fixed-order reduction in double: reproducible.
+ * Needs no workspace (the context owns 64 KB for the block sums).  T == 0: loss 0, RL_OK.
+ * Errors: eps_low outside [0, 1), eps_high < 0, beta < 0, ent_coef < 0, NULL required pointer -> RL_ERR_INVALID_ARG. */
+rl_status rl_token_loss(rl_ctx* ctx, const float* logp, const float* entropy, const float* old_logp,
+                        const float* ref_logp, const float* adv, const uint8_t* mask, int64_t T, float eps_low,
+                        float eps_high, float beta, float ent_coef, const float* token_weight, const void* token_count,
+                        float* loss, float* dlogp, float* dentropy, float* metrics_out);
+
 /* Padding-free row map on its own (section 4.4, training without padding tokens): row_map[i] = index of
  * the i-th row with mask != 0, ascending, for i < *n_valid; entries past that are left untouched.
  * mask NULL = all rows valid.  row_map[T] (int32) and n_valid[1] (int32) are device pointers; the

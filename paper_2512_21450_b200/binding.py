@@ -128,6 +128,8 @@ def load_library():
     lib.rl_mask_scan.restype = c_int
     lib.rl_kl_shaped_returns.argtypes = [P, P, P, P, P, P, P, c_int64, c_int64, c_float, c_float, c_int, P, P]
     lib.rl_kl_shaped_returns.restype = c_int
+    lib.rl_token_loss.argtypes = [P, P, P, P, P, P, P, c_int64, c_float, c_float, c_float, c_float, P, P, P, P, P, P]
+    lib.rl_token_loss.restype = c_int
     lib.rl_token_logprobs_multi.argtypes = [P, c_int, POINTER(c_void_p), POINTER(c_int64), POINTER(c_void_p),
                                             POINTER(c_int64), POINTER(c_int64), P, P, c_int64, c_int64,
                                             POINTER(c_void_p), POINTER(c_void_p)]
@@ -371,6 +373,30 @@ class Context:
                                              self.KL_ESTIMATES[kind], _ptr(shaped), _ptr(returns)),
                "rl_kl_shaped_returns")
         return shaped, returns
+
+    def rl_token_loss(self, logp, entropy, old_logp, ref_logp, adv, mask, eps_low, eps_high, beta, ent_coef=0.0,
+                      token_weight=None, token_count=None, want_grads=True, want_metrics=True, out=None):
+        """The per-token loss arithmetic on its own, from log-probabilities (and entropies) the caller holds:
+        returns dict(loss [1], dlogp [T], dentropy [T], metrics [8]); `out` may carry preallocated tensors."""
+        self._bind_stream()
+        T = logp.numel()
+        for x in (logp, entropy, old_logp, ref_logp, adv, token_weight):
+            assert x is None or (x.dtype == torch.float32 and x.is_contiguous() and x.numel() == T)
+        assert mask is None or (mask.dtype == torch.uint8 and mask.numel() == T)
+        assert token_count is None or token_count.dtype == torch.int64
+        dev = logp.device
+        out = dict(out or {})
+        out.setdefault("loss", torch.empty(1, dtype=torch.float32, device=dev))
+        if want_grads:
+            out.setdefault("dlogp", torch.empty(T, dtype=torch.float32, device=dev))
+            out.setdefault("dentropy", torch.empty(T, dtype=torch.float32, device=dev))
+        if want_metrics:
+            out.setdefault("metrics", torch.empty(8, dtype=torch.float32, device=dev))
+        _check(self.lib.rl_token_loss(self.handle, _ptr(logp), _ptr(entropy), _ptr(old_logp), _ptr(ref_logp), _ptr(adv),
+                                      _ptr(mask), T, eps_low, eps_high, beta, ent_coef, _ptr(token_weight),
+                                      _ptr(token_count), _ptr(out["loss"]), _ptr(out.get("dlogp")),
+                                      _ptr(out.get("dentropy")), _ptr(out.get("metrics"))), "rl_token_loss")
+        return out
 
     def rl_mask_scan(self, mask, T=None, row_map=None, n_valid=None):
         """Row map of the valid rows: returns (row_map [T] int32, n_valid [1] int32), both on the device."""

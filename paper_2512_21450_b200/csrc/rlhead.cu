@@ -59,6 +59,12 @@ namespace {
 
 constexpr long long kRowGroupBytes = 36ll << 20;   // A panels walked together by the rows-first passes (L2 is 126 MB)
 constexpr int kSlabRowsMax = 32768;        // rows of one gradient slab
+// Device words a context owns besides the workspace: the status record, a few scalars of the small kernels
+// (byte 64: batch statistics, 96: longest response, 128: valid-row count of rl_token_loss) and, from byte 256 on,
+// the block partials of rl_token_loss.
+constexpr int kTokenLossBlocks = 1024;
+constexpr size_t kStatusBytes = 256 + (size_t)kTokenLossBlocks * kLossSums * sizeof(double);
+constexpr int kAdvRowsMinGroups = 2048;     // from this many groups on, GRPO advantages run one thread per group
 constexpr int kDhSplitMax = 4;             // most K slices (separate fp32 accumulators) of the dH pass
 constexpr int kSlabColsMax = 148 * 256;    // vocabulary columns of one gradient slab (148 tiles of 256: two per SM pair)
 
@@ -463,8 +469,8 @@ rl_status rl_create(rl_ctx** out, int device) {
   }
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
   // device block: status word, then two doubles for batch statistics
-  if (cudaMalloc(&c->dstatus, 256) != cudaSuccess) { delete c; return RL_ERR_CUDA; }
-  cudaMemset(c->dstatus, 0, 256);
+  if (cudaMalloc(&c->dstatus, kStatusBytes) != cudaSuccess) { delete c; return RL_ERR_CUDA; }
+  cudaMemset(c->dstatus, 0, kStatusBytes);
   bool ok = set_smem_attr<EpiStats, 0, 0>() == cudaSuccess && set_smem_attr<EpiGrad, 0, 0>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 0, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 0, 1>() == cudaSuccess &&
             set_smem_attr<EpiAcc, 1, 0>() == cudaSuccess && set_smem_attr<EpiAcc, 1, 1>() == cudaSuccess &&
@@ -691,8 +697,27 @@ rl_status rl_grpo_advantages_ex(rl_ctx* c, const float* rewards, int64_t n_seq, 
   while (seg > 1 && (seg >> 1) >= group_size) seg >>= 1;
   const int groups_per_block = warps * (32 / seg);
   const int pr_adv = prof_begin(c, 8);
-  grpo_adv_kernel<<<(n_groups + groups_per_block - 1) / groups_per_block, warps * 32, 0, c->stream>>>(
-      rewards, n_groups, group_size, ddof, eps_std, adv_seq);
+  // many groups of 4, 8, ... 32 responses in 16-byte aligned arrays: one thread per group; else shuffle segments
+  const bool rows_path = n_groups >= kAdvRowsMinGroups && group_size % 4 == 0 && group_size <= 32 &&
+                         ((reinterpret_cast<uintptr_t>(rewards) | reinterpret_cast<uintptr_t>(adv_seq)) & 15) == 0;
+  if (rows_path) {
+    const int blocks = (n_groups + 255) / 256;
+    const float4* r4 = reinterpret_cast<const float4*>(rewards);
+    float4* a4 = reinterpret_cast<float4*>(adv_seq);
+    switch (group_size / 4) {
+      case 1: grpo_adv_rows_kernel<1><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+      case 2: grpo_adv_rows_kernel<2><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+      case 3: grpo_adv_rows_kernel<3><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+      case 4: grpo_adv_rows_kernel<4><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+      case 5: grpo_adv_rows_kernel<5><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+      case 6: grpo_adv_rows_kernel<6><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+      case 7: grpo_adv_rows_kernel<7><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+      default: grpo_adv_rows_kernel<8><<<blocks, 256, 0, c->stream>>>(r4, n_groups, ddof, eps_std, a4); break;
+    }
+  } else {
+    grpo_adv_kernel<<<(n_groups + groups_per_block - 1) / groups_per_block, warps * 32, 0, c->stream>>>(
+        rewards, n_groups, group_size, ddof, eps_std, adv_seq);
+  }
   c->launches++;
   if (adv_tok) {
     if (T > 0) {
@@ -732,6 +757,59 @@ rl_status rl_advantages(rl_ctx* c, int estimator, const float* rewards, const in
     c->launches += 2;
   }
   prof_end(c, pr, 8);
+  return cuda_ok();
+}
+
+rl_status rl_token_loss(rl_ctx* c, const float* logp, const float* entropy, const float* old_logp,
+                        const float* ref_logp, const float* adv, const uint8_t* mask, int64_t T, float eps_low,
+                        float eps_high, float beta, float ent_coef, const float* token_weight, const void* token_count,
+                        float* loss, float* dlogp, float* dentropy, float* metrics_out) {
+  if (!c || T < 0 || !loss) return RL_ERR_INVALID_ARG;
+  if (!(eps_low >= 0.f && eps_low < 1.f) || !(eps_high >= 0.f) || !(beta >= 0.f) || !(ent_coef >= 0.f))
+    return RL_ERR_INVALID_ARG;
+  if (T > 0 && (!logp || !old_logp || !adv)) return RL_ERR_INVALID_ARG;
+  if (T > 0 && beta != 0.f && !ref_logp) return RL_ERR_INVALID_ARG;
+  if (T > 0 && ent_coef != 0.f && !entropy) return RL_ERR_INVALID_ARG;
+  cudaStream_t st = c->stream;
+  if (T == 0) {
+    cudaMemsetAsync(loss, 0, 4, st);
+    if (metrics_out) cudaMemsetAsync(metrics_out, 0, 32, st);
+    return cuda_ok();
+  }
+  char* base = reinterpret_cast<char*>(c->dstatus);
+  unsigned long long* count = reinterpret_cast<unsigned long long*>(base + 128);
+  double* block_sums = reinterpret_cast<double*>(base + 256);
+  const int pr = prof_begin(c, 6);
+  if (mask) {
+    cudaMemsetAsync(count, 0, 8, st);
+    long long cb = (T / 16 + 255) / 256 + 1;
+    if (cb > (long long)c->n_sm * 8) cb = (long long)c->n_sm * 8;
+    count_valid_kernel<<<(int)cb, 256, 0, st>>>(mask, (long long)T, count);
+    c->launches++;
+  }
+  TokenLossParams p;
+  memset(&p, 0, sizeof(p));
+  p.logp = logp; p.entropy = entropy; p.old_logp = old_logp; p.ref_logp = beta != 0.f ? ref_logp : nullptr;
+  p.adv = adv; p.mask = mask; p.token_weight = token_weight;
+  p.count = token_count ? reinterpret_cast<const unsigned long long*>(token_count) : (mask ? count : nullptr);
+  p.n_known = (unsigned long long)T;
+  p.T = (long long)T;
+  p.eps_low = eps_low; p.eps_high = eps_high; p.beta = beta; p.ent_coef = ent_coef;
+  p.dlogp = dlogp; p.dentropy = dentropy; p.block_sums = block_sums;
+  long long blocks = ((T + 3) / 4 + kLossThreads - 1) / kLossThreads;
+  if (blocks > kTokenLossBlocks) blocks = kTokenLossBlocks;
+  if (blocks > (long long)c->n_sm * 4) blocks = (long long)c->n_sm * 4;   // one wave: four blocks are resident per SM
+  uintptr_t all = reinterpret_cast<uintptr_t>(logp) | reinterpret_cast<uintptr_t>(old_logp) | reinterpret_cast<uintptr_t>(adv) |
+                  reinterpret_cast<uintptr_t>(entropy) | reinterpret_cast<uintptr_t>(p.ref_logp) |
+                  reinterpret_cast<uintptr_t>(token_weight) | reinterpret_cast<uintptr_t>(dlogp) |
+                  reinterpret_cast<uintptr_t>(dentropy);
+  const bool vec = (all & 15) == 0 && (reinterpret_cast<uintptr_t>(mask) & 3) == 0;
+  if (vec) token_loss_kernel<true><<<(int)blocks, kLossThreads, 0, st>>>(p);
+  else     token_loss_kernel<false><<<(int)blocks, kLossThreads, 0, st>>>(p);
+  finalize_token_loss_kernel<<<1, 32 * kLossSums, 0, st>>>(block_sums, (int)blocks, loss, metrics_out, mask ? count : nullptr,
+                                               (unsigned long long)T);
+  c->launches += 2;
+  prof_end(c, pr, 6);
   return cuda_ok();
 }
 
@@ -974,7 +1052,7 @@ static rl_status loss_fwd_bwd_impl(rl_ctx* c, const void* H, int64_t ldH, const 
     seq_loss_kernel<<<blocks, kLossThreads, 0, st>>>(q, c->dstatus);
     c->launches += 3;
   }
-  finalize_loss_kernel<<<1, 32, 0, st>>>(p.block_sums, blocks, loss, o.metrics_out, c->dstatus);
+  finalize_loss_kernel<<<1, 32 * kLossSums, 0, st>>>(p.block_sums, blocks, loss, o.metrics_out, c->dstatus);
   prof_end(c, pr_loss, 6);
   c->launches++;
 

@@ -214,6 +214,52 @@ __global__ void __launch_bounds__(256) grpo_adv_kernel(const float* __restrict__
     adv_seq[(size_t)g * G + i] = (mx == mn) ? 0.f : (float)(((double)r[i] - mu) * inv);
 }
 
+// The same arithmetic with one THREAD per group, for batches of many groups whose size is a multiple of four
+// (G = 4 * G4 <= 32): a thread reads its group as G4 16-byte words (a warp reads 32 * G * 4 contiguous bytes), keeps
+// it in registers and needs no shuffles, so the double-precision mean / variance / square root / reciprocal are
+// paid once per group instead of once per lane of a segment.  At 2^20 groups of 8 this is what lets the kernel
+// run at memory speed; the shuffle kernel above serves small batches (one warp instruction covers 32 / seg groups,
+// which keeps the launch short when there are only a few groups) and every other group size.
+template <int G4>
+__global__ void __launch_bounds__(256) grpo_adv_rows_kernel(const float4* __restrict__ rewards, int n_groups, int ddof,
+                                                            float eps_std, float4* __restrict__ adv_seq) {
+  constexpr int G = 4 * G4;
+  const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= n_groups) return;
+  float x[G];
+#pragma unroll
+  for (int j = 0; j < G4; ++j) {
+    const float4 v = rewards[g * G4 + j];
+    x[4 * j] = v.x; x[4 * j + 1] = v.y; x[4 * j + 2] = v.z; x[4 * j + 3] = v.w;
+  }
+  double sum = 0.0;
+  float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+#pragma unroll
+  for (int i = 0; i < G; ++i) {
+    sum += (double)x[i];
+    mx = fmaxf(mx, x[i]);
+    mn = fminf(mn, x[i]);
+  }
+  const double mu = sum / (double)G;
+  double ss = 0.0;
+#pragma unroll
+  for (int i = 0; i < G; ++i) {
+    const double c = (double)x[i] - mu;
+    ss = fma(c, c, ss);
+  }
+  const double sigma = sqrt(ss / (double)(G - ddof));
+  const double inv = (mx == mn) ? 0.0 : 1.0 / (sigma + (double)eps_std);
+#pragma unroll
+  for (int j = 0; j < G4; ++j) {
+    float4 o;
+    o.x = (mx == mn) ? 0.f : (float)(((double)x[4 * j] - mu) * inv);
+    o.y = (mx == mn) ? 0.f : (float)(((double)x[4 * j + 1] - mu) * inv);
+    o.z = (mx == mn) ? 0.f : (float)(((double)x[4 * j + 2] - mu) * inv);
+    o.w = (mx == mn) ? 0.f : (float)(((double)x[4 * j + 3] - mu) * inv);
+    adv_seq[g * G4 + j] = o;
+  }
+}
+
 // Other critic-free estimators named in section 4.2 (no formula printed there; readings):
 //   est 1 RLOO: A_i = r_i - mean of the other responses of the group
 //   est 2 OPO : A_i = r_i - sum_j(len_j r_j) / sum_j(len_j)          (length-weighted baseline)
@@ -499,6 +545,24 @@ struct LossParams {
 constexpr int kLossSums = 8;  // loss, pg, kl, ent, clip, ratio, ratio_max, unused
 constexpr int kLossThreads = 256;
 
+// Fixed-order sum of column k of the block partials by one warp: lane l adds blocks l, l + 32, ... in order, then a
+// butterfly over the lanes; the order depends on n_blocks alone, so the result is reproducible.
+__device__ __forceinline__ double reduce_block_sums(const double* __restrict__ block_sums, int n_blocks, int k) {
+  const int lane = threadIdx.x & 31;
+  double v = 0.0;
+  for (int b = lane; b < n_blocks; b += 32) {
+    const double u = block_sums[(size_t)b * kLossSums + k];
+    v = (k == 6) ? fmax(v, u) : v + u;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const double u = __shfl_xor_sync(0xffffffffu, v, o);
+    v = (k == 6) ? fmax(v, u) : v + u;
+  }
+  return v;
+}
+
+
 __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossParams p, DevStatus* st) {
   const int n = st->n_valid;
   const int n_ranges = p.ext_lse ? 0 : gemm_extents(p.fwd_shape, n, p.fwd_cg, p.fwd_workers).n_ranges;
@@ -605,6 +669,177 @@ __global__ void __launch_bounds__(kLossThreads) combine_loss_kernel(const LossPa
     double v = red[0][k];
     for (int w = 1; w < kLossThreads / 32; ++w) v = (k == 6) ? fmax(v, red[w][k]) : v + red[w][k];
     p.block_sums[(size_t)blockIdx.x * kLossSums + k] = v;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// The per-token loss arithmetic on its own (Eq. 6 with the clipped surrogate of section 3.1 and the k3
+// estimate of the KL term), for a caller that already holds the log-probability and entropy of every
+// token: works on the original rows, four consecutive rows per thread (16-byte loads and stores when
+// every array is 16-byte aligned), masked rows give zero derivatives.  Same arithmetic, in the same
+// order, as combine_loss_kernel applies to the statistics it has merged.
+__global__ void __launch_bounds__(256) count_valid_kernel(const uint8_t* __restrict__ mask, long long T,
+                                                          unsigned long long* __restrict__ count) {
+  unsigned int n = 0;
+  const bool vec = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
+  const long long n16 = vec ? T / 16 : 0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (long long)gridDim.x * blockDim.x) {
+    const uint4 m = reinterpret_cast<const uint4*>(mask)[i];
+    const unsigned int w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) n += ((w[k] >> (8 * b)) & 0xffu) != 0u;
+  }
+  for (long long t = n16 * 16 + (long long)blockIdx.x * blockDim.x + threadIdx.x; t < T;
+       t += (long long)gridDim.x * blockDim.x)
+    n += mask[t] != 0;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+  __shared__ unsigned int red[8];
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = n;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long tot = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+    if (tot) atomicAdd(count, tot);   // integer sum: the order of the blocks does not change it
+  }
+}
+
+struct TokenLossParams {
+  const float* logp;
+  const float* entropy;       // or NULL: taken as 0
+  const float* old_logp;
+  const float* ref_logp;      // or NULL (beta == 0)
+  const float* adv;
+  const uint8_t* mask;        // or NULL: every row valid
+  const float* token_weight;  // or NULL: token mean
+  const unsigned long long* count;   // divisor of the token mean (valid rows, or the caller's global count) ...
+  unsigned long long n_known;        // ... or, when count is NULL, the divisor itself
+  long long T;
+  float eps_low, eps_high, beta, ent_coef;
+  float* dlogp;               // or NULL
+  float* dentropy;            // or NULL
+  double* block_sums;         // [gridDim.x][kLossSums]
+};
+
+template <bool VEC>
+__global__ void __launch_bounds__(kLossThreads, 4) token_loss_kernel(const TokenLossParams p) {
+  double acc[kLossSums];
+#pragma unroll
+  for (int k = 0; k < kLossSums; ++k) acc[k] = 0.0;
+  const unsigned long long n_mean = p.count ? *p.count : p.n_known;
+  const float w_mean = n_mean > 0 ? (float)(1.0 / (double)n_mean) : 0.f;
+  const long long n4 = (p.T + 3) / 4;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += (long long)gridDim.x * blockDim.x) {
+    const long long t0 = q * 4;
+    const int nrow = (int)(p.T - t0 < 4 ? p.T - t0 : 4);
+    float lp[4], en[4], ol[4], rf[4], av[4], tw[4];
+    unsigned int mk[4];
+    if (VEC && nrow == 4) {
+      const float4 a = *reinterpret_cast<const float4*>(p.logp + t0);
+      const float4 b = *reinterpret_cast<const float4*>(p.old_logp + t0);
+      const float4 c = *reinterpret_cast<const float4*>(p.adv + t0);
+      lp[0] = a.x; lp[1] = a.y; lp[2] = a.z; lp[3] = a.w;
+      ol[0] = b.x; ol[1] = b.y; ol[2] = b.z; ol[3] = b.w;
+      av[0] = c.x; av[1] = c.y; av[2] = c.z; av[3] = c.w;
+      const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      const float4 e = p.entropy ? *reinterpret_cast<const float4*>(p.entropy + t0) : z;
+      const float4 r = p.ref_logp ? *reinterpret_cast<const float4*>(p.ref_logp + t0) : z;
+      const float4 w = p.token_weight ? *reinterpret_cast<const float4*>(p.token_weight + t0) : z;
+      en[0] = e.x; en[1] = e.y; en[2] = e.z; en[3] = e.w;
+      rf[0] = r.x; rf[1] = r.y; rf[2] = r.z; rf[3] = r.w;
+      tw[0] = w.x; tw[1] = w.y; tw[2] = w.z; tw[3] = w.w;
+      const unsigned int m4 = p.mask ? *reinterpret_cast<const unsigned int*>(p.mask + t0) : 0x01010101u;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) mk[i] = (m4 >> (8 * i)) & 0xffu;
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const bool in = i < nrow;
+        lp[i] = in ? p.logp[t0 + i] : 0.f;
+        ol[i] = in ? p.old_logp[t0 + i] : 0.f;
+        av[i] = in ? p.adv[t0 + i] : 0.f;
+        en[i] = (in && p.entropy) ? p.entropy[t0 + i] : 0.f;
+        rf[i] = (in && p.ref_logp) ? p.ref_logp[t0 + i] : 0.f;
+        tw[i] = (in && p.token_weight) ? p.token_weight[t0 + i] : 0.f;
+        mk[i] = in ? (p.mask ? p.mask[t0 + i] : 1u) : 0u;
+      }
+    }
+    float dl[4], de[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      dl[i] = 0.f;
+      de[i] = 0.f;
+      if (!mk[i]) continue;
+      const float w = p.token_weight ? tw[i] : w_mean;
+      const float rho = expf(lp[i] - ol[i]);
+      const float clipped = fminf(fmaxf(rho, 1.f - p.eps_low), 1.f + p.eps_high);
+      const float su = rho * av[i], sc = clipped * av[i];
+      const bool active = su <= sc;          // unclipped branch is the minimum (ties: unclipped)
+      const float s = active ? su : sc;
+      float k3 = 0.f, dk3 = 0.f;
+      if (p.beta != 0.f) {
+        const float delta = rf[i] - lp[i];
+        const float ed = expf(delta);
+        k3 = ed - delta - 1.f;
+        dk3 = 1.f - ed;
+      }
+      const float dlogp = -(active ? av[i] * rho : 0.f) + p.beta * dk3;
+      dl[i] = w * dlogp;
+      de[i] = -(w * p.ent_coef);
+      acc[0] += (double)w * (double)(-s + p.beta * k3 - p.ent_coef * en[i]);
+      acc[1] += (double)w * (double)(-s);
+      acc[2] += (double)w * (double)k3;
+      acc[3] += (double)w * (double)en[i];
+      acc[4] += active ? 0.0 : (double)w;
+      acc[5] += (double)w * (double)rho;
+      acc[6] = fmax(acc[6], (double)rho);
+    }
+    if (VEC && nrow == 4) {
+      if (p.dlogp) *reinterpret_cast<float4*>(p.dlogp + t0) = make_float4(dl[0], dl[1], dl[2], dl[3]);
+      if (p.dentropy) *reinterpret_cast<float4*>(p.dentropy + t0) = make_float4(de[0], de[1], de[2], de[3]);
+    } else {
+      for (int i = 0; i < nrow; ++i) {
+        if (p.dlogp) p.dlogp[t0 + i] = dl[i];
+        if (p.dentropy) p.dentropy[t0 + i] = de[i];
+      }
+    }
+  }
+  __shared__ double red[kLossThreads / 32][kLossSums];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int k = 0; k < kLossSums; ++k) {
+    double v = acc[k];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double u = __shfl_xor_sync(0xffffffffu, v, o);
+      v = (k == 6) ? fmax(v, u) : v + u;
+    }
+    if (lane == 0) red[warp][k] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < kLossSums) {
+    const int k = threadIdx.x;
+    double v = red[0][k];
+    for (int w = 1; w < kLossThreads / 32; ++w) v = (k == 6) ? fmax(v, red[w][k]) : v + red[w][k];
+    p.block_sums[(size_t)blockIdx.x * kLossSums + k] = v;
+  }
+}
+
+// Fixed-order sum of the block partials of token_loss_kernel -> loss[1], metrics[8].  One warp per sum.
+__global__ void __launch_bounds__(32 * kLossSums) finalize_token_loss_kernel(const double* __restrict__ block_sums,
+                                                                             int n_blocks, float* __restrict__ loss,
+                                                                             float* __restrict__ metrics,
+                                                                             const unsigned long long* __restrict__ count,
+                                                                             unsigned long long n_rows_valid_known) {
+  const int k = threadIdx.x >> 5;
+  const double v = reduce_block_sums(block_sums, n_blocks, k);
+  if ((threadIdx.x & 31) != 0) return;
+  if (k == 0) loss[0] = (float)v;
+  if (metrics) {
+    if (k >= 1 && k <= 6) metrics[k - 1] = (float)v;
+    if (k == 7) { metrics[6] = (float)(count ? *count : n_rows_valid_known); metrics[7] = 0.f; }
   }
 }
 
@@ -747,17 +982,13 @@ __global__ void __launch_bounds__(kLossThreads) seq_loss_kernel(const SeqParams 
   }
 }
 
-// Second stage: fixed-order sum of the block partials -> loss[1] and metrics[8].
-__global__ void __launch_bounds__(32) finalize_loss_kernel(const double* __restrict__ block_sums, int n_blocks,
-                                                           float* __restrict__ loss, float* __restrict__ metrics,
-                                                           const DevStatus* st) {
-  const int k = threadIdx.x;
-  if (k >= kLossSums) return;
-  double v = 0.0;
-  for (int b = 0; b < n_blocks; ++b) {
-    const double u = block_sums[(size_t)b * kLossSums + k];
-    v = (k == 6) ? fmax(v, u) : v + u;
-  }
+// Second stage: fixed-order sum of the block partials -> loss[1] and metrics[8].  One warp per sum.
+__global__ void __launch_bounds__(32 * kLossSums) finalize_loss_kernel(const double* __restrict__ block_sums, int n_blocks,
+                                                                       float* __restrict__ loss, float* __restrict__ metrics,
+                                                                       const DevStatus* st) {
+  const int k = threadIdx.x >> 5;
+  const double v = reduce_block_sums(block_sums, n_blocks, k);
+  if ((threadIdx.x & 31) != 0) return;
   if (k == 0) loss[0] = (float)v;
   if (metrics) {
     if (k >= 1 && k <= 6) metrics[k - 1] = (float)v;

@@ -211,8 +211,10 @@ def test_mask_scan_row_map_is_exact(ctx, T):
     _assert_status_ok(ctx)
 
 
+# from 2048 groups of 4, 8, ... 32 responses on, the library runs one thread per group instead of shuffle segments
 @pytest.mark.parametrize("n_groups,G", [(4, 4), (8, 8), (64, 16), (7, 5), (3, 40), (1024, 8), (9, 2), (5, 32), (3, 33),
-                                        (100, 3)])
+                                        (100, 3), (2048, 8), (5000, 4), (3001, 12), (2500, 16), (2049, 28), (2048, 32),
+                                        (4000, 6), (2047, 8)])
 def test_advantages(ctx, n_groups, G):
     rng = np.random.default_rng(100 + G)
     for kind in ("bernoulli", "uniform", "zero_var"):
