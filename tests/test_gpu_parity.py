@@ -233,7 +233,9 @@ def test_advantages(ctx, n_groups, G):
                 assert not _np64(a).any()
 
 
-@pytest.mark.parametrize("case", ["long", "short", "ragged", "empty_ranges", "inner_span", "one_row"])
+# the big_* cases have more than 2^20 rows: several 8192-row block shares per block, searches that span many responses
+@pytest.mark.parametrize("case", ["long", "short", "ragged", "empty_ranges", "inner_span", "one_row",
+                                  "big_long", "big_short", "big_tiny", "big_ragged", "big_empty_inner", "big_one"])
 def test_advantage_broadcast_is_exact(ctx, case):
     # a copy: every row must carry exactly its response's value, rows outside the span of the ranges 0
     rng = np.random.default_rng(sum(map(ord, case)))
@@ -251,11 +253,29 @@ def test_advantage_broadcast_is_exact(ctx, case):
         lens[700] = 5
     elif case == "inner_span":
         lens = rng.integers(10, 2000, size=64)
+    elif case == "big_long":
+        lens = rng.integers(64, 4097, size=1024)            # about 2.1 M rows, a few responses per 8192-row block share
+    elif case == "big_short":
+        lens = rng.integers(1, 17, size=160000)             # about 1.4 M rows, a thousand responses per block share
+    elif case == "big_tiny":
+        lens = np.concatenate([np.ones(40000, dtype=np.int64), rng.integers(0, 3, size=600000),
+                               rng.integers(2000, 9000, size=100)])   # thousands of responses per 8192-row block share
+    elif case == "big_ragged":
+        lens = np.concatenate([rng.integers(1, 5, size=3000), rng.integers(20000, 90000, size=24)])
+        rng.shuffle(lens)
+    elif case == "big_empty_inner":
+        lens = rng.integers(100, 3000, size=900) * (rng.uniform(size=900) < 0.8)
+        lens[:50] = 0                                       # the span starts with empty ranges, inside a block share
+    elif case == "big_one":
+        lens = np.array([1 << 20, 1, 0, 5], dtype=np.int64)
     else:
         lens = np.ones(4, dtype=np.int64)
-    first = 1237 if case == "inner_span" else 0
+    inner = case in ("inner_span", "big_empty_inner", "big_ragged")
+    first = 1237 if inner else 0
     off = np.concatenate([[first], first + np.cumsum(lens)]).astype(np.int32)
-    T = int(off[-1]) + (4321 if case == "inner_span" else 0)
+    T = int(off[-1]) + (4321 if inner else 0)
+    if case.startswith("big"):
+        T = max(T, (1 << 20) + 13)
     if case == "ragged":
         T += 3                                              # rows past the last range, T not a multiple of 4
     n_seq = len(lens)
